@@ -1,0 +1,170 @@
+"""ctypes front end of the CPU oracle (``ilre_oracle.c``).  TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the bench's CPU-baseline leg may import this package.
+It builds the C file with gcc on first use and never touches the CUDA library.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ilre_oracle.c")
+_LIB = os.path.join(_HERE, "_build", "libilre_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle (gcc, -O2, OpenMP).  Returns the path of the shared object."""
+    os.makedirs(os.path.dirname(_LIB), exist_ok=True)
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".{os.getpid()}.tmp"
+        subprocess.check_call(["gcc", "-O2", "-std=c99", "-fopenmp", "-fPIC", "-shared",
+                               "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        c_i32p = ctypes.POINTER(ctypes.c_int32)
+        c_i64p = ctypes.POINTER(ctypes.c_int64)
+        c_u16p = ctypes.POINTER(ctypes.c_uint16)
+        c_f64p = ctypes.POINTER(ctypes.c_double)
+        lib.ilre_oracle_row_stats.argtypes = [c_u16p, ctypes.c_int64, ctypes.c_int, c_u16p,
+                                              ctypes.c_int, ctypes.c_int, ctypes.c_int, c_i32p,
+                                              ctypes.c_int, c_f64p, c_f64p]
+        lib.ilre_oracle_scores_at.argtypes = [c_u16p, ctypes.c_int64, ctypes.c_int, c_u16p,
+                                              ctypes.c_int, ctypes.c_int, ctypes.c_int, c_f64p,
+                                              c_f64p, c_i64p, ctypes.c_int64, c_f64p]
+        lib.ilre_oracle_scores.argtypes = [c_u16p, ctypes.c_int64, ctypes.c_int, c_u16p,
+                                           ctypes.c_int, ctypes.c_int, ctypes.c_int, c_f64p,
+                                           c_f64p, c_f64p]
+        lib.ilre_oracle_maxpool.argtypes = [c_f64p, ctypes.c_int64, ctypes.c_int, c_f64p]
+        lib.ilre_oracle_maxpool.restype = ctypes.c_int64
+        lib.ilre_oracle_winpool.argtypes = [c_f64p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
+                                            c_f64p]
+        lib.ilre_oracle_winpool.restype = None
+        lib.ilre_oracle_allocate.argtypes = [c_f64p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
+                                             c_i32p, ctypes.c_int, c_i32p, ctypes.c_int,
+                                             ctypes.c_int, c_i32p, c_i32p, c_i32p, c_f64p, c_f64p]
+        _lib = lib
+    return _lib
+
+
+def _u16(x) -> np.ndarray:
+    """bf16 torch tensor (CPU) or uint16 array -> contiguous uint16 numpy array."""
+    if isinstance(x, np.ndarray):
+        assert x.dtype == np.uint16
+        return np.ascontiguousarray(x)
+    import torch
+    assert x.dtype == torch.bfloat16 and x.device.type == "cpu"
+    return x.contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def _p(a: np.ndarray, ty):
+    return a.ctypes.data_as(ctypes.POINTER(ty))
+
+
+def row_stats(K, Q, rows: Sequence[int]):
+    """(row_max, row_sum) of Eq. 4's softmax for rows given as i * n_q_heads + h."""
+    k, q = _u16(K), _u16(Q)
+    L, n_kv, d = k.shape
+    q_len, n_q, _ = q.shape
+    r = np.ascontiguousarray(np.asarray(rows, dtype=np.int32))
+    m = np.empty(len(r), dtype=np.float64)
+    z = np.empty(len(r), dtype=np.float64)
+    rc = _load().ilre_oracle_row_stats(_p(k, ctypes.c_uint16), L, n_kv, _p(q, ctypes.c_uint16),
+                                       q_len, n_q, d, _p(r, ctypes.c_int32), len(r),
+                                       _p(m, ctypes.c_double), _p(z, ctypes.c_double))
+    if rc != 0:
+        raise RuntimeError(f"ilre_oracle_row_stats failed: {rc}")
+    return m, z
+
+
+def scores_at(K, Q, row_max: np.ndarray, row_sum: np.ndarray, positions: Sequence[int]):
+    """Eq. 5 at chosen positions, given the statistics of all q_len * n_q_heads rows."""
+    k, q = _u16(K), _u16(Q)
+    L, n_kv, d = k.shape
+    q_len, n_q, _ = q.shape
+    pos = np.ascontiguousarray(np.asarray(positions, dtype=np.int64))
+    m = np.ascontiguousarray(row_max, dtype=np.float64)
+    z = np.ascontiguousarray(row_sum, dtype=np.float64)
+    assert m.size == q_len * n_q and z.size == q_len * n_q
+    a = np.empty(len(pos), dtype=np.float64)
+    rc = _load().ilre_oracle_scores_at(_p(k, ctypes.c_uint16), L, n_kv, _p(q, ctypes.c_uint16),
+                                       q_len, n_q, d, _p(m, ctypes.c_double),
+                                       _p(z, ctypes.c_double), _p(pos, ctypes.c_int64), len(pos),
+                                       _p(a, ctypes.c_double))
+    if rc != 0:
+        raise RuntimeError(f"ilre_oracle_scores_at failed: {rc}")
+    return a
+
+
+def scores(K, Q, with_stats: bool = False):
+    """A^C [L] of Eq. 4 + Eq. 5 (fp64); optionally also (row_max, row_sum)."""
+    k, q = _u16(K), _u16(Q)
+    L, n_kv, d = k.shape
+    q_len, n_q, _ = q.shape
+    a = np.empty(L, dtype=np.float64)
+    m = np.empty(q_len * n_q, dtype=np.float64)
+    z = np.empty(q_len * n_q, dtype=np.float64)
+    rc = _load().ilre_oracle_scores(_p(k, ctypes.c_uint16), L, n_kv, _p(q, ctypes.c_uint16),
+                                    q_len, n_q, d, _p(a, ctypes.c_double),
+                                    _p(m, ctypes.c_double), _p(z, ctypes.c_double))
+    if rc != 0:
+        raise RuntimeError(f"ilre_oracle_scores failed: {rc}")
+    return (a, m, z) if with_stats else a
+
+
+def maxpool(a: np.ndarray, m: int) -> np.ndarray:
+    a = np.ascontiguousarray(a, dtype=np.float64)
+    out = np.empty((len(a) + m - 1) // m, dtype=np.float64)
+    n = _load().ilre_oracle_maxpool(_p(a, ctypes.c_double), len(a), m, _p(out, ctypes.c_double))
+    assert n == len(out)
+    return out
+
+
+def winpool(p: np.ndarray, n: int, op: int) -> np.ndarray:
+    p = np.ascontiguousarray(p, dtype=np.float64)
+    out = np.empty(len(p), dtype=np.float64)
+    _load().ilre_oracle_winpool(_p(p, ctypes.c_double), len(p), n, op, _p(out, ctypes.c_double))
+    return out
+
+
+def allocate(A: np.ndarray, budget: int, max_sizes: Sequence[int], win_sizes: Sequence[int],
+             win_op: int, n_sink: int = 0, diagnostics: bool = False):
+    """Algorithm 1 on a score array: ascending positions [n_sink + budget] (int32)."""
+    a = np.ascontiguousarray(A, dtype=np.float64)
+    ms = np.ascontiguousarray(np.asarray(max_sizes, dtype=np.int32))
+    ws = np.ascontiguousarray(np.asarray(win_sizes, dtype=np.int32))
+    nc = len(ms) * len(ws)
+    out = np.empty(max(n_sink + budget, 1), dtype=np.int32)
+    quota = np.zeros(nc, dtype=np.int32)
+    taken = np.zeros(nc, dtype=np.int32)
+    last_v = np.zeros(nc, dtype=np.float64)
+    kth_v = np.zeros(nc, dtype=np.float64)
+    rc = _load().ilre_oracle_allocate(_p(a, ctypes.c_double), len(a), n_sink, budget,
+                                      _p(ms, ctypes.c_int32), len(ms), _p(ws, ctypes.c_int32),
+                                      len(ws), win_op, _p(out, ctypes.c_int32),
+                                      _p(quota, ctypes.c_int32), _p(taken, ctypes.c_int32),
+                                      _p(last_v, ctypes.c_double), _p(kth_v, ctypes.c_double))
+    if rc != 0:
+        raise RuntimeError(f"ilre_oracle_allocate failed: {rc}")
+    out = out[: n_sink + budget]
+    if diagnostics:
+        return out, dict(quota=quota, taken=taken, last_value=last_v, kth_value=kth_v)
+    return out
+
+
+def recall(K, Q, budget: int, max_sizes: Sequence[int], win_sizes: Sequence[int], win_op: int,
+           n_sink: int = 0):
+    """The whole path: (ascending indices, A^C)."""
+    a = scores(K, Q)
+    return allocate(a, budget, max_sizes, win_sizes, win_op, n_sink), a
