@@ -1,0 +1,146 @@
+/*
+ * ilre_recall.h -- C ABI of the B200 (sm_100a) implementation of ILRe's token-recall path.
+ *
+ * The path is the part of the paper's pipeline that runs once per request at the retrieval
+ * layer l_R (Section 3.3, bullets "Calculate A^C ..." and "Apply Algorithm 1 ..."):
+ *
+ *   Eq. 4   s[h,i,t] = q[i,h,:] . K[t, kv(h), :] / sqrt(d_h),  softmax over the L context keys
+ *   Eq. 5   A^C[t]   = max over all query heads h and query tokens i of that softmax
+ *   Alg. 1  "Context Allocation": strided max pooling (size = stride = m_i), stride-1
+ *           window pooling (size n_j), top-K_m per (m_i, n_j) combination, an even budget
+ *           split B_c over the combinations with de-duplication ("next-highest-ranked
+ *           candidate"), and an ascending sort of the chosen positions.
+ *
+ * All pointers whose name ends in _dev are device pointers on the handle's device; _host
+ * pointers are host pointers.  No torch or C++ types cross this boundary.  Every function
+ * returns ILRE_OK (0) or a negative ilre_status code; nothing is launched when argument
+ * validation fails.  The library never falls back to the CPU.
+ */
+#ifndef ILRE_RECALL_H_
+#define ILRE_RECALL_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ilre_recall ilre_recall_t;   /* opaque; owns workspace, events, nothing else */
+
+enum ilre_status {
+  ILRE_OK = 0,
+  ILRE_ERR_INVALID_ARG = -1,  /* null pointer, L < 1, q_len < 1, a pooling size < 1, ...    */
+  ILRE_ERR_UNSUPPORTED = -2,  /* head_dim != 128, n_q_heads % n_kv_heads != 0, not sm_100,  */
+                              /* reduce_op != 0                                              */
+  ILRE_ERR_CAPACITY = -3,     /* L, q_len, budget or #combinations above the create() caps  */
+  ILRE_ERR_BUDGET = -4,       /* budget > L - n_sink                                         */
+  ILRE_ERR_ALIGNMENT = -5,    /* key cache or query base address not 16-byte aligned         */
+  ILRE_ERR_CUDA = -6,         /* a CUDA runtime/driver call failed                           */
+  ILRE_ERR_DEVICE_WAIT = -7,  /* a bounded wait inside a kernel gave up (see _status)        */
+  ILRE_ERR_QUOTA = -8,        /* a combination ran out of candidates (cannot happen for valid */
+                              /* inputs; reported by _status)                                */
+  ILRE_ERR_NOMEM = -9         /* workspace allocation failed in create()                     */
+};
+
+/* Capacities fixed at create(); run() never allocates. */
+typedef struct {
+  int32_t n_kv_heads;        /* e.g. 8                                                       */
+  int32_t n_q_heads;         /* e.g. 32; query head h reads kv head h / (n_q/n_kv)           */
+  int32_t head_dim;          /* must be 128                                                  */
+  int64_t max_L;             /* largest context length, < 2^31 - 256                         */
+  int32_t max_q_len;         /* largest number of query tokens                               */
+  int32_t max_budget;        /* largest budget B, <= 16382                                   */
+  int32_t max_combinations;  /* largest N_M * N_A, e.g. 48                                   */
+  int32_t device;            /* CUDA device ordinal                                          */
+  int32_t host_staging;      /* != 0: also allocate device staging for ilre_recall_run_host  */
+} ilre_recall_config_t;
+
+/* Pooling spec of Algorithm 1.  The arrays are host memory, read before run() returns. */
+typedef struct {
+  int32_t n_max;             /* N_M */
+  const int32_t* max_sizes;  /* m_i: MaxPooling size == stride; {1} switches it off           */
+  int32_t n_win;             /* N_A */
+  const int32_t* win_sizes;  /* n_j: stride-1 window; covers cells [c - n/2, c - n/2 + n-1]  */
+  int32_t win_op;            /* 0 = average (Algorithm 1; zero padding, divisor n), 1 = max   */
+  int32_t reduce_op;         /* 0 = max over (head, query token) (Eq. 5); others reserved    */
+  int32_t n_sink;            /* S: leading positions always returned, excluded from pooling  */
+} ilre_pool_spec_t;
+
+/*
+ * Create a handle on cfg->device: allocates all device workspace (row statistics, packed
+ * query, scores, pooled arrays [max_combinations][max_L], candidate lists, bitmap, status).
+ * *out is set only on success.  The handle may be used from one host thread and one stream
+ * at a time.
+ */
+int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out);
+
+/*
+ * One recall (Eq. 4, Eq. 5, Algorithm 1), asynchronous on cuda_stream (a cudaStream_t passed
+ * as void*; NULL = default stream).  Does not synchronise.
+ *   k_cache_dev   bf16 [L][n_kv_heads][128], RoPE already applied, 16-byte aligned; read only
+ *   query_dev     bf16 [q_len][n_q_heads][128], 16-byte aligned; read only
+ *   budget        B, 0 <= B <= L - n_sink
+ *   out_idx_dev   int32 [n_sink + budget]: chosen context positions, ascending
+ *   out_scores_dev  optional fp32 [L]: A^C of Eq. 5 (NULL to skip)
+ * Ranking inside a combination is (pooled value descending, cell index ascending); K_m =
+ * B/m + 1 (+1 when L - n_sink is not a multiple of m), B_c = B/N_c with the remainder given
+ * to the first combinations in loop order (max sizes outer, window sizes inner).
+ */
+int ilre_recall_run(ilre_recall_t* h,
+                    const void* k_cache_dev, int64_t L,
+                    const void* query_dev, int32_t q_len,
+                    int32_t budget, const ilre_pool_spec_t* spec,
+                    int32_t* out_idx_dev, float* out_scores_dev,
+                    void* cuda_stream);
+
+/*
+ * Same computation from HOST buffers (handle created with host_staging != 0): copies the
+ * key cache and query to device staging, runs, copies the indices (and scores if asked)
+ * back, and synchronises the stream before returning.  For throughput the host buffers
+ * should be page-locked.
+ */
+int ilre_recall_run_host(ilre_recall_t* h,
+                         const void* k_cache_host, int64_t L,
+                         const void* query_host, int32_t q_len,
+                         int32_t budget, const ilre_pool_spec_t* spec,
+                         int32_t* out_idx_host, float* out_scores_host,
+                         void* cuda_stream);
+
+/*
+ * Row statistics of the last run (Eq. 4's softmax denominator): copies
+ * lse[i * n_q_heads + h] = log(sum_t exp(s[h,i,t])) (natural log, fp32) for the q_len rows
+ * of that run into out_lse_dev, asynchronously on cuda_stream.
+ */
+int ilre_recall_copy_row_lse(ilre_recall_t* h, float* out_lse_dev, int32_t q_len,
+                             void* cuda_stream);
+
+/*
+ * Device status word of the handle.  Synchronises the stream of the last run, then returns
+ * ILRE_OK, ILRE_ERR_DEVICE_WAIT or ILRE_ERR_QUOTA, and clears the word.
+ */
+int ilre_recall_status(ilre_recall_t* h);
+
+/*
+ * Stage timing.  With profiling on, run() records CUDA events between its stages on the
+ * caller's stream.  ilre_recall_stage_times synchronises on the last event and writes up to
+ * n entries (milliseconds) in this order:
+ *   0 prepare (query packing, clears)   1 row statistics (QK^T + online softmax)
+ *   2 statistics merge                  3 scores (QK^T + max over rows)
+ *   4 pooling                           5 top-K_m selection and ranking
+ *   6 allocation and ascending output
+ * Returns the number of entries written, or a negative status.
+ */
+int ilre_recall_set_profiling(ilre_recall_t* h, int32_t on);
+int ilre_recall_stage_times(ilre_recall_t* h, float* ms_host, int32_t n);
+
+/* Number of kernel launches issued by the last run(). */
+int ilre_recall_last_launch_count(ilre_recall_t* h);
+
+int ilre_recall_destroy(ilre_recall_t* h);
+
+const char* ilre_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ILRE_RECALL_H_ */

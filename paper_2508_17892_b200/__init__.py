@@ -1,0 +1,9 @@
+"""B200 (sm_100a) implementation of ILRe's token-recall path behind a C ABI.
+
+``IlreRecall`` wraps ``libilre_recall.so`` (built in-tree by ``paper_2508_17892_b200.build``).
+"""
+from .recall import (EXPORTED_SYMBOLS, LIB_PATH, STAGE_NAMES, IlreConfig, IlreError, IlrePoolSpec,
+                     IlreRecall, load_library, strerror)
+
+__all__ = ["EXPORTED_SYMBOLS", "LIB_PATH", "STAGE_NAMES", "IlreConfig", "IlreError",
+           "IlrePoolSpec", "IlreRecall", "load_library", "strerror"]

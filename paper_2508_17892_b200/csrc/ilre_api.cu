@@ -1,0 +1,456 @@
+// C ABI of the recall library: handle, argument validation, workspace, launch sequence.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdint>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "../../include/ilre_recall.h"
+#include "qk_kernels.cuh"
+#include "select_kernels.cuh"
+#include "sm100_ptx.cuh"
+
+using namespace ilre;
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+constexpr int kNumStages = 7;            // timed stages (see ilre_recall_stage_times)
+constexpr int kMaxSinkStaging = 65536;
+
+struct Geometry {
+  int group_size, n_rb, rb_rows, n_groups, cpg, n_tiles, stages;
+};
+
+}  // namespace
+
+struct ilre_recall {
+  ilre_recall_config_t cfg;
+  int n_sm;
+  EncodeTiledFn encode;
+  // workspace (device)
+  void* qp;
+  float* partial;
+  float* nlse2;
+  float* row_lse;
+  uint32_t* enc;
+  float* scores;
+  float* pooled;
+  uint32_t* hist;
+  unsigned long long* sel_prefix;
+  uint32_t* sel_krem;
+  uint32_t* sel_done;
+  uint32_t* sel_ticket;
+  unsigned long long* cand;
+  uint32_t* cand_count;
+  int* ranked;
+  uint32_t* bitmap;
+  int* status;
+  // optional staging for the host entry point
+  void* stage_k;
+  void* stage_q;
+  int* stage_idx;
+  // bookkeeping
+  cudaEvent_t ev[kNumStages + 1];
+  int profiling;
+  int have_times;
+  int last_launches;
+  int last_q_len;
+  cudaStream_t last_stream;
+  int cand_stride;
+};
+
+namespace {
+
+struct DeviceGuard {
+  int prev;
+  bool ok;
+  explicit DeviceGuard(int dev) : prev(-1), ok(false) {
+    if (cudaGetDevice(&prev) != cudaSuccess) return;
+    ok = (prev == dev) || (cudaSetDevice(dev) == cudaSuccess);
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+int rows_padded_bound(int group_size, int q_len) {
+  const long long rg = static_cast<long long>(group_size) * q_len;
+  const long long n_rb = (rg + kMaxRbRows - 1) / kMaxRbRows;
+  return static_cast<int>(rg + 128 * (n_rb + 1));
+}
+
+Geometry make_geometry(const ilre_recall_config_t& c, int n_sm, long long L, int q_len) {
+  Geometry g;
+  g.group_size = c.n_q_heads / c.n_kv_heads;
+  const int rg = g.group_size * q_len;
+  g.n_rb = (rg + kMaxRbRows - 1) / kMaxRbRows;
+  const int per = (rg + g.n_rb - 1) / g.n_rb;
+  g.rb_rows = ((per + 127) / 128) * 128;
+  g.n_groups = c.n_kv_heads * g.n_rb;
+  g.n_tiles = static_cast<int>((L + kTileKeys - 1) / kTileKeys);
+  g.cpg = n_sm / g.n_groups;
+  if (g.cpg < 1) g.cpg = 1;
+  if (g.cpg > g.n_tiles) g.cpg = g.n_tiles;
+  const long long fixed = static_cast<long long>(g.rb_rows) * 256 + kSmemTailBytes +
+                          static_cast<long long>(g.rb_rows) * 4;
+  g.stages = static_cast<int>((kMaxDynSmem - fixed) / kStageBytes);
+  if (g.stages > kMaxStages) g.stages = kMaxStages;
+  return g;
+}
+
+template <class T>
+bool dev_alloc(T** p, size_t count) {
+  *p = nullptr;
+  return cudaMalloc(reinterpret_cast<void**>(p), (count ? count : 1) * sizeof(T)) == cudaSuccess;
+}
+
+void free_all(ilre_recall* h) {
+  cudaFree(h->qp); cudaFree(h->partial); cudaFree(h->nlse2); cudaFree(h->row_lse);
+  cudaFree(h->enc); cudaFree(h->scores); cudaFree(h->pooled); cudaFree(h->hist);
+  cudaFree(h->sel_prefix); cudaFree(h->sel_krem); cudaFree(h->sel_done); cudaFree(h->sel_ticket);
+  cudaFree(h->cand); cudaFree(h->cand_count); cudaFree(h->ranked); cudaFree(h->bitmap);
+  cudaFree(h->status); cudaFree(h->stage_k); cudaFree(h->stage_q); cudaFree(h->stage_idx);
+  for (int i = 0; i <= kNumStages; ++i)
+    if (h->ev[i]) cudaEventDestroy(h->ev[i]);
+}
+
+bool encode_2d(EncodeTiledFn fn, CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows,
+               uint64_t row_pitch_bytes) {
+  const cuuint64_t gdim[2] = {inner, rows};
+  const cuuint64_t gstride[1] = {row_pitch_bytes};
+  const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(kTileKeys)};
+  const cuuint32_t estride[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box,
+            estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int validate_run(const ilre_recall* h, const void* k, long long L, const void* q, int q_len,
+                 int budget, const ilre_pool_spec_t* spec, const void* out_idx) {
+  if (!h || !k || !q || !spec || !out_idx) return ILRE_ERR_INVALID_ARG;
+  if (L < 1 || q_len < 1 || budget < 0) return ILRE_ERR_INVALID_ARG;
+  if (spec->n_max < 1 || spec->n_win < 1 || !spec->max_sizes || !spec->win_sizes)
+    return ILRE_ERR_INVALID_ARG;
+  if (spec->n_sink < 0 || spec->win_op < 0 || spec->win_op > 1) return ILRE_ERR_INVALID_ARG;
+  if (spec->reduce_op != 0) return ILRE_ERR_UNSUPPORTED;
+  for (int i = 0; i < spec->n_max; ++i) {
+    if (spec->max_sizes[i] < 1) return ILRE_ERR_INVALID_ARG;
+    if (spec->max_sizes[i] > kMaxMaxSize) return ILRE_ERR_UNSUPPORTED;
+  }
+  for (int j = 0; j < spec->n_win; ++j) {
+    if (spec->win_sizes[j] < 1) return ILRE_ERR_INVALID_ARG;
+    if (spec->win_sizes[j] > kMaxWin) return ILRE_ERR_UNSUPPORTED;
+  }
+  const long long n_comb = static_cast<long long>(spec->n_max) * spec->n_win;
+  if (L > h->cfg.max_L || q_len > h->cfg.max_q_len || budget > h->cfg.max_budget ||
+      n_comb > h->cfg.max_combinations)
+    return ILRE_ERR_CAPACITY;
+  if (spec->n_sink > L || budget > L - spec->n_sink) return ILRE_ERR_BUDGET;
+  if ((reinterpret_cast<uintptr_t>(k) & 15u) || (reinterpret_cast<uintptr_t>(q) & 15u))
+    return ILRE_ERR_ALIGNMENT;
+  return ILRE_OK;
+}
+
+#define ILRE_CUDA(expr)                                   \
+  do {                                                    \
+    if ((expr) != cudaSuccess) return ILRE_ERR_CUDA;      \
+  } while (0)
+
+}  // namespace
+
+extern "C" {
+
+int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out) {
+  if (!cfg || !out) return ILRE_ERR_INVALID_ARG;
+  if (cfg->n_kv_heads < 1 || cfg->n_q_heads < 1 || cfg->max_L < 1 || cfg->max_q_len < 1 ||
+      cfg->max_budget < 0 || cfg->max_combinations < 1 || cfg->device < 0)
+    return ILRE_ERR_INVALID_ARG;
+  if (cfg->head_dim != kHeadDim || cfg->n_q_heads % cfg->n_kv_heads != 0)
+    return ILRE_ERR_UNSUPPORTED;
+  if (cfg->max_L > 2147483647LL - 256 || cfg->max_budget > kMaxKm - 2 ||
+      cfg->max_combinations > kMaxCombos)
+    return ILRE_ERR_CAPACITY;
+  if (static_cast<long long>(cfg->n_q_heads / cfg->n_kv_heads) * cfg->max_q_len > (1 << 24))
+    return ILRE_ERR_CAPACITY;
+
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || cfg->device >= n_dev) return ILRE_ERR_CUDA;
+  DeviceGuard guard(cfg->device);
+  if (!guard.ok) return ILRE_ERR_CUDA;
+  cudaDeviceProp prop;
+  ILRE_CUDA(cudaGetDeviceProperties(&prop, cfg->device));
+  if (prop.major != 10) return ILRE_ERR_UNSUPPORTED;       // tcgen05 / TMEM kernels: sm_100 only
+
+  ilre_recall* h = new (std::nothrow) ilre_recall();
+  if (!h) return ILRE_ERR_NOMEM;
+  std::memset(h, 0, sizeof(*h));
+  h->cfg = *cfg;
+  h->n_sm = prop.multiProcessorCount;
+
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) !=
+          cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+    delete h;
+    return ILRE_ERR_CUDA;
+  }
+  h->encode = reinterpret_cast<EncodeTiledFn>(fn);
+
+  const int group_size = cfg->n_q_heads / cfg->n_kv_heads;
+  const size_t rows_pad = static_cast<size_t>(rows_padded_bound(group_size, cfg->max_q_len));
+  const size_t max_groups = static_cast<size_t>(cfg->n_kv_heads) *
+      ((static_cast<size_t>(group_size) * cfg->max_q_len + kMaxRbRows - 1) / kMaxRbRows);
+  const size_t max_items = max_groups > static_cast<size_t>(h->n_sm) ? max_groups : h->n_sm;
+  const size_t maxL = static_cast<size_t>(cfg->max_L);
+  const size_t ncomb = static_cast<size_t>(cfg->max_combinations);
+  h->cand_stride = cfg->max_budget + 2;
+
+  bool ok = true;
+  ok = ok && dev_alloc(reinterpret_cast<uint8_t**>(&h->qp), cfg->n_kv_heads * rows_pad * 256);
+  ok = ok && dev_alloc(&h->partial, max_items * kMaxRbRows * 2);
+  ok = ok && dev_alloc(&h->nlse2, cfg->n_kv_heads * rows_pad);
+  ok = ok && dev_alloc(&h->row_lse, static_cast<size_t>(cfg->max_q_len) * cfg->n_q_heads);
+  ok = ok && dev_alloc(&h->enc, maxL);
+  ok = ok && dev_alloc(&h->scores, maxL);
+  ok = ok && dev_alloc(&h->pooled, ncomb * maxL);
+  ok = ok && dev_alloc(&h->hist, ncomb * kHistBins);
+  ok = ok && dev_alloc(&h->sel_prefix, ncomb);
+  ok = ok && dev_alloc(&h->sel_krem, ncomb);
+  ok = ok && dev_alloc(&h->sel_done, ncomb);
+  ok = ok && dev_alloc(&h->sel_ticket, ncomb);
+  ok = ok && dev_alloc(&h->cand, ncomb * h->cand_stride);
+  ok = ok && dev_alloc(&h->cand_count, ncomb);
+  ok = ok && dev_alloc(&h->ranked, ncomb * h->cand_stride);
+  ok = ok && dev_alloc(&h->bitmap, (maxL + 31) / 32);
+  ok = ok && dev_alloc(&h->status, 1);
+  if (ok && cfg->host_staging) {
+    ok = ok && dev_alloc(reinterpret_cast<uint8_t**>(&h->stage_k), maxL * cfg->n_kv_heads * 256);
+    ok = ok && dev_alloc(reinterpret_cast<uint8_t**>(&h->stage_q),
+                         static_cast<size_t>(cfg->max_q_len) * cfg->n_q_heads * 256);
+    ok = ok && dev_alloc(&h->stage_idx, static_cast<size_t>(cfg->max_budget) + kMaxSinkStaging);
+  }
+  for (int i = 0; ok && i <= kNumStages; ++i) ok = (cudaEventCreate(&h->ev[i]) == cudaSuccess);
+  if (ok) ok = (cudaMemset(h->status, 0, sizeof(int)) == cudaSuccess);
+  if (ok) ok = (cudaDeviceSynchronize() == cudaSuccess);
+  if (!ok) {
+    cudaGetLastError();
+    free_all(h);
+    delete h;
+    return ILRE_ERR_NOMEM;
+  }
+  *out = h;
+  return ILRE_OK;
+}
+
+int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const void* query_dev,
+                    int32_t q_len, int32_t budget, const ilre_pool_spec_t* spec,
+                    int32_t* out_idx_dev, float* out_scores_dev, void* cuda_stream) {
+  const int v = validate_run(h, k_cache_dev, L, query_dev, q_len, budget, spec, out_idx_dev);
+  if (v != ILRE_OK) return v;
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return ILRE_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const Geometry g = make_geometry(h->cfg, h->n_sm, L, q_len);
+  if (g.stages < 2) return ILRE_ERR_UNSUPPORTED;
+
+  // combination table (Algorithm 1 loop order: max sizes outer, window sizes inner)
+  ComboTable tbl;
+  std::memset(&tbl, 0, sizeof(tbl));
+  const long long Lp = L - spec->n_sink;
+  int max_len = 0, max_km = 1;
+  tbl.n_comb = (budget > 0) ? spec->n_max * spec->n_win : 0;
+  for (int i = 0, c = 0; i < spec->n_max && tbl.n_comb; ++i)
+    for (int j = 0; j < spec->n_win; ++j, ++c) {
+      const int m = spec->max_sizes[i];
+      const long long len = (Lp + m - 1) / m;
+      long long km = budget / m + 1 + ((Lp % m) != 0 ? 1 : 0);
+      if (km > len) km = len;
+      tbl.m[c] = m;
+      tbl.n[c] = spec->win_sizes[j];
+      tbl.len[c] = static_cast<int>(len);
+      tbl.k_m[c] = static_cast<int>(km);
+      tbl.quota[c] = budget / tbl.n_comb + (c < budget % tbl.n_comb ? 1 : 0);
+      if (len > max_len) max_len = static_cast<int>(len);
+      if (km > max_km) max_km = static_cast<int>(km);
+    }
+
+  CUtensorMap map_k, map_q;
+  if (!encode_2d(h->encode, &map_k, k_cache_dev, static_cast<uint64_t>(h->cfg.n_kv_heads) * 128,
+                 static_cast<uint64_t>(L), static_cast<uint64_t>(h->cfg.n_kv_heads) * 256))
+    return ILRE_ERR_CUDA;
+  if (!encode_2d(h->encode, &map_q, h->qp, 128, static_cast<uint64_t>(g.n_groups) * g.rb_rows, 256))
+    return ILRE_ERR_CUDA;
+
+  QkParams qk;
+  qk.L = L; qk.n_tiles = g.n_tiles; qk.n_groups = g.n_groups; qk.n_rb = g.n_rb;
+  qk.rb_rows = g.rb_rows; qk.cpg = g.cpg; qk.stages = g.stages;
+  qk.c2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(kHeadDim)));
+  qk.partial = h->partial; qk.nlse2 = h->nlse2; qk.enc = h->enc; qk.status = h->status;
+
+  PrepParams pp;
+  std::memset(&pp, 0, sizeof(pp));
+  pp.n_kv = h->cfg.n_kv_heads; pp.n_q = h->cfg.n_q_heads; pp.group_size = g.group_size;
+  pp.q_len = q_len; pp.n_rb = g.n_rb; pp.rb_rows = g.rb_rows; pp.L = L; pp.n_sink = spec->n_sink;
+  pp.enc = h->enc; pp.bitmap = h->bitmap; pp.hist = h->hist; pp.hist_bins = kHistBins;
+  pp.n_comb = tbl.n_comb;
+  for (int c = 0; c < tbl.n_comb; ++c) pp.k_m[c] = tbl.k_m[c];
+  pp.sel_prefix = h->sel_prefix; pp.sel_krem = h->sel_krem; pp.sel_done = h->sel_done;
+  pp.sel_ticket = h->sel_ticket; pp.cand_count = h->cand_count;
+
+  MergeParams mp;
+  mp.n_groups = g.n_groups; mp.n_rb = g.n_rb; mp.rb_rows = g.rb_rows; mp.cpg = g.cpg;
+  mp.group_size = g.group_size; mp.q_len = q_len; mp.n_q = h->cfg.n_q_heads;
+  mp.partial = h->partial; mp.nlse2 = h->nlse2; mp.row_lse = h->row_lse;
+
+  SelectParams sp;
+  std::memset(&sp, 0, sizeof(sp));
+  sp.scores = h->scores; sp.L = L; sp.n_sink = spec->n_sink; sp.win_op = spec->win_op;
+  sp.pooled = h->pooled; sp.pooled_stride = h->cfg.max_L; sp.hist = h->hist;
+  sp.sel_prefix = h->sel_prefix; sp.sel_krem = h->sel_krem; sp.sel_done = h->sel_done;
+  sp.sel_ticket = h->sel_ticket; sp.cand = h->cand; sp.cand_stride = h->cand_stride;
+  sp.cand_count = h->cand_count; sp.ranked = h->ranked; sp.bitmap = h->bitmap;
+  sp.out_idx = out_idx_dev; sp.budget = budget; sp.status = h->status;
+
+  const bool prof = h->profiling != 0;
+  int launches = 0;
+  h->have_times = 0;
+  h->last_stream = st;
+  h->last_q_len = q_len;
+#define ILRE_MARK(i) do { if (prof) ILRE_CUDA(cudaEventRecord(h->ev[i], st)); } while (0)
+
+  ILRE_MARK(0);
+  ILRE_CUDA(launch_prepare(query_dev, h->qp, pp, h->n_sm, st)); ++launches;
+  ILRE_MARK(1);
+  ILRE_CUDA(launch_row_stats(map_k, map_q, qk, st)); ++launches;
+  ILRE_MARK(2);
+  ILRE_CUDA(launch_merge_stats(mp, st)); ++launches;
+  ILRE_MARK(3);
+  ILRE_CUDA(launch_scores(map_k, map_q, qk, st)); ++launches;
+  ILRE_CUDA(launch_finalize_scores(h->enc, h->scores, out_scores_dev, L, st)); ++launches;
+  ILRE_MARK(4);
+  if (tbl.n_comb > 0) {
+    ILRE_CUDA(launch_pool(tbl, sp, max_len, st)); ++launches;
+  }
+  ILRE_MARK(5);
+  if (tbl.n_comb > 0) {
+    for (int pass = 0; pass < kSelectPasses; ++pass) {
+      ILRE_CUDA(launch_select_pass(tbl, sp, max_len, pass, st)); ++launches;
+    }
+    ILRE_CUDA(launch_gather(tbl, sp, max_len, st)); ++launches;
+    ILRE_CUDA(launch_rank_sort(tbl, sp, max_km, st)); ++launches;
+  }
+  ILRE_MARK(6);
+  ILRE_CUDA(launch_allocate(tbl, sp, st)); ++launches;
+  ILRE_MARK(7);
+#undef ILRE_MARK
+  h->last_launches = launches;
+  h->have_times = prof ? 1 : 0;
+  return ILRE_OK;
+}
+
+int ilre_recall_run_host(ilre_recall_t* h, const void* k_cache_host, int64_t L,
+                         const void* query_host, int32_t q_len, int32_t budget,
+                         const ilre_pool_spec_t* spec, int32_t* out_idx_host,
+                         float* out_scores_host, void* cuda_stream) {
+  if (!h || !h->stage_k) return ILRE_ERR_INVALID_ARG;
+  const int v = validate_run(h, k_cache_host, L, query_host, q_len, budget, spec, out_idx_host);
+  if (v != ILRE_OK && v != ILRE_ERR_ALIGNMENT) return v;
+  if (spec->n_sink > kMaxSinkStaging) return ILRE_ERR_CAPACITY;
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return ILRE_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t k_bytes = static_cast<size_t>(L) * h->cfg.n_kv_heads * 256;
+  const size_t q_bytes = static_cast<size_t>(q_len) * h->cfg.n_q_heads * 256;
+  ILRE_CUDA(cudaMemcpyAsync(h->stage_k, k_cache_host, k_bytes, cudaMemcpyHostToDevice, st));
+  ILRE_CUDA(cudaMemcpyAsync(h->stage_q, query_host, q_bytes, cudaMemcpyHostToDevice, st));
+  const int rc = ilre_recall_run(h, h->stage_k, L, h->stage_q, q_len, budget, spec, h->stage_idx,
+                                 nullptr, st);
+  if (rc != ILRE_OK) return rc;
+  ILRE_CUDA(cudaMemcpyAsync(out_idx_host, h->stage_idx,
+                            static_cast<size_t>(spec->n_sink + budget) * sizeof(int32_t),
+                            cudaMemcpyDeviceToHost, st));
+  if (out_scores_host)
+    ILRE_CUDA(cudaMemcpyAsync(out_scores_host, h->scores, static_cast<size_t>(L) * sizeof(float),
+                              cudaMemcpyDeviceToHost, st));
+  ILRE_CUDA(cudaStreamSynchronize(st));
+  return ILRE_OK;
+}
+
+int ilre_recall_copy_row_lse(ilre_recall_t* h, float* out_lse_dev, int32_t q_len,
+                             void* cuda_stream) {
+  if (!h || !out_lse_dev || q_len < 1 || q_len > h->cfg.max_q_len) return ILRE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return ILRE_ERR_CUDA;
+  ILRE_CUDA(cudaMemcpyAsync(out_lse_dev, h->row_lse,
+                            static_cast<size_t>(q_len) * h->cfg.n_q_heads * sizeof(float),
+                            cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(cuda_stream)));
+  return ILRE_OK;
+}
+
+int ilre_recall_status(ilre_recall_t* h) {
+  if (!h) return ILRE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return ILRE_ERR_CUDA;
+  ILRE_CUDA(cudaStreamSynchronize(h->last_stream));
+  int word = 0;
+  ILRE_CUDA(cudaMemcpy(&word, h->status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (word != 0) ILRE_CUDA(cudaMemset(h->status, 0, sizeof(int)));
+  if (word == 0) return ILRE_OK;
+  return (word == kDevQuota) ? ILRE_ERR_QUOTA : ILRE_ERR_DEVICE_WAIT;
+}
+
+int ilre_recall_set_profiling(ilre_recall_t* h, int32_t on) {
+  if (!h) return ILRE_ERR_INVALID_ARG;
+  h->profiling = on ? 1 : 0;
+  h->have_times = 0;
+  return ILRE_OK;
+}
+
+int ilre_recall_stage_times(ilre_recall_t* h, float* ms_host, int32_t n) {
+  if (!h || !ms_host || n < 1) return ILRE_ERR_INVALID_ARG;
+  if (!h->have_times) return ILRE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return ILRE_ERR_CUDA;
+  ILRE_CUDA(cudaEventSynchronize(h->ev[kNumStages]));
+  const int cnt = n < kNumStages ? n : kNumStages;
+  for (int i = 0; i < cnt; ++i) ILRE_CUDA(cudaEventElapsedTime(&ms_host[i], h->ev[i], h->ev[i + 1]));
+  return cnt;
+}
+
+int ilre_recall_last_launch_count(ilre_recall_t* h) {
+  return h ? h->last_launches : ILRE_ERR_INVALID_ARG;
+}
+
+int ilre_recall_destroy(ilre_recall_t* h) {
+  if (!h) return ILRE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return ILRE_ERR_CUDA;
+  cudaDeviceSynchronize();
+  free_all(h);
+  delete h;
+  return ILRE_OK;
+}
+
+const char* ilre_strerror(int code) {
+  switch (code) {
+    case ILRE_OK: return "ok";
+    case ILRE_ERR_INVALID_ARG: return "invalid argument";
+    case ILRE_ERR_UNSUPPORTED: return "unsupported configuration (needs head_dim 128, sm_100)";
+    case ILRE_ERR_CAPACITY: return "size exceeds the capacity given at create()";
+    case ILRE_ERR_BUDGET: return "budget larger than the context without its sink part";
+    case ILRE_ERR_ALIGNMENT: return "key cache / query base address must be 16-byte aligned";
+    case ILRE_ERR_CUDA: return "CUDA call failed";
+    case ILRE_ERR_DEVICE_WAIT: return "a bounded wait inside a kernel gave up";
+    case ILRE_ERR_QUOTA: return "a combination ran out of candidates";
+    case ILRE_ERR_NOMEM: return "device allocation failed";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

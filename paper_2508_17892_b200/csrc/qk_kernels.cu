@@ -1,0 +1,488 @@
+// Query-context attention kernels of the recall path (Eq. 4 and Eq. 5 of the paper).
+//
+// The [heads, q_len, L] probability tensor is never written to memory.  Two passes over the
+// key cache, both TMA -> shared memory -> tcgen05.mma -> tensor memory:
+//   row statistics: D[row, key] tiles, one thread per query row keeps an online (max, sum-exp);
+//   scores:         D[key, row] tiles (operands swapped), one thread per context position keeps
+//                   max over rows of (logit - lse_row); exp is monotone, so one exp per position
+//                   is taken afterwards.
+#include "qk_kernels.cuh"
+#include "sm100_ptx.cuh"
+
+namespace ilre {
+
+// ---------------------------------------------------------------------------------------
+// shared-memory tail layout (after the Q block and the K stages)
+// ---------------------------------------------------------------------------------------
+struct SmemTail {
+  uint64_t q_full;
+  uint64_t k_full[kMaxStages];
+  uint64_t k_empty[kMaxStages];
+  uint64_t acc_full[4];
+  uint64_t acc_empty[4];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+static_assert(sizeof(SmemTail) <= kSmemTailBytes, "tail too large");
+
+struct CtaItem {
+  int chunk, group, g;
+  int tile_begin, n_tiles;
+};
+
+__device__ __forceinline__ CtaItem decode_item(const QkParams& p) {
+  CtaItem it;
+  it.chunk = blockIdx.x / p.n_groups;
+  it.group = blockIdx.x % p.n_groups;
+  it.g = it.group / p.n_rb;
+  const long long t0 = static_cast<long long>(it.chunk) * p.n_tiles / p.cpg;
+  const long long t1 = static_cast<long long>(it.chunk + 1) * p.n_tiles / p.cpg;
+  it.tile_begin = static_cast<int>(t0);
+  it.n_tiles = static_cast<int>(t1 - t0);
+  return it;
+}
+
+// Common prologue: barrier init, TMEM allocation.  Returns the TMEM base address.
+__device__ __forceinline__ uint32_t cta_setup(SmemTail* tail, uint32_t smem_base, int stages,
+                                              int n_acc, int* status) {
+  const int warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) {
+    tail->abort_flag = 0;
+    if (smem_base & 1023u) {                       // swizzled tiles need 1024-byte alignment
+      tail->abort_flag = 1;
+      atomicCAS(status, 0, kDevSmemAlign);
+    }
+    mbar_init(smem_u32(&tail->q_full), 1);
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(smem_u32(&tail->k_full[s]), 1);
+      mbar_init(smem_u32(&tail->k_empty[s]), 1);
+    }
+    for (int b = 0; b < n_acc; ++b) {
+      mbar_init(smem_u32(&tail->acc_full[b]), 1);
+      mbar_init(smem_u32(&tail->acc_empty[b]), kConsumerWarps);
+    }
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&tail->tmem_base), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  return tail->tmem_base;
+}
+
+__device__ __forceinline__ void cta_teardown(uint32_t tmem_base) {
+  tc_fence_before();
+  __syncthreads();
+  if ((threadIdx.x >> 5) == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// TMA producer: the resident Q block once, then the K tiles of this CTA's key range.
+__device__ __forceinline__ void producer_loop(const CUtensorMap* tmapK, const CUtensorMap* tmapQ,
+                                              const QkParams& p, const CtaItem& it,
+                                              SmemTail* tail, uint32_t q_s, uint32_t k_s) {
+  volatile int* abort_flag = &tail->abort_flag;
+  const uint32_t qf = smem_u32(&tail->q_full);
+  mbar_arrive_expect_tx(qf, static_cast<uint32_t>(p.rb_rows) * 256u);
+  for (int kb = 0; kb < 2; ++kb)
+    for (int mt = 0; mt < p.rb_rows / 128; ++mt)
+      tma_load_2d(q_s + kb * p.rb_rows * 128 + mt * 16384, tmapQ, kb * 64,
+                  it.group * p.rb_rows + mt * 128, qf);
+  for (int i = 0; i < it.n_tiles; ++i) {
+    const int s = i % p.stages;
+    const uint32_t use = static_cast<uint32_t>(i / p.stages);
+    if (!mbar_wait(smem_u32(&tail->k_empty[s]), (use & 1u) ^ 1u, abort_flag, p.status,
+                   kDevWaitKEmpty))
+      break;
+    const uint32_t kf = smem_u32(&tail->k_full[s]);
+    mbar_arrive_expect_tx(kf, kStageBytes);
+    const int row = (it.tile_begin + i) * kTileKeys;
+    tma_load_2d(k_s + s * kStageBytes, tmapK, it.g * 128, row, kf);
+    tma_load_2d(k_s + s * kStageBytes + 16384, tmapK, it.g * 128 + 64, row, kf);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Pass A: row statistics.  MT = number of 128-row tiles of the resident Q block.
+// ---------------------------------------------------------------------------------------
+template <int MT>
+__global__ void __launch_bounds__(kQkThreads, 1)
+row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
+                 const __grid_constant__ CUtensorMap tmapQ, const QkParams p) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const uint32_t smem_base = smem_u32(smem);
+  const uint32_t q_s = smem_base;
+  const uint32_t k_s = smem_base + MT * 128 * 256;
+  SmemTail* tail = reinterpret_cast<SmemTail*>(smem + MT * 128 * 256 + p.stages * kStageBytes);
+  volatile int* abort_flag = &tail->abort_flag;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const CtaItem it = decode_item(p);
+
+  const uint32_t tmem_base = cta_setup(tail, smem_base, p.stages, 4, p.status);
+  const bool run = (it.n_tiles > 0) && (*abort_flag == 0);
+
+  if (warp == 0) {
+    if (lane == 0 && run) producer_loop(&tmapK, &tmapQ, p, it, tail, q_s, k_s);
+  } else if (warp == 1) {
+    if (lane == 0 && run) {
+      constexpr uint32_t idesc = umma_idesc_bf16(128, kTileKeys);
+      bool ok = mbar_wait(smem_u32(&tail->q_full), 0, abort_flag, p.status, kDevWaitQFull);
+      tc_fence_after();
+      uint32_t u = 0;
+      for (int i = 0; i < it.n_tiles && ok; ++i) {
+        const int s = i % p.stages;
+        const uint32_t kuse = static_cast<uint32_t>(i / p.stages);
+        ok = mbar_wait(smem_u32(&tail->k_full[s]), kuse & 1u, abort_flag, p.status,
+                       kDevWaitKFull);
+        if (!ok) break;
+        tc_fence_after();
+        for (int mt = 0; mt < MT; ++mt, ++u) {
+          const uint32_t b = u & 3u, use = u >> 2;
+          ok = mbar_wait(smem_u32(&tail->acc_empty[b]), (use & 1u) ^ 1u, abort_flag, p.status,
+                         kDevWaitAccEmpty);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+              const uint64_t a = umma_desc_sw128(q_s + kb * (MT * 128 * 128) + mt * 16384 + ks * 32);
+              const uint64_t bd = umma_desc_sw128(k_s + s * kStageBytes + kb * 16384 + ks * 32);
+              umma_bf16(tmem_base + b * 128, a, bd, idesc, (kb | ks) != 0);
+            }
+          umma_commit(smem_u32(&tail->acc_full[b]));
+        }
+        umma_commit(smem_u32(&tail->k_empty[s]));
+      }
+    }
+  } else if (warp >= 4) {
+    const int wg = (warp - 4) >> 2;          // which 64-column half of every tile
+    const int quad = warp & 3;               // TMEM lane quadrant this warp may read
+    float m[MT], z[MT];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) { m[mt] = -1e30f; z[mt] = 0.f; }
+    const float c2 = p.c2;
+    bool ok = run;
+    uint32_t u = 0;
+    for (int i = 0; i < it.n_tiles && ok; ++i) {
+      const long long key0 = static_cast<long long>(it.tile_begin + i) * kTileKeys;
+      const int valid = static_cast<int>(min(static_cast<long long>(kTileKeys), p.L - key0));
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        if (!ok) break;
+        const uint32_t b = u & 3u, use = u >> 2;
+        ++u;
+        ok = mbar_wait(smem_u32(&tail->acc_full[b]), use & 1u, abort_flag, p.status,
+                       kDevWaitAccFull);
+        if (!ok) break;
+        tc_fence_after();
+        float v0[32], v1[32];
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + b * 128 + wg * 64;
+        tmem_ld32(taddr, v0);
+        tmem_ld32(taddr + 32, v1);
+        tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&tail->acc_empty[b]));
+        if (valid < kTileKeys) {              // ragged last tile: keys past L do not exist
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            if (wg * 64 + j >= valid) v0[j] = -INFINITY;
+            if (wg * 64 + 32 + j >= valid) v1[j] = -INFINITY;
+          }
+        }
+        float cm0 = v0[0], cm1 = v0[1], cm2 = v1[0], cm3 = v1[1];
+#pragma unroll
+        for (int j = 2; j < 32; j += 2) {
+          cm0 = fmaxf(cm0, v0[j]); cm1 = fmaxf(cm1, v0[j + 1]);
+          cm2 = fmaxf(cm2, v1[j]); cm3 = fmaxf(cm3, v1[j + 1]);
+        }
+        const float m_new = fmaxf(m[mt], fmaxf(fmaxf(cm0, cm1), fmaxf(cm2, cm3)));
+        const float nm = -m_new * c2;
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+        for (int j = 0; j < 32; j += 2) {
+          s0 += ex2_approx(fmaf(v0[j], c2, nm));
+          s1 += ex2_approx(fmaf(v0[j + 1], c2, nm));
+          s2 += ex2_approx(fmaf(v1[j], c2, nm));
+          s3 += ex2_approx(fmaf(v1[j + 1], c2, nm));
+        }
+        z[mt] = z[mt] * ex2_approx((m[mt] - m_new) * c2) + ((s0 + s1) + (s2 + s3));
+        m[mt] = m_new;
+      }
+    }
+    // Merge the two column halves through shared memory (the K stages are idle by now) and
+    // write this CTA's partial statistics: (max in log2 units, sum).
+    float2* scratch = reinterpret_cast<float2*>(smem + MT * 128 * 256);
+    const int row_in_tile = quad * 32 + lane;
+    if (wg == 1) {
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) scratch[mt * 128 + row_in_tile] = make_float2(m[mt], z[mt]);
+    }
+    asm volatile("bar.sync 1, %0;" ::"r"(kConsumerWarps * 32) : "memory");
+    if (wg == 0) {
+      float2* out = reinterpret_cast<float2*>(p.partial) +
+                    (static_cast<size_t>(it.group) * p.cpg + it.chunk) * (MT * 128);
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        const float2 o = scratch[mt * 128 + row_in_tile];
+        const float mm = fmaxf(m[mt], o.x);
+        const float zz = z[mt] * exp2f((m[mt] - mm) * c2) + o.y * exp2f((o.x - mm) * c2);
+        out[mt * 128 + row_in_tile] = make_float2(mm * c2, zz);
+      }
+    }
+  }
+  cta_teardown(tmem_base);
+}
+
+// ---------------------------------------------------------------------------------------
+// Pass B: scores.  D[key, row]; per context position max over rows of log2-probability.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kQkThreads, 1)
+scores_kernel(const __grid_constant__ CUtensorMap tmapK,
+              const __grid_constant__ CUtensorMap tmapQ, const QkParams p) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const uint32_t smem_base = smem_u32(smem);
+  const uint32_t q_s = smem_base;
+  const uint32_t k_s = smem_base + p.rb_rows * 256;
+  SmemTail* tail = reinterpret_cast<SmemTail*>(smem + p.rb_rows * 256 + p.stages * kStageBytes);
+  float* nl = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(tail) + kSmemTailBytes);
+  volatile int* abort_flag = &tail->abort_flag;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const CtaItem it = decode_item(p);
+  const int n_nh = (p.rb_rows + 255) / 256;
+
+  for (int i = threadIdx.x; i < p.rb_rows; i += blockDim.x)
+    nl[i] = p.nlse2[static_cast<size_t>(it.group) * p.rb_rows + i];
+  const uint32_t tmem_base = cta_setup(tail, smem_base, p.stages, 2, p.status);
+  const bool run = (it.n_tiles > 0) && (*abort_flag == 0);
+
+  if (warp == 0) {
+    if (lane == 0 && run) producer_loop(&tmapK, &tmapQ, p, it, tail, q_s, k_s);
+  } else if (warp == 1) {
+    if (lane == 0 && run) {
+      bool ok = mbar_wait(smem_u32(&tail->q_full), 0, abort_flag, p.status, kDevWaitQFull);
+      tc_fence_after();
+      uint32_t u = 0;
+      for (int i = 0; i < it.n_tiles && ok; ++i) {
+        const int s = i % p.stages;
+        const uint32_t kuse = static_cast<uint32_t>(i / p.stages);
+        ok = mbar_wait(smem_u32(&tail->k_full[s]), kuse & 1u, abort_flag, p.status,
+                       kDevWaitKFull);
+        if (!ok) break;
+        tc_fence_after();
+        for (int nh = 0; nh < n_nh; ++nh, ++u) {
+          const int N = min(256, p.rb_rows - nh * 256);
+          const uint32_t idesc = umma_idesc_bf16(128, N);
+          const uint32_t b = u & 1u, use = u >> 1;
+          ok = mbar_wait(smem_u32(&tail->acc_empty[b]), (use & 1u) ^ 1u, abort_flag, p.status,
+                         kDevWaitAccEmpty);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+              const uint64_t a = umma_desc_sw128(k_s + s * kStageBytes + kb * 16384 + ks * 32);
+              const uint64_t bd =
+                  umma_desc_sw128(q_s + kb * (p.rb_rows * 128) + nh * (256 * 128) + ks * 32);
+              umma_bf16(tmem_base + b * 256, a, bd, idesc, (kb | ks) != 0);
+            }
+          umma_commit(smem_u32(&tail->acc_full[b]));
+        }
+        umma_commit(smem_u32(&tail->k_empty[s]));
+      }
+    }
+  } else if (warp >= 4) {
+    const int wg = (warp - 4) >> 2;
+    const int quad = warp & 3;
+    const float c2 = p.c2;
+    bool ok = run;
+    uint32_t u = 0;
+    for (int i = 0; i < it.n_tiles && ok; ++i) {
+      float best = -INFINITY;
+      for (int nh = 0; nh < n_nh && ok; ++nh) {
+        const int N = min(256, p.rb_rows - nh * 256);
+        const int half = N >> 1;
+        const uint32_t b = u & 1u, use = u >> 1;
+        ++u;
+        ok = mbar_wait(smem_u32(&tail->acc_full[b]), use & 1u, abort_flag, p.status,
+                       kDevWaitAccFull);
+        if (!ok) break;
+        tc_fence_after();
+        const int col0 = wg * half;
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + b * 256 + col0;
+        const float4* nl4 = reinterpret_cast<const float4*>(nl + nh * 256 + col0);
+        float b0 = -INFINITY, b1 = -INFINITY, b2 = -INFINITY, b3 = -INFINITY;
+        for (int c = 0; c < half; c += 32) {
+          float v[32];
+          tmem_ld32(taddr + c, v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            const float4 n4 = nl4[(c + j) >> 2];
+            b0 = fmaxf(b0, fmaf(v[j], c2, n4.x));
+            b1 = fmaxf(b1, fmaf(v[j + 1], c2, n4.y));
+            b2 = fmaxf(b2, fmaf(v[j + 2], c2, n4.z));
+            b3 = fmaxf(b3, fmaf(v[j + 3], c2, n4.w));
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&tail->acc_empty[b]));
+        best = fmaxf(best, fmaxf(fmaxf(b0, b1), fmaxf(b2, b3)));
+      }
+      const long long t = static_cast<long long>(it.tile_begin + i) * kTileKeys + quad * 32 + lane;
+      if (ok && t < p.L) atomicMax(p.enc + t, float_to_ordered(best));
+    }
+  }
+  cta_teardown(tmem_base);
+}
+
+// ---------------------------------------------------------------------------------------
+// small kernels around the two passes
+// ---------------------------------------------------------------------------------------
+
+// Packs the query rows of every (kv head, row block) contiguously, zero-padded to rb_rows,
+// and clears the per-run state (encoded scores, bitmap with the sink bits set, selection
+// state).
+__global__ void prepare_kernel(const uint4* __restrict__ q, uint4* __restrict__ qp, PrepParams p) {
+  const long long tid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const long long nthreads = static_cast<long long>(gridDim.x) * blockDim.x;
+  // packed query: 16 x uint4 per 128-element row
+  const long long n_pack = static_cast<long long>(p.n_kv) * p.n_rb * p.rb_rows * 16;
+  for (long long e = tid; e < n_pack; e += nthreads) {
+    const int part = static_cast<int>(e & 15);
+    const long long prow = e >> 4;
+    const int within = static_cast<int>(prow % p.rb_rows);
+    const int group = static_cast<int>(prow / p.rb_rows);
+    const int g = group / p.n_rb, rb = group % p.n_rb;
+    const int rg = rb * p.rb_rows + within;               // row inside the kv head's group
+    uint4 val = make_uint4(0, 0, 0, 0);
+    if (rg < p.group_size * p.q_len) {
+      const int i = rg / p.group_size, j = rg % p.group_size;
+      val = q[(static_cast<long long>(i) * p.n_q + g * p.group_size + j) * 16 + part];
+    }
+    qp[e] = val;
+  }
+  for (long long t = tid; t < p.L; t += nthreads) p.enc[t] = 0u;
+  const long long n_words = (p.L + 31) / 32;
+  for (long long w = tid; w < n_words; w += nthreads) {
+    const long long lo = w * 32;
+    uint32_t bits = 0;
+    if (p.n_sink > lo) bits = (p.n_sink - lo >= 32) ? 0xFFFFFFFFu : ((1u << (p.n_sink - lo)) - 1u);
+    p.bitmap[w] = bits;
+  }
+  for (long long e = tid; e < static_cast<long long>(p.n_comb) * p.hist_bins; e += nthreads)
+    p.hist[e] = 0u;
+  for (long long c = tid; c < p.n_comb; c += nthreads) {
+    p.sel_prefix[c] = 0ull;
+    p.sel_krem[c] = static_cast<uint32_t>(p.k_m[c]);
+    p.sel_done[c] = 0u;
+    p.sel_ticket[c] = 0u;
+    p.cand_count[c] = 0u;
+  }
+}
+
+// Combines the per-key-chunk partial statistics of every row into lse (log2 units, negated
+// for the scores pass; -inf marks padding rows) and the user-visible natural-log lse.
+__global__ void merge_stats_kernel(MergeParams p) {
+  const int prow = blockIdx.x * blockDim.x + threadIdx.x;
+  if (prow >= p.n_groups * p.rb_rows) return;
+  const int within = prow % p.rb_rows, group = prow / p.rb_rows;
+  const int g = group / p.n_rb, rb = group % p.n_rb;
+  const int rg = rb * p.rb_rows + within;
+  if (rg >= p.group_size * p.q_len) { p.nlse2[prow] = -INFINITY; return; }
+  const float2* part = reinterpret_cast<const float2*>(p.partial) +
+                       static_cast<size_t>(group) * p.cpg * p.rb_rows + within;
+  float mm = -INFINITY;
+  for (int c = 0; c < p.cpg; ++c) mm = fmaxf(mm, part[static_cast<size_t>(c) * p.rb_rows].x);
+  float zz = 0.f;
+  for (int c = 0; c < p.cpg; ++c) {
+    const float2 v = part[static_cast<size_t>(c) * p.rb_rows];
+    zz += v.y * exp2f(v.x - mm);
+  }
+  const float lse2 = mm + log2f(zz);
+  p.nlse2[prow] = -lse2;
+  const int i = rg / p.group_size, j = rg % p.group_size;
+  p.row_lse[i * p.n_q + g * p.group_size + j] = lse2 * 0.69314718055994530942f;
+}
+
+// A^C[t] = exp2(max_r log2 p_rt): decode the atomically-maximised value, one exp per position.
+__global__ void finalize_scores_kernel(const uint32_t* __restrict__ enc, float* __restrict__ scores,
+                                       float* __restrict__ user_scores, long long L) {
+  const long long t = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (t >= L) return;
+  const float a = exp2f(ordered_to_float(enc[t]));
+  scores[t] = a;
+  if (user_scores) user_scores[t] = a;
+}
+
+// ---------------------------------------------------------------------------------------
+// host-side launchers
+// ---------------------------------------------------------------------------------------
+size_t row_stats_smem_bytes(int rb_rows, int stages) {
+  return static_cast<size_t>(rb_rows) * 256 + static_cast<size_t>(stages) * kStageBytes +
+         kSmemTailBytes;
+}
+size_t scores_smem_bytes(int rb_rows, int stages) {
+  return row_stats_smem_bytes(rb_rows, stages) + static_cast<size_t>(rb_rows) * sizeof(float);
+}
+
+template <int MT>
+static cudaError_t launch_row_stats_mt(const CUtensorMap& tk, const CUtensorMap& tq,
+                                       const QkParams& p, cudaStream_t st) {
+  const size_t smem = row_stats_smem_bytes(MT * 128, p.stages);
+  cudaError_t e = cudaFuncSetAttribute(row_stats_kernel<MT>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  row_stats_kernel<MT><<<p.n_groups * p.cpg, kQkThreads, smem, st>>>(tk, tq, p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_row_stats(const CUtensorMap& tk, const CUtensorMap& tq, const QkParams& p,
+                             cudaStream_t st) {
+  switch (p.rb_rows / 128) {
+    case 1: return launch_row_stats_mt<1>(tk, tq, p, st);
+    case 2: return launch_row_stats_mt<2>(tk, tq, p, st);
+    case 3: return launch_row_stats_mt<3>(tk, tq, p, st);
+    case 4: return launch_row_stats_mt<4>(tk, tq, p, st);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+cudaError_t launch_scores(const CUtensorMap& tk, const CUtensorMap& tq, const QkParams& p,
+                          cudaStream_t st) {
+  const size_t smem = scores_smem_bytes(p.rb_rows, p.stages);
+  cudaError_t e = cudaFuncSetAttribute(scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)smem);
+  if (e != cudaSuccess) return e;
+  scores_kernel<<<p.n_groups * p.cpg, kQkThreads, smem, st>>>(tk, tq, p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_prepare(const void* q, void* qp, const PrepParams& p, int n_sm,
+                           cudaStream_t st) {
+  prepare_kernel<<<n_sm * 4, 256, 0, st>>>(static_cast<const uint4*>(q), static_cast<uint4*>(qp), p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_merge_stats(const MergeParams& p, cudaStream_t st) {
+  const int n = p.n_groups * p.rb_rows;
+  merge_stats_kernel<<<(n + 127) / 128, 128, 0, st>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_finalize_scores(const uint32_t* enc, float* scores, float* user_scores,
+                                   long long L, cudaStream_t st) {
+  finalize_scores_kernel<<<static_cast<unsigned>((L + 255) / 256), 256, 0, st>>>(enc, scores,
+                                                                                user_scores, L);
+  return cudaGetLastError();
+}
+
+}  // namespace ilre

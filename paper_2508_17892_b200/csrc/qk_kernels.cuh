@@ -1,0 +1,71 @@
+// Parameters and launchers of the query-context attention kernels (Eq. 4, Eq. 5).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ilre {
+
+static constexpr int kHeadDim = 128;
+static constexpr int kTileKeys = 128;              // keys per K tile (one TMA stage)
+static constexpr int kStageBytes = kTileKeys * kHeadDim * 2;
+static constexpr int kMaxStages = 6;
+static constexpr int kMaxRbRows = 512;             // query rows resident in shared memory
+static constexpr int kQkThreads = 384;             // warp 0 TMA, warp 1 MMA, warps 4..11 consumers
+static constexpr int kConsumerWarps = 8;
+static constexpr int kSmemTailBytes = 256;
+static constexpr int kMaxDynSmem = 232448;         // 227 KB per CTA on sm_100
+
+// Geometry of one recall, shared by both passes.
+struct QkParams {
+  long long L;
+  int n_tiles;       // ceil(L / kTileKeys)
+  int n_groups;      // n_kv_heads * n_rb
+  int n_rb;          // row blocks per kv head
+  int rb_rows;       // rows per block, multiple of 128, <= kMaxRbRows
+  int cpg;           // key chunks (CTAs) per group
+  int stages;
+  float c2;          // log2(e) / sqrt(d)
+  float* partial;    // [n_groups][cpg][rb_rows][2]: (max * c2, sum-exp) per key chunk
+  const float* nlse2;  // [n_groups][rb_rows]: -lse in log2 units, -inf for padding rows
+  uint32_t* enc;     // [L]: order-preserving uint of max_r log2 p_rt
+  int* status;
+};
+
+struct PrepParams {
+  int n_kv, n_q, group_size, q_len, n_rb, rb_rows;
+  long long L;
+  int n_sink;
+  uint32_t* enc;
+  uint32_t* bitmap;
+  uint32_t* hist;
+  int hist_bins;
+  int n_comb;
+  int k_m[64];
+  unsigned long long* sel_prefix;
+  uint32_t* sel_krem;
+  uint32_t* sel_done;
+  uint32_t* sel_ticket;
+  uint32_t* cand_count;
+};
+
+struct MergeParams {
+  int n_groups, n_rb, rb_rows, cpg, group_size, q_len, n_q;
+  const float* partial;
+  float* nlse2;
+  float* row_lse;    // [q_len][n_q] natural-log lse
+};
+
+size_t row_stats_smem_bytes(int rb_rows, int stages);
+size_t scores_smem_bytes(int rb_rows, int stages);
+
+cudaError_t launch_prepare(const void* q, void* qp, const PrepParams& p, int n_sm, cudaStream_t st);
+cudaError_t launch_row_stats(const CUtensorMap& tk, const CUtensorMap& tq, const QkParams& p,
+                             cudaStream_t st);
+cudaError_t launch_merge_stats(const MergeParams& p, cudaStream_t st);
+cudaError_t launch_scores(const CUtensorMap& tk, const CUtensorMap& tq, const QkParams& p,
+                          cudaStream_t st);
+cudaError_t launch_finalize_scores(const uint32_t* enc, float* scores, float* user_scores,
+                                   long long L, cudaStream_t st);
+
+}  // namespace ilre

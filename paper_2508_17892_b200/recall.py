@@ -1,0 +1,195 @@
+"""Python binding of the C ABI in ``include/ilre_recall.h`` (argument marshalling only).
+
+Every step of the recall path runs inside ``libilre_recall.so``; this module only turns torch
+tensors into pointers and sizes.  There is no CPU fallback: a missing library or a non-sm_100
+device raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libilre_recall.so")
+
+STAGE_NAMES = ("prepare", "row_stats", "merge_stats", "scores", "pool", "select", "allocate")
+
+EXPORTED_SYMBOLS = (
+    "ilre_recall_create", "ilre_recall_run", "ilre_recall_run_host", "ilre_recall_copy_row_lse",
+    "ilre_recall_status", "ilre_recall_set_profiling", "ilre_recall_stage_times",
+    "ilre_recall_last_launch_count", "ilre_recall_destroy", "ilre_strerror",
+)
+
+
+class IlreConfig(ctypes.Structure):
+    _fields_ = [("n_kv_heads", ctypes.c_int32), ("n_q_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("max_L", ctypes.c_int64),
+                ("max_q_len", ctypes.c_int32), ("max_budget", ctypes.c_int32),
+                ("max_combinations", ctypes.c_int32), ("device", ctypes.c_int32),
+                ("host_staging", ctypes.c_int32)]
+
+
+class IlrePoolSpec(ctypes.Structure):
+    _fields_ = [("n_max", ctypes.c_int32), ("max_sizes", ctypes.POINTER(ctypes.c_int32)),
+                ("n_win", ctypes.c_int32), ("win_sizes", ctypes.POINTER(ctypes.c_int32)),
+                ("win_op", ctypes.c_int32), ("reduce_op", ctypes.c_int32),
+                ("n_sink", ctypes.c_int32)]
+
+
+class IlreError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {code} ({strerror(code)})")
+        self.code = code
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """dlopen the in-tree shared library and declare the prototypes.  Raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(
+            f"{LIB_PATH} not found: build it with `python -m paper_2508_17892_b200.build`")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    lib.ilre_recall_create.argtypes = [ctypes.POINTER(IlreConfig), ctypes.POINTER(vp)]
+    lib.ilre_recall_run.argtypes = [vp, vp, i64, vp, i32, i32, ctypes.POINTER(IlrePoolSpec), vp, vp, vp]
+    lib.ilre_recall_run_host.argtypes = lib.ilre_recall_run.argtypes
+    lib.ilre_recall_copy_row_lse.argtypes = [vp, vp, i32, vp]
+    lib.ilre_recall_status.argtypes = [vp]
+    lib.ilre_recall_set_profiling.argtypes = [vp, i32]
+    lib.ilre_recall_stage_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float), i32]
+    lib.ilre_recall_last_launch_count.argtypes = [vp]
+    lib.ilre_recall_destroy.argtypes = [vp]
+    lib.ilre_strerror.argtypes = [ctypes.c_int]
+    lib.ilre_strerror.restype = ctypes.c_char_p
+    for name in EXPORTED_SYMBOLS:
+        if name != "ilre_strerror":
+            getattr(lib, name).restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load_library().ilre_strerror(code).decode()
+
+
+def _spec(max_sizes: Sequence[int], win_sizes: Sequence[int], win_op: int, n_sink: int):
+    ms = (ctypes.c_int32 * len(max_sizes))(*max_sizes)
+    ws = (ctypes.c_int32 * len(win_sizes))(*win_sizes)
+    spec = IlrePoolSpec(len(max_sizes), ms, len(win_sizes), ws, win_op, 0, n_sink)
+    return spec, (ms, ws)
+
+
+class IlreRecall:
+    """Owns one ``ilre_recall_t`` handle (device workspace sized at construction)."""
+
+    def __init__(self, max_L: int, max_q_len: int, max_budget: int = 4096,
+                 max_combinations: int = 48, n_kv_heads: int = 8, n_q_heads: int = 32,
+                 head_dim: int = 128, device: int = 0, host_staging: bool = False):
+        self._lib = load_library()
+        self.cfg = IlreConfig(n_kv_heads, n_q_heads, head_dim, max_L, max_q_len, max_budget,
+                              max_combinations, device, int(host_staging))
+        self._h = ctypes.c_void_p()
+        rc = self._lib.ilre_recall_create(ctypes.byref(self.cfg), ctypes.byref(self._h))
+        if rc != 0:
+            self._h = ctypes.c_void_p()
+            raise IlreError(rc, "ilre_recall_create")
+        self.device = torch.device("cuda", device)
+
+    # -- the recall --------------------------------------------------------------------
+    def run(self, K: torch.Tensor, Q: torch.Tensor, budget: int, max_sizes: Sequence[int],
+            win_sizes: Sequence[int], win_op: int = 0, n_sink: int = 0,
+            out_idx: Optional[torch.Tensor] = None, out_scores: Optional[torch.Tensor] = None,
+            want_scores: bool = False, stream: Optional[torch.cuda.Stream] = None):
+        """Asynchronous recall on ``stream`` (default: torch's current stream).
+
+        K: bf16 [L, n_kv_heads, 128] on the device; Q: bf16 [q_len, n_q_heads, 128].
+        Returns (indices int32 [n_sink + budget], scores fp32 [L] or None).
+        """
+        assert K.is_cuda and Q.is_cuda and K.dtype == torch.bfloat16 and Q.dtype == torch.bfloat16
+        assert K.is_contiguous() and Q.is_contiguous()
+        L, q_len = K.shape[0], Q.shape[0]
+        assert K.shape[1:] == (self.cfg.n_kv_heads, self.cfg.head_dim)
+        assert Q.shape[1:] == (self.cfg.n_q_heads, self.cfg.head_dim)
+        if out_idx is None:
+            out_idx = torch.empty(n_sink + budget, dtype=torch.int32, device=K.device)
+        if out_scores is None and want_scores:
+            out_scores = torch.empty(L, dtype=torch.float32, device=K.device)
+        spec, _keep = _spec(max_sizes, win_sizes, win_op, n_sink)
+        st = stream if stream is not None else torch.cuda.current_stream(K.device)
+        rc = self._lib.ilre_recall_run(self._h, K.data_ptr(), L, Q.data_ptr(), q_len, budget,
+                                       ctypes.byref(spec), out_idx.data_ptr(),
+                                       out_scores.data_ptr() if out_scores is not None else None,
+                                       st.cuda_stream)
+        if rc != 0:
+            raise IlreError(rc, "ilre_recall_run")
+        return out_idx, out_scores
+
+    def run_host(self, K: torch.Tensor, Q: torch.Tensor, budget: int, max_sizes: Sequence[int],
+                 win_sizes: Sequence[int], win_op: int = 0, n_sink: int = 0,
+                 out_idx: Optional[torch.Tensor] = None, out_scores: Optional[torch.Tensor] = None,
+                 stream: Optional[torch.cuda.Stream] = None):
+        """Recall from HOST tensors (pinned for speed); synchronises before returning."""
+        assert not K.is_cuda and not Q.is_cuda
+        assert K.dtype == torch.bfloat16 and Q.dtype == torch.bfloat16
+        assert K.is_contiguous() and Q.is_contiguous()
+        L, q_len = K.shape[0], Q.shape[0]
+        if out_idx is None:
+            out_idx = torch.empty(n_sink + budget, dtype=torch.int32)
+        spec, _keep = _spec(max_sizes, win_sizes, win_op, n_sink)
+        st = stream if stream is not None else torch.cuda.current_stream(self.device)
+        rc = self._lib.ilre_recall_run_host(self._h, K.data_ptr(), L, Q.data_ptr(), q_len, budget,
+                                            ctypes.byref(spec), out_idx.data_ptr(),
+                                            out_scores.data_ptr() if out_scores is not None else None,
+                                            st.cuda_stream)
+        if rc != 0:
+            raise IlreError(rc, "ilre_recall_run_host")
+        return out_idx, out_scores
+
+    # -- diagnostics -------------------------------------------------------------------
+    def row_lse(self, q_len: int, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        out = torch.empty(q_len, self.cfg.n_q_heads, dtype=torch.float32, device=self.device)
+        st = stream if stream is not None else torch.cuda.current_stream(self.device)
+        rc = self._lib.ilre_recall_copy_row_lse(self._h, out.data_ptr(), q_len, st.cuda_stream)
+        if rc != 0:
+            raise IlreError(rc, "ilre_recall_copy_row_lse")
+        return out
+
+    def status(self) -> int:
+        return self._lib.ilre_recall_status(self._h)
+
+    def check_status(self) -> None:
+        rc = self.status()
+        if rc != 0:
+            raise IlreError(rc, "ilre_recall_status")
+
+    def set_profiling(self, on: bool) -> None:
+        self._lib.ilre_recall_set_profiling(self._h, int(on))
+
+    def stage_times(self) -> dict:
+        buf = (ctypes.c_float * len(STAGE_NAMES))()
+        n = self._lib.ilre_recall_stage_times(self._h, buf, len(STAGE_NAMES))
+        if n < 0:
+            raise IlreError(n, "ilre_recall_stage_times")
+        return {STAGE_NAMES[i]: float(buf[i]) for i in range(n)}
+
+    def last_launch_count(self) -> int:
+        return self._lib.ilre_recall_last_launch_count(self._h)
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h.value:
+            self._lib.ilre_recall_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
