@@ -1,0 +1,327 @@
+#!/usr/bin/env python
+"""Benchmark of the ILRe token-recall path on B200.
+
+A "step" is one whole recall (query packing, row statistics, scores, pooling, top-K_m
+selection, allocation) on the L = 1M benchmark configuration: key cache [1048576, 8, 128]
+bf16 (2 GiB), q_len = 256, budget 4096, window sizes {1,7,15,31,63}.  The headline value is
+key-cache GB/s = bytes of K / time of one recall, with the inputs resident in HBM; `e2e` is
+the same metric through the host entry point (host buffers, copies inside the timed region).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config NAME]
+
+With N > 1 (under torchrun) every rank runs an independent replica of the same recall on its
+own GPU (the path has no exchange step); the value is the sum over ranks divided by the
+slowest rank's time.  `--impl reference` times the CPU oracle on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+METRIC = "key_cache_GBps_per_recall_L1M"
+UNIT = "GB/s"
+CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0,
+                source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={CLOCK_QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100", "-i", str(self.gpu_index), "-f", self.path],
+                stdout=subprocess.DEVNULL, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            with open(self.path) as f:
+                for line in f:
+                    cols = [c.strip() for c in line.split(",")]
+                    if len(cols) < 9:
+                        continue
+                    try:
+                        sm.append(float(cols[1]))
+                        smax.append(float(cols[2]))
+                    except ValueError:
+                        continue
+                    for name, val in zip(names, cols[5:9]):
+                        if val.lower().startswith("active"):
+                            reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(smax)),
+                       reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def dist_setup(n_gpus: int):
+    """Process-group plumbing for N > 1 (barrier and max-over-ranks only; no data exchange)."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        backend = "nccl" if torch.cuda.is_available() else "gloo"
+        dist.init_process_group(backend=backend)
+    return world, rank, local
+
+
+def aggregate(elapsed_ms: float, units: float, device=None):
+    """(max elapsed over ranks, sum of units over ranks).  Works on gloo (CPU) and nccl."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return elapsed_ms, units
+    dev = device if device is not None else torch.device("cpu")
+    t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
+    u = torch.tensor([units], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def barrier():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.barrier()
+
+
+def workload_string(w) -> str:
+    return (f"{w.name}: L={w.L}, q_len={w.q_len}, kv_heads={w.n_kv_heads}, "
+            f"q_heads={w.n_q_heads}, d={w.d}, budget={w.budget}, "
+            f"windows={list(w.win_sizes)} (max), max_sizes={list(w.max_sizes)}")
+
+
+def oracle_sample_run(x, sample_keys: int):
+    """One oracle recall on the first `sample_keys` positions of the workload."""
+    import oracle
+    w = x.workload
+    Ks = x.K[:sample_keys].contiguous()
+    budget = min(w.budget, sample_keys)
+    t0 = time.perf_counter()
+    oracle.recall(Ks, x.Q, budget, w.max_sizes, w.win_sizes, w.win_op, 0)
+    return time.perf_counter() - t0, Ks.numel() * 2
+
+
+def run_reference(args, world, rank):
+    """Reference arm: the CPU oracle, as it stands, on a bounded sample of the workload."""
+    if rank != 0:
+        return
+    from workloads import CONFIGS, make_inputs
+    import dataclasses
+    w = CONFIGS[args.config]
+    cores = len(os.sched_getaffinity(0))
+    sample_keys = args.ref_sample_keys
+    # only the sampled prefix of the cache is needed; the generator is prefix-stable in L
+    # except for span placement, so build a workload of the sample length with the same seed
+    ws = dataclasses.replace(w, L=sample_keys, n_spans=max(1, w.n_spans * sample_keys // w.L),
+                             budget=min(w.budget, sample_keys))
+    x = make_inputs(ws)
+    for _ in range(args.warmup):
+        oracle_sample_run(x, sample_keys)
+    t_total, nbytes = 0.0, 0
+    for _ in range(args.steps):
+        dt, nb = oracle_sample_run(x, sample_keys)
+        t_total += dt
+        nbytes = nb
+    ms = 1e3 * t_total / args.steps
+    value = nbytes / (ms * 1e-3) / 1e9
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus,
+                steps=args.steps, warmup=args.warmup, ms_per_step=ms, higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                config=dict(workload=workload_string(w),
+                            sample=f"each step: first {sample_keys} of {w.L} keys, budget "
+                                   f"{ws.budget}"),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle",
+                                  sample=f"first {sample_keys} keys of the cache, all "
+                                         f"{w.q_len * w.n_q_heads} query rows, per step"),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, world, rank, local):
+    from paper_2508_17892_b200 import IlreRecall, build
+    from workloads import CONFIGS, make_inputs
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (sm_100); there is no CPU fallback")
+    build.build()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    w = CONFIGS[args.config]
+    x = make_inputs(w)
+    eng = IlreRecall(max_L=w.L, max_q_len=w.q_len, max_budget=w.budget, n_kv_heads=w.n_kv_heads,
+                     n_q_heads=w.n_q_heads, device=local, host_staging=not args.no_e2e)
+    K, Q = x.K.to(dev), x.Q.to(dev)
+    out_idx = torch.empty(w.n_sink + w.budget, dtype=torch.int32, device=dev)
+    spec = (w.budget, w.max_sizes, w.win_sizes, w.win_op, w.n_sink)
+    k_bytes = K.numel() * 2
+
+    def step():
+        eng.run(K, Q, *spec, out_idx=out_idx)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    eng.check_status()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    eng.set_profiling(True)
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    start.record()
+    for _ in range(args.steps):
+        step()
+    stop.record()
+    torch.cuda.synchronize()
+    barrier()
+    elapsed_ms = start.elapsed_time(stop)
+    stages = eng.stage_times()
+    eng.set_profiling(False)
+    launches = eng.last_launch_count() * args.steps
+    eng.check_status()
+    clocks = sampler.stop() if rank == 0 else None
+
+    # end to end through the host entry point: pinned host inputs, copies inside the timing
+    e2e = None
+    if not args.no_e2e:
+        Kh, Qh = x.K.pin_memory(), x.Q.pin_memory()
+        idx_h = torch.empty(w.n_sink + w.budget, dtype=torch.int32).pin_memory()
+        e2e_steps = max(3, min(args.steps, 10))
+        eng.run_host(Kh, Qh, *spec, out_idx=idx_h)
+        barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            eng.run_host(Kh, Qh, *spec, out_idx=idx_h)
+        torch.cuda.synchronize()
+        e2e_ms = 1e3 * (time.perf_counter() - t0) / e2e_steps
+        e2e_ms_max, e2e_units = aggregate(e2e_ms, float(k_bytes), dev)
+        assert torch.equal(idx_h, out_idx.cpu())
+        e2e = dict(value=e2e_units / (e2e_ms_max * 1e-3) / 1e9, unit=UNIT, ms_per_step=e2e_ms_max,
+                   h2d_bytes_per_step=int(k_bytes + Q.numel() * 2),
+                   d2h_bytes_per_step=int(idx_h.numel() * 4), steps=e2e_steps)
+
+    elapsed_max, units = aggregate(elapsed_ms, float(k_bytes) * args.steps, dev)
+    if rank != 0:
+        return
+    ms_per_step = elapsed_max / args.steps
+    value = units / (elapsed_max * 1e-3) / 1e9
+    peaks = measured_peaks()
+    R = w.q_len * w.n_q_heads
+    flops = 2.0 * R * w.L * w.d                         # one QK^T (Eq. 4), algorithmic
+    dom = max(("row_stats", "scores"), key=lambda k: stages[k])
+    dom_tflops = flops / (stages[dom] * 1e-3) / 1e12
+    roofline = dict(bound="tensor", kernel=f"{dom}_kernel", achieved=dom_tflops,
+                    peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s",
+                    frac=dom_tflops / peaks["bf16_tflops_sustained"], traffic=None,
+                    peak_source=f"{peaks['source']} (sustained bf16)",
+                    kernel_ms=stages[dom], algorithmic_flops_per_launch=flops,
+                    algorithmic_bytes_per_launch=k_bytes,
+                    kernel_hbm_gbs=k_bytes / (stages[dom] * 1e-3) / 1e9)
+    step_hbm_frac = (k_bytes / (ms_per_step * 1e-3) / 1e9) / peaks["hbm_gbs"]
+    step_tensor_frac = (flops / (ms_per_step * 1e-3) / 1e12) / peaks["bf16_tflops_sustained"]
+
+    cpu_baseline = None
+    if not args.no_cpu_baseline and world == 1:
+        cores = len(os.sched_getaffinity(0))
+        dt, nb = oracle_sample_run(x, args.cpu_sample_keys)
+        cpu_baseline = dict(value=nb / dt / 1e9, unit=UNIT, cores=cores, kind="oracle",
+                            seconds=dt,
+                            sample=f"first {args.cpu_sample_keys} of {w.L} keys, all {R} query "
+                                   f"rows, full Algorithm 1 on that prefix")
+
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps,
+                warmup=max(args.warmup, 3), ms_per_step=ms_per_step, higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic",
+                config=dict(workload=workload_string(w),
+                            l2="key cache (2 GiB) is larger than L2; no flush needed",
+                            parallelism="replicas only" if world > 1 else "single GPU"),
+                clocks=clocks, e2e=e2e, gpu_launches=launches, roofline=roofline,
+                cpu_baseline=cpu_baseline,
+                stages_ms=stages,
+                whole_step=dict(hbm_frac_one_read_of_K=step_hbm_frac,
+                                tensor_frac_one_qk=step_tensor_frac,
+                                hbm_frac_of_8TBps=(k_bytes / (ms_per_step * 1e-3) / 1e9) / 8000.0))
+    print(json.dumps(line), flush=True)
+    eng.close()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--config", default="cfg5_L1m")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-sample-keys", type=int, default=16384)
+    ap.add_argument("--ref-sample-keys", type=int, default=4096)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        rank = int(os.environ.get("RANK", "0"))
+        run_reference(args, int(os.environ.get("WORLD_SIZE", "1")), rank)
+        return
+    world, rank, local = dist_setup(args.gpus)
+    try:
+        run_ours(args, world, rank, local)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+            if dist.is_initialized():
+                dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -122,8 +122,9 @@ int ilre_recall_status(ilre_recall_t* h);
 
 /*
  * Stage timing.  With profiling on, run() records CUDA events between its stages on the
- * caller's stream.  ilre_recall_stage_times synchronises on the last event and writes up to
- * n entries (milliseconds) in this order:
+ * caller's stream (the events of the 32 most recent runs are kept).  Switching profiling on
+ * resets the history.  ilre_recall_stage_times synchronises on those events and writes up to
+ * n entries, each the mean over the recorded runs (milliseconds), in this order:
  *   0 prepare (query packing, clears)   1 row statistics (QK^T + online softmax)
  *   2 statistics merge                  3 scores (QK^T + max over rows)
  *   4 pooling                           5 top-K_m selection and ranking

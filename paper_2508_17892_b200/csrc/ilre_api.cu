@@ -23,6 +23,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 constexpr int kNumStages = 7;            // timed stages (see ilre_recall_stage_times)
+constexpr int kProfRing = 32;            // runs whose stage events are kept for averaging
 constexpr int kMaxSinkStaging = 65536;
 
 struct Geometry {
@@ -58,9 +59,9 @@ struct ilre_recall {
   void* stage_q;
   int* stage_idx;
   // bookkeeping
-  cudaEvent_t ev[kNumStages + 1];
+  cudaEvent_t ev[kProfRing][kNumStages + 1];
   int profiling;
-  int have_times;
+  long long prof_runs;                  // runs recorded since profiling was switched on
   int last_launches;
   int last_q_len;
   cudaStream_t last_stream;
@@ -116,8 +117,9 @@ void free_all(ilre_recall* h) {
   cudaFree(h->sel_prefix); cudaFree(h->sel_krem); cudaFree(h->sel_done); cudaFree(h->sel_ticket);
   cudaFree(h->cand); cudaFree(h->cand_count); cudaFree(h->ranked); cudaFree(h->bitmap);
   cudaFree(h->status); cudaFree(h->stage_k); cudaFree(h->stage_q); cudaFree(h->stage_idx);
-  for (int i = 0; i <= kNumStages; ++i)
-    if (h->ev[i]) cudaEventDestroy(h->ev[i]);
+  for (int r = 0; r < kProfRing; ++r)
+    for (int i = 0; i <= kNumStages; ++i)
+      if (h->ev[r][i]) cudaEventDestroy(h->ev[r][i]);
 }
 
 bool encode_2d(EncodeTiledFn fn, CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows,
@@ -235,7 +237,9 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out) {
                          static_cast<size_t>(cfg->max_q_len) * cfg->n_q_heads * 256);
     ok = ok && dev_alloc(&h->stage_idx, static_cast<size_t>(cfg->max_budget) + kMaxSinkStaging);
   }
-  for (int i = 0; ok && i <= kNumStages; ++i) ok = (cudaEventCreate(&h->ev[i]) == cudaSuccess);
+  for (int r = 0; ok && r < kProfRing; ++r)
+    for (int i = 0; ok && i <= kNumStages; ++i)
+      ok = (cudaEventCreate(&h->ev[r][i]) == cudaSuccess);
   if (ok) ok = (cudaMemset(h->status, 0, sizeof(int)) == cudaSuccess);
   if (ok) ok = (cudaDeviceSynchronize() == cudaSuccess);
   if (!ok) {
@@ -319,10 +323,10 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
 
   const bool prof = h->profiling != 0;
   int launches = 0;
-  h->have_times = 0;
   h->last_stream = st;
   h->last_q_len = q_len;
-#define ILRE_MARK(i) do { if (prof) ILRE_CUDA(cudaEventRecord(h->ev[i], st)); } while (0)
+  cudaEvent_t* ev = h->ev[h->prof_runs % kProfRing];
+#define ILRE_MARK(i) do { if (prof) ILRE_CUDA(cudaEventRecord(ev[i], st)); } while (0)
 
   ILRE_MARK(0);
   ILRE_CUDA(launch_prepare(query_dev, h->qp, pp, h->n_sm, st)); ++launches;
@@ -350,7 +354,7 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
   ILRE_MARK(7);
 #undef ILRE_MARK
   h->last_launches = launches;
-  h->have_times = prof ? 1 : 0;
+  if (prof) ++h->prof_runs;
   return ILRE_OK;
 }
 
@@ -408,18 +412,27 @@ int ilre_recall_status(ilre_recall_t* h) {
 int ilre_recall_set_profiling(ilre_recall_t* h, int32_t on) {
   if (!h) return ILRE_ERR_INVALID_ARG;
   h->profiling = on ? 1 : 0;
-  h->have_times = 0;
+  h->prof_runs = 0;
   return ILRE_OK;
 }
 
 int ilre_recall_stage_times(ilre_recall_t* h, float* ms_host, int32_t n) {
   if (!h || !ms_host || n < 1) return ILRE_ERR_INVALID_ARG;
-  if (!h->have_times) return ILRE_ERR_INVALID_ARG;
+  if (h->prof_runs < 1) return ILRE_ERR_INVALID_ARG;
   DeviceGuard guard(h->cfg.device);
   if (!guard.ok) return ILRE_ERR_CUDA;
-  ILRE_CUDA(cudaEventSynchronize(h->ev[kNumStages]));
+  const int runs = h->prof_runs < kProfRing ? static_cast<int>(h->prof_runs) : kProfRing;
   const int cnt = n < kNumStages ? n : kNumStages;
-  for (int i = 0; i < cnt; ++i) ILRE_CUDA(cudaEventElapsedTime(&ms_host[i], h->ev[i], h->ev[i + 1]));
+  for (int i = 0; i < cnt; ++i) ms_host[i] = 0.f;
+  for (int r = 0; r < runs; ++r) {
+    cudaEvent_t* ev = h->ev[(h->prof_runs - 1 - r) % kProfRing];
+    ILRE_CUDA(cudaEventSynchronize(ev[kNumStages]));
+    for (int i = 0; i < cnt; ++i) {
+      float ms = 0.f;
+      ILRE_CUDA(cudaEventElapsedTime(&ms, ev[i], ev[i + 1]));
+      ms_host[i] += ms / static_cast<float>(runs);
+    }
+  }
   return cnt;
 }
 
