@@ -139,6 +139,17 @@ def workload_string(w) -> str:
             f"windows={list(w.win_sizes)} (max), max_sizes={list(w.max_sizes)}")
 
 
+def pick_workload(args):
+    import dataclasses
+    from workloads import CONFIGS
+    w = CONFIGS[args.config]
+    if args.L and args.L != w.L:
+        w = dataclasses.replace(w, name=f"{w.name}_L{args.L}", L=args.L,
+                                n_spans=max(1, w.n_spans * args.L // w.L),
+                                budget=min(w.budget, args.L))
+    return w
+
+
 def oracle_sample_run(x, sample_keys: int):
     """One oracle recall on the first `sample_keys` positions of the workload."""
     import oracle
@@ -154,9 +165,9 @@ def run_reference(args, world, rank):
     """Reference arm: the CPU oracle, as it stands, on a bounded sample of the workload."""
     if rank != 0:
         return
-    from workloads import CONFIGS, make_inputs
+    from workloads import make_inputs
     import dataclasses
-    w = CONFIGS[args.config]
+    w = pick_workload(args)
     cores = len(os.sched_getaffinity(0))
     sample_keys = args.ref_sample_keys
     # only the sampled prefix of the cache is needed; the generator is prefix-stable in L
@@ -188,13 +199,13 @@ def run_reference(args, world, rank):
 
 def run_ours(args, world, rank, local):
     from paper_2508_17892_b200 import IlreRecall, build
-    from workloads import CONFIGS, make_inputs
+    from workloads import make_inputs
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (sm_100); there is no CPU fallback")
     build.build()
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    w = CONFIGS[args.config]
+    w = pick_workload(args)
     x = make_inputs(w)
     eng = IlreRecall(max_L=w.L, max_q_len=w.q_len, max_budget=w.budget, n_kv_heads=w.n_kv_heads,
                      n_q_heads=w.n_q_heads, device=local, host_staging=not args.no_e2e)
@@ -275,10 +286,10 @@ def run_ours(args, world, rank, local):
     cpu_baseline = None
     if not args.no_cpu_baseline and world == 1:
         cores = len(os.sched_getaffinity(0))
-        dt, nb = oracle_sample_run(x, args.cpu_sample_keys)
+        dt, nb = oracle_sample_run(x, min(args.cpu_sample_keys, w.L))
         cpu_baseline = dict(value=nb / dt / 1e9, unit=UNIT, cores=cores, kind="oracle",
                             seconds=dt,
-                            sample=f"first {args.cpu_sample_keys} of {w.L} keys, all {R} query "
+                            sample=f"first {min(args.cpu_sample_keys, w.L)} of {w.L} keys, all {R} query "
                                    f"rows, full Algorithm 1 on that prefix")
 
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps,
@@ -306,7 +317,9 @@ def main():
     ap.add_argument("--config", default="cfg5_L1m")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-sample-keys", type=int, default=16384)
+    ap.add_argument("--L", type=int, default=0,
+                    help="override the context length of --config (profiling on a small case)")
+    ap.add_argument("--cpu-sample-keys", type=int, default=131072)
     ap.add_argument("--ref-sample-keys", type=int, default=4096)
     args = ap.parse_args()
     if args.impl == "reference":
