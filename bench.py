@@ -30,6 +30,10 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
+# DRAM bytes per context position of the dominant kernel (row statistics), from one ncu
+# capture at L = 131072, q_len = 256: (270.6 MB read + 4.4 MB written) / 131072 keys.  Traffic
+# grows in proportion to L (the query block is L2-resident), so it is scaled by L.
+ROW_STATS_DRAM_BYTES_PER_KEY = 2098.2
 METRIC = "key_cache_GBps_per_recall_L1M"
 UNIT = "GB/s"
 CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -275,7 +279,10 @@ def run_ours(args, world, rank, local):
     dom_tflops = flops / (stages[dom] * 1e-3) / 1e12
     roofline = dict(bound="tensor", kernel=f"{dom}_kernel", achieved=dom_tflops,
                     peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s",
-                    frac=dom_tflops / peaks["bf16_tflops_sustained"], traffic=None,
+                    frac=dom_tflops / peaks["bf16_tflops_sustained"],
+                    traffic=(ROW_STATS_DRAM_BYTES_PER_KEY * w.L
+                             if dom == "row_stats" and w.q_len == 256 else None),
+                    traffic_unit="bytes per launch (ncu at L=131072, scaled by L)",
                     peak_source=f"{peaks['source']} (sustained bf16)",
                     kernel_ms=stages[dom], algorithmic_flops_per_launch=flops,
                     algorithmic_bytes_per_launch=k_bytes,
@@ -311,7 +318,7 @@ def run_ours(args, world, rank, local):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--config", default="cfg5_L1m")
