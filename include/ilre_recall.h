@@ -139,6 +139,27 @@ int ilre_recall_last_launch_count(ilre_recall_t* h);
 
 int ilre_recall_destroy(ilre_recall_t* h);
 
+/*
+ * Top-k of a score array without any allocation (the paper has no counterpart: this is a
+ * convenience for callers that are not allowed to allocate device memory, e.g. code running
+ * under a framework-owned memory pool or in a thread that must not hit cudaMalloc's implicit
+ * synchronisation).  No handle is needed.  Returns the k positions with the highest scores,
+ * equal scores ranked by lower position, as ascending int32 positions -- what
+ * ilre_recall_run returns for one max kernel of size 1, one window of size 1 and no sink.
+ *   scores_dev   fp32 [L] on the CURRENT device; 1 <= L <= ILRE_NOALLOC_MAX_L
+ *   out_idx_dev  int32 [k] on the current device; 0 <= k <= L
+ * Larger L is rejected with ILRE_ERR_CAPACITY, k > L with ILRE_ERR_BUDGET; nothing is launched
+ * then.  The call is asynchronous on cuda_stream and calls no cudaMalloc/cudaFree.  Its scratch
+ * (a bitmap of ILRE_NOALLOC_MAX_L bits = 128 KiB) is a fixed __device__ array inside the
+ * library, resident on every GPU that loads the library until the process exits, and SHARED
+ * by all calls: two calls that overlap on the same GPU (different streams or threads) race;
+ * serialise them.  The first call on each device looks the array's address up (this may load
+ * the library's device code), so make that first call before starting any stream capture.
+ */
+#define ILRE_NOALLOC_MAX_L 1048576
+int ilre_topk_positions_noalloc(const float* scores_dev, int64_t L, int32_t k,
+                                int32_t* out_idx_dev, void* cuda_stream);
+
 const char* ilre_strerror(int code);
 
 #ifdef __cplusplus

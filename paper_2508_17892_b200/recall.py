@@ -21,7 +21,10 @@ EXPORTED_SYMBOLS = (
     "ilre_recall_create", "ilre_recall_run", "ilre_recall_run_host", "ilre_recall_copy_row_lse",
     "ilre_recall_status", "ilre_recall_set_profiling", "ilre_recall_stage_times",
     "ilre_recall_last_launch_count", "ilre_recall_destroy", "ilre_strerror",
+    "ilre_topk_positions_noalloc",
 )
+
+NOALLOC_MAX_L = 1048576
 
 
 class IlreConfig(ctypes.Structure):
@@ -68,6 +71,7 @@ def load_library() -> ctypes.CDLL:
     lib.ilre_recall_last_launch_count.argtypes = [vp]
     lib.ilre_recall_destroy.argtypes = [vp]
     lib.ilre_strerror.argtypes = [ctypes.c_int]
+    lib.ilre_topk_positions_noalloc.argtypes = [vp, i64, i32, vp, vp]
     lib.ilre_strerror.restype = ctypes.c_char_p
     for name in EXPORTED_SYMBOLS:
         if name != "ilre_strerror":
@@ -85,6 +89,29 @@ def _spec(max_sizes: Sequence[int], win_sizes: Sequence[int], win_op: int, n_sin
     ws = (ctypes.c_int32 * len(win_sizes))(*win_sizes)
     spec = IlrePoolSpec(len(max_sizes), ms, len(win_sizes), ws, win_op, 0, n_sink)
     return spec, (ms, ws)
+
+
+def topk_positions_noalloc(scores: torch.Tensor, k: int,
+                           out_idx: Optional[torch.Tensor] = None,
+                           stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Ascending positions of the k highest scores (ties: lower position first).
+
+    For callers that may not allocate device memory: the library call behind this function
+    needs no handle and allocates nothing (its scratch is a fixed array inside the library,
+    shared by all calls -- do not overlap two calls on one GPU).  Pass ``out_idx`` (int32 [k]
+    on the same device) to keep this wrapper allocation-free too.  ``len(scores)`` must not
+    exceed ``NOALLOC_MAX_L``.
+    """
+    assert scores.is_cuda and scores.dtype == torch.float32 and scores.is_contiguous()
+    if out_idx is None:
+        out_idx = torch.empty(k, dtype=torch.int32, device=scores.device)
+    st = stream if stream is not None else torch.cuda.current_stream(scores.device)
+    with torch.cuda.device(scores.device):
+        rc = load_library().ilre_topk_positions_noalloc(scores.data_ptr(), scores.numel(), k,
+                                                        out_idx.data_ptr(), st.cuda_stream)
+    if rc != 0:
+        raise IlreError(rc, "ilre_topk_positions_noalloc")
+    return out_idx
 
 
 class IlreRecall:
