@@ -44,7 +44,7 @@ __device__ __forceinline__ CtaItem decode_item(const QkParams& p) {
 
 // Common prologue: barrier init, TMEM allocation.  Returns the TMEM base address.
 __device__ __forceinline__ uint32_t cta_setup(SmemTail* tail, uint32_t smem_base, int stages,
-                                              int n_acc, int* status) {
+                                              int n_acc, int acc_readers, int* status) {
   const int warp = threadIdx.x >> 5;
   if (threadIdx.x == 0) {
     tail->abort_flag = 0;
@@ -59,7 +59,7 @@ __device__ __forceinline__ uint32_t cta_setup(SmemTail* tail, uint32_t smem_base
     }
     for (int b = 0; b < n_acc; ++b) {
       mbar_init(smem_u32(&tail->acc_full[b]), 1);
-      mbar_init(smem_u32(&tail->acc_empty[b]), kConsumerWarps);
+      mbar_init(smem_u32(&tail->acc_empty[b]), acc_readers);
     }
     fence_mbar_init();
   }
@@ -107,11 +107,56 @@ __device__ __forceinline__ void producer_loop(const CUtensorMap* tmapK, const CU
   }
 }
 
+// Sum over 32 logits of 2^(v * c2 + nm).  Of every 16 pairs, NPOLY take the polynomial on the
+// FMA pipe and the rest the special-function unit, so that both pipes work in parallel.
+template <int NPOLY>
+__device__ __forceinline__ float chunk_sum_exp2(const float (&v)[32], float c2, float nm) {
+  const float2 c2v = make_float2(c2, c2), nmv = make_float2(nm, nm);
+  float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+#pragma unroll
+  for (int pr = 0; pr < 16; ++pr) {
+    const float2 x = ffma2(make_float2(v[2 * pr], v[2 * pr + 1]), c2v, nmv);
+    float2 e;
+    if (((pr + 1) * NPOLY) / 16 > (pr * NPOLY) / 16) {
+      e = exp2_poly2(x);
+    } else {
+      e.x = ex2_approx(x.x);
+      e.y = ex2_approx(x.y);
+    }
+    if (pr & 1) acc1 = fadd2(acc1, e); else acc0 = fadd2(acc0, e);
+  }
+  return (acc0.x + acc0.y) + (acc1.x + acc1.y);
+}
+
+// Online (max, sum-exp) update of one query row with 32 more logits of the key tile.  Keys
+// past L (ragged last tile) become -inf: the special-function path maps them to 0 and the
+// polynomial's clamp to 2^-125, which vanishes against the row's sum (>= 1).
+template <int NPOLY>
+__device__ __forceinline__ void row_chunk_update(float (&v)[32], int col0, int valid, float c2,
+                                                 float& m, float& z) {
+  if (valid < kTileKeys) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (col0 + j >= valid) v[j] = -INFINITY;
+  }
+  float cm0 = fmax3(v[0], v[1], v[2]), cm1 = fmax3(v[3], v[4], v[5]);
+#pragma unroll
+  for (int j = 6; j < 30; j += 4) {
+    cm0 = fmax3(cm0, v[j], v[j + 1]);
+    cm1 = fmax3(cm1, v[j + 2], v[j + 3]);
+  }
+  const float m_new = fmaxf(fmax3(m, cm0, cm1), fmaxf(v[30], v[31]));
+  const float nm = -m_new * c2;
+  const float sum = chunk_sum_exp2<NPOLY>(v, c2, nm);
+  z = fmaf(z, ex2_approx((m - m_new) * c2), sum);
+  m = m_new;
+}
+
 // ---------------------------------------------------------------------------------------
 // Pass A: row statistics.  MT = number of 128-row tiles of the resident Q block.
 // ---------------------------------------------------------------------------------------
-template <int MT>
-__global__ void __launch_bounds__(kQkThreads, 1)
+template <int MT, int NPOLY>
+__global__ void __launch_bounds__(kStatsThreads, 1)
 row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
                  const __grid_constant__ CUtensorMap tmapQ, const QkParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -123,7 +168,7 @@ row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const CtaItem it = decode_item(p);
 
-  const uint32_t tmem_base = cta_setup(tail, smem_base, p.stages, 4, p.status);
+  const uint32_t tmem_base = cta_setup(tail, smem_base, p.stages, 4, 4, p.status);
   const bool run = (it.n_tiles > 0) && (*abort_flag == 0);
 
   if (warp == 0) {
@@ -160,79 +205,87 @@ row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
         umma_commit(smem_u32(&tail->k_empty[s]));
       }
     }
-  } else if (warp >= 4) {
-    const int wg = (warp - 4) >> 2;          // which 64-column half of every tile
+  } else if (warp >= 2) {
+    // Consumer warpgroups take the accumulator buffers in turn, so that they sit in different
+    // phases (waiting, loading, taking maxima, exponentials) and keep the special-function
+    // and FMA pipes fed.  Each thread owns one query row of the buffer and walks its 128
+    // columns in chunks of 32, loading the next chunk from tensor memory while it works on
+    // the current one.
+    const int wg = (warp - 2) >> 2;
     const int quad = warp & 3;               // TMEM lane quadrant this warp may read
     float m[MT], z[MT];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) { m[mt] = -1e30f; z[mt] = 0.f; }
     const float c2 = p.c2;
-    bool ok = run;
-    uint32_t u = 0;
-    for (int i = 0; i < it.n_tiles && ok; ++i) {
+    const uint32_t n_acc = run ? static_cast<uint32_t>(it.n_tiles) * MT : 0u;
+    // One copy of the loop body serves every (key tile, row tile): the warpgroups run at
+    // different places of the loop, and a body unrolled over the row tiles would not fit the
+    // instruction cache between them.
+#pragma unroll 1
+    for (uint32_t u = wg; u < n_acc; u += kStatsWarpgroups) {
+      const int i = static_cast<int>(u / MT), mt = static_cast<int>(u % MT);
       const long long key0 = static_cast<long long>(it.tile_begin + i) * kTileKeys;
       const int valid = static_cast<int>(min(static_cast<long long>(kTileKeys), p.L - key0));
+      const uint32_t b = u & 3u, use = u >> 2;
+      if (!mbar_wait(smem_u32(&tail->acc_full[b]), use & 1u, abort_flag, p.status,
+                     kDevWaitAccFull))
+        break;
+      tc_fence_after();
+      float mr = m[0], zr = z[0];
 #pragma unroll
-      for (int mt = 0; mt < MT; ++mt) {
-        if (!ok) break;
-        const uint32_t b = u & 3u, use = u >> 2;
-        ++u;
-        ok = mbar_wait(smem_u32(&tail->acc_full[b]), use & 1u, abort_flag, p.status,
-                       kDevWaitAccFull);
-        if (!ok) break;
-        tc_fence_after();
-        float v0[32], v1[32];
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + b * 128 + wg * 64;
-        tmem_ld32(taddr, v0);
-        tmem_ld32(taddr + 32, v1);
+      for (int j = 1; j < MT; ++j)
+        if (j == mt) { mr = m[j]; zr = z[j]; }
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + b * 128;
+      float va[32], vb[32];
+      tmem_ld32(taddr, va);
+      tmem_ld_wait();
+#pragma unroll 1
+      for (int h = 0; h < 2; ++h) {
+        tmem_ld32(taddr + 64 * h + 32, vb);
+        row_chunk_update<NPOLY>(va, 64 * h, valid, c2, mr, zr);
         tmem_ld_wait();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&tail->acc_empty[b]));
-        if (valid < kTileKeys) {              // ragged last tile: keys past L do not exist
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            if (wg * 64 + j >= valid) v0[j] = -INFINITY;
-            if (wg * 64 + 32 + j >= valid) v1[j] = -INFINITY;
-          }
+        if (h == 0) {
+          tmem_ld32(taddr + 64, va);
+        } else {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&tail->acc_empty[b]));
         }
-        float cm0 = v0[0], cm1 = v0[1], cm2 = v1[0], cm3 = v1[1];
-#pragma unroll
-        for (int j = 2; j < 32; j += 2) {
-          cm0 = fmaxf(cm0, v0[j]); cm1 = fmaxf(cm1, v0[j + 1]);
-          cm2 = fmaxf(cm2, v1[j]); cm3 = fmaxf(cm3, v1[j + 1]);
-        }
-        const float m_new = fmaxf(m[mt], fmaxf(fmaxf(cm0, cm1), fmaxf(cm2, cm3)));
-        const float nm = -m_new * c2;
-        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-        for (int j = 0; j < 32; j += 2) {
-          s0 += ex2_approx(fmaf(v0[j], c2, nm));
-          s1 += ex2_approx(fmaf(v0[j + 1], c2, nm));
-          s2 += ex2_approx(fmaf(v1[j], c2, nm));
-          s3 += ex2_approx(fmaf(v1[j + 1], c2, nm));
-        }
-        z[mt] = z[mt] * ex2_approx((m[mt] - m_new) * c2) + ((s0 + s1) + (s2 + s3));
-        m[mt] = m_new;
+        row_chunk_update<NPOLY>(vb, 64 * h + 32, valid, c2, mr, zr);
+        if (h == 0) tmem_ld_wait();
       }
+#pragma unroll
+      for (int j = 0; j < MT; ++j)
+        if (j == mt) { m[j] = mr; z[j] = zr; }
     }
-    // Merge the two column halves through shared memory (the K stages are idle by now) and
-    // write this CTA's partial statistics: (max in log2 units, sum).
+    // Merge the warpgroups' statistics through shared memory and write this CTA's partial
+    // statistics: (max in log2 units, sum).  The scratch aliases the first K stage, which is
+    // idle once every warpgroup has read its last accumulator (every MMA, hence every TMA
+    // load, has completed by then).
     float2* scratch = reinterpret_cast<float2*>(smem + MT * 128 * 256);
     const int row_in_tile = quad * 32 + lane;
-    if (wg == 1) {
+    asm volatile("bar.sync 1, %0;" ::"r"(kStatsConsumerWarps * 32) : "memory");
+    if (wg > 0) {
 #pragma unroll
-      for (int mt = 0; mt < MT; ++mt) scratch[mt * 128 + row_in_tile] = make_float2(m[mt], z[mt]);
+      for (int mt = 0; mt < MT; ++mt)
+        scratch[((wg - 1) * MT + mt) * 128 + row_in_tile] = make_float2(m[mt], z[mt]);
     }
-    asm volatile("bar.sync 1, %0;" ::"r"(kConsumerWarps * 32) : "memory");
+    asm volatile("bar.sync 1, %0;" ::"r"(kStatsConsumerWarps * 32) : "memory");
     if (wg == 0) {
       float2* out = reinterpret_cast<float2*>(p.partial) +
                     (static_cast<size_t>(it.group) * p.cpg + it.chunk) * (MT * 128);
 #pragma unroll
       for (int mt = 0; mt < MT; ++mt) {
-        const float2 o = scratch[mt * 128 + row_in_tile];
-        const float mm = fmaxf(m[mt], o.x);
-        const float zz = z[mt] * exp2f((m[mt] - mm) * c2) + o.y * exp2f((o.x - mm) * c2);
+        float mm = m[mt];
+#pragma unroll
+        for (int w = 1; w < kStatsWarpgroups; ++w)
+          mm = fmaxf(mm, scratch[((w - 1) * MT + mt) * 128 + row_in_tile].x);
+        float zz = z[mt] * exp2f((m[mt] - mm) * c2);
+#pragma unroll
+        for (int w = 1; w < kStatsWarpgroups; ++w) {
+          const float2 o = scratch[((w - 1) * MT + mt) * 128 + row_in_tile];
+          zz += o.y * exp2f((o.x - mm) * c2);
+        }
         out[mt * 128 + row_in_tile] = make_float2(mm * c2, zz);
       }
     }
@@ -259,7 +312,7 @@ scores_kernel(const __grid_constant__ CUtensorMap tmapK,
 
   for (int i = threadIdx.x; i < p.rb_rows; i += blockDim.x)
     nl[i] = p.nlse2[static_cast<size_t>(it.group) * p.rb_rows + i];
-  const uint32_t tmem_base = cta_setup(tail, smem_base, p.stages, 2, p.status);
+  const uint32_t tmem_base = cta_setup(tail, smem_base, p.stages, 2, kConsumerWarps, p.status);
   const bool run = (it.n_tiles > 0) && (*abort_flag == 0);
 
   if (warp == 0) {
@@ -438,10 +491,10 @@ template <int MT>
 static cudaError_t launch_row_stats_mt(const CUtensorMap& tk, const CUtensorMap& tq,
                                        const QkParams& p, cudaStream_t st) {
   const size_t smem = row_stats_smem_bytes(MT * 128, p.stages);
-  cudaError_t e = cudaFuncSetAttribute(row_stats_kernel<MT>,
+  cudaError_t e = cudaFuncSetAttribute(row_stats_kernel<MT, kRowStatsPolyPairs>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  row_stats_kernel<MT><<<p.n_groups * p.cpg, kQkThreads, smem, st>>>(tk, tq, p);
+  row_stats_kernel<MT, kRowStatsPolyPairs><<<p.n_groups * p.cpg, kStatsThreads, smem, st>>>(tk, tq, p);
   return cudaGetLastError();
 }
 

@@ -11,10 +11,25 @@ static constexpr int kTileKeys = 128;              // keys per K tile (one TMA s
 static constexpr int kStageBytes = kTileKeys * kHeadDim * 2;
 static constexpr int kMaxStages = 6;
 static constexpr int kMaxRbRows = 512;             // query rows resident in shared memory
-static constexpr int kQkThreads = 384;             // warp 0 TMA, warp 1 MMA, warps 4..11 consumers
+static constexpr int kQkThreads = 384;             // scores: warp 0 TMA, warp 1 MMA, warps 4..11 consumers
 static constexpr int kConsumerWarps = 8;
+// Row statistics: warp 0 TMA, warp 1 MMA, then kStatsWarpgroups consumer warpgroups of four
+// warps (one per TMEM lane quadrant); accumulator buffer u belongs to warpgroup u % kStatsWarpgroups.
+#ifndef ILRE_STATS_WARPGROUPS
+#define ILRE_STATS_WARPGROUPS 4
+#endif
+static constexpr int kStatsWarpgroups = ILRE_STATS_WARPGROUPS;
+static constexpr int kStatsConsumerWarps = 4 * kStatsWarpgroups;
+static constexpr int kStatsThreads = 64 + 32 * kStatsConsumerWarps;
 static constexpr int kSmemTailBytes = 256;
 static constexpr int kMaxDynSmem = 232448;         // 227 KB per CTA on sm_100
+
+// Row statistics: how many of every 16 logit pairs take 2^x from the FMA-pipe polynomial
+// instead of the special-function unit (0 = none).  Balances the two pipes.
+#ifndef ILRE_ROW_STATS_POLY_PAIRS
+#define ILRE_ROW_STATS_POLY_PAIRS 6
+#endif
+static constexpr int kRowStatsPolyPairs = ILRE_ROW_STATS_POLY_PAIRS;
 
 // Geometry of one recall, shared by both passes.
 struct QkParams {

@@ -159,6 +159,53 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
+// ---- packed fp32 arithmetic (two lanes per instruction) and three-input max ----
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+  float2 d;
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d.x), "=f"(d.y)
+      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+  return d;
+}
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
+  float2 d;
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "add.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d.x), "=f"(d.y)
+      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return d;
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
+// 2^x for two values on the FMA pipe instead of the special-function unit: round-to-nearest
+// split x = n + r with |r| <= 1/2 (adding 1.5 * 2^23 leaves n in the low mantissa bits), a
+// degree-4 minimax polynomial for 2^r (relative error 2.7e-6 in fp32), and n added into the
+// exponent field.  Inputs are clamped at -125 so the result stays a normal number.
+__device__ __forceinline__ float2 exp2_poly2(float2 x) {
+  const float kMagic = 12582912.f;
+  x.x = fmaxf(x.x, -125.f);
+  x.y = fmaxf(x.y, -125.f);
+  const float2 t = fadd2(x, make_float2(kMagic, kMagic));
+  const float2 n = fadd2(t, make_float2(-kMagic, -kMagic));
+  const float2 r = ffma2(n, make_float2(-1.f, -1.f), x);
+  float2 p = ffma2(r, make_float2(0.009570102f, 0.009570102f),
+                   make_float2(0.05591786f, 0.05591786f));
+  p = ffma2(p, r, make_float2(0.24024744f, 0.24024744f));
+  p = ffma2(p, r, make_float2(0.6931218f, 0.6931218f));
+  p = ffma2(p, r, make_float2(0.9999993f, 0.9999993f));
+  float2 e;
+  e.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23));
+  e.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23));
+  return e;
+}
+
 // Order-preserving map float -> uint32 (larger float <=> larger uint) and back.
 __host__ __device__ __forceinline__ uint32_t float_to_ordered(float f) {
   uint32_t b;
