@@ -127,8 +127,8 @@ int ilre_recall_status(ilre_recall_t* h);
  * n entries, each the mean over the recorded runs (milliseconds), in this order:
  *   0 prepare (query packing, clears)   1 row statistics (QK^T + online softmax)
  *   2 statistics merge                  3 scores (QK^T + max over rows)
- *   4 pooling                           5 top-K_m selection and ranking
- *   6 allocation and ascending output
+ *   4 Algorithm 1 (A^C from the maxima, pooling, top-K_m selection and ranking, allocation,
+ *     ascending output; one kernel)
  * Returns the number of entries written, or a negative status.
  */
 int ilre_recall_set_profiling(ilre_recall_t* h, int32_t on);

@@ -22,7 +22,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-constexpr int kNumStages = 7;            // timed stages (see ilre_recall_stage_times)
+constexpr int kNumStages = 5;            // timed stages (see ilre_recall_stage_times)
 constexpr int kProfRing = 32;            // runs whose stage events are kept for averaging
 constexpr int kMaxSinkStaging = 65536;
 
@@ -48,7 +48,7 @@ struct ilre_recall {
   unsigned long long* sel_prefix;
   uint32_t* sel_krem;
   uint32_t* sel_done;
-  uint32_t* sel_ticket;
+  uint32_t* grid_barrier;
   unsigned long long* cand;
   uint32_t* cand_count;
   int* ranked;
@@ -66,6 +66,7 @@ struct ilre_recall {
   int last_q_len;
   cudaStream_t last_stream;
   int cand_stride;
+  int select_max_grid;                  // co-resident CTAs of the selection kernel
 };
 
 namespace {
@@ -114,7 +115,7 @@ bool dev_alloc(T** p, size_t count) {
 void free_all(ilre_recall* h) {
   cudaFree(h->qp); cudaFree(h->partial); cudaFree(h->nlse2); cudaFree(h->row_lse);
   cudaFree(h->enc); cudaFree(h->scores); cudaFree(h->pooled); cudaFree(h->hist);
-  cudaFree(h->sel_prefix); cudaFree(h->sel_krem); cudaFree(h->sel_done); cudaFree(h->sel_ticket);
+  cudaFree(h->sel_prefix); cudaFree(h->sel_krem); cudaFree(h->sel_done); cudaFree(h->grid_barrier);
   cudaFree(h->cand); cudaFree(h->cand_count); cudaFree(h->ranked); cudaFree(h->bitmap);
   cudaFree(h->status); cudaFree(h->stage_k); cudaFree(h->stage_q); cudaFree(h->stage_idx);
   for (int r = 0; r < kProfRing; ++r)
@@ -225,7 +226,7 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out) {
   ok = ok && dev_alloc(&h->sel_prefix, ncomb);
   ok = ok && dev_alloc(&h->sel_krem, ncomb);
   ok = ok && dev_alloc(&h->sel_done, ncomb);
-  ok = ok && dev_alloc(&h->sel_ticket, ncomb);
+  ok = ok && dev_alloc(&h->grid_barrier, 1);
   ok = ok && dev_alloc(&h->cand, ncomb * h->cand_stride);
   ok = ok && dev_alloc(&h->cand_count, ncomb);
   ok = ok && dev_alloc(&h->ranked, ncomb * h->cand_stride);
@@ -241,6 +242,8 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out) {
     for (int i = 0; ok && i <= kNumStages; ++i)
       ok = (cudaEventCreate(&h->ev[r][i]) == cudaSuccess);
   if (ok) ok = (cudaMemset(h->status, 0, sizeof(int)) == cudaSuccess);
+  if (ok) ok = (cudaMemset(h->grid_barrier, 0, sizeof(uint32_t)) == cudaSuccess);
+  if (ok) ok = (select_max_grid(h->n_sm, &h->select_max_grid) == cudaSuccess);
   if (ok) ok = (cudaDeviceSynchronize() == cudaSuccess);
   if (!ok) {
     cudaGetLastError();
@@ -267,7 +270,6 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
   ComboTable tbl;
   std::memset(&tbl, 0, sizeof(tbl));
   const long long Lp = L - spec->n_sink;
-  int max_len = 0, max_km = 1;
   tbl.n_comb = (budget > 0) ? spec->n_max * spec->n_win : 0;
   for (int i = 0, c = 0; i < spec->n_max && tbl.n_comb; ++i)
     for (int j = 0; j < spec->n_win; ++j, ++c) {
@@ -280,8 +282,7 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
       tbl.len[c] = static_cast<int>(len);
       tbl.k_m[c] = static_cast<int>(km);
       tbl.quota[c] = budget / tbl.n_comb + (c < budget % tbl.n_comb ? 1 : 0);
-      if (len > max_len) max_len = static_cast<int>(len);
-      if (km > max_km) max_km = static_cast<int>(km);
+      tbl.tile_begin[c + 1] = tbl.tile_begin[c] + static_cast<int>((len + kSelTile - 1) / kSelTile);
     }
 
   CUtensorMap map_k, map_q;
@@ -305,7 +306,7 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
   pp.n_comb = tbl.n_comb;
   for (int c = 0; c < tbl.n_comb; ++c) pp.k_m[c] = tbl.k_m[c];
   pp.sel_prefix = h->sel_prefix; pp.sel_krem = h->sel_krem; pp.sel_done = h->sel_done;
-  pp.sel_ticket = h->sel_ticket; pp.cand_count = h->cand_count;
+  pp.cand_count = h->cand_count; pp.grid_barrier = h->grid_barrier;
 
   MergeParams mp;
   mp.n_groups = g.n_groups; mp.n_rb = g.n_rb; mp.rb_rows = g.rb_rows; mp.cpg = g.cpg;
@@ -314,12 +315,25 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
 
   SelectParams sp;
   std::memset(&sp, 0, sizeof(sp));
-  sp.scores = h->scores; sp.L = L; sp.n_sink = spec->n_sink; sp.win_op = spec->win_op;
+  sp.enc = h->enc; sp.scores = h->scores; sp.user_scores = out_scores_dev;
+  sp.L = L; sp.n_sink = spec->n_sink; sp.win_op = spec->win_op;
   sp.pooled = h->pooled; sp.pooled_stride = h->cfg.max_L; sp.hist = h->hist;
   sp.sel_prefix = h->sel_prefix; sp.sel_krem = h->sel_krem; sp.sel_done = h->sel_done;
-  sp.sel_ticket = h->sel_ticket; sp.cand = h->cand; sp.cand_stride = h->cand_stride;
+  sp.cand = h->cand; sp.cand_stride = h->cand_stride;
   sp.cand_count = h->cand_count; sp.ranked = h->ranked; sp.bitmap = h->bitmap;
-  sp.out_idx = out_idx_dev; sp.budget = budget; sp.status = h->status;
+  sp.out_idx = out_idx_dev; sp.budget = budget; sp.barrier = h->grid_barrier;
+  sp.status = h->status;
+  const size_t select_smem = select_smem_bytes(L, &sp.bitmap_in_smem);
+  // Grid of the selection kernel: enough CTAs for the scan tiles and for the ranking
+  // (K_m^2 comparisons per combination), but no more, since every grid barrier pays for them.
+  long long want_grid = tbl.tile_begin[tbl.n_comb];
+  long long rank_items = 0;
+  for (int c = 0; c < tbl.n_comb; ++c)
+    rank_items += (tbl.k_m[c] + kRankKeysPerItem - 1) / kRankKeysPerItem;
+  if (rank_items / 4 > want_grid) want_grid = rank_items / 4;
+  if (want_grid < 1) want_grid = 1;
+  if (want_grid > h->select_max_grid) want_grid = h->select_max_grid;
+  const int select_grid = static_cast<int>(want_grid);
 
   const bool prof = h->profiling != 0;
   int launches = 0;
@@ -336,22 +350,9 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
   ILRE_CUDA(launch_merge_stats(mp, st)); ++launches;
   ILRE_MARK(3);
   ILRE_CUDA(launch_scores(map_k, map_q, qk, st)); ++launches;
-  ILRE_CUDA(launch_finalize_scores(h->enc, h->scores, out_scores_dev, L, st)); ++launches;
   ILRE_MARK(4);
-  if (tbl.n_comb > 0) {
-    ILRE_CUDA(launch_pool(tbl, sp, max_len, st)); ++launches;
-  }
+  ILRE_CUDA(launch_select(tbl, sp, select_grid, select_smem, st)); ++launches;
   ILRE_MARK(5);
-  if (tbl.n_comb > 0) {
-    for (int pass = 0; pass < kSelectPasses; ++pass) {
-      ILRE_CUDA(launch_select_pass(tbl, sp, max_len, pass, st)); ++launches;
-    }
-    ILRE_CUDA(launch_gather(tbl, sp, max_len, st)); ++launches;
-    ILRE_CUDA(launch_rank_sort(tbl, sp, max_km, st)); ++launches;
-  }
-  ILRE_MARK(6);
-  ILRE_CUDA(launch_allocate(tbl, sp, st)); ++launches;
-  ILRE_MARK(7);
 #undef ILRE_MARK
   h->last_launches = launches;
   if (prof) ++h->prof_runs;

@@ -433,11 +433,11 @@ __global__ void prepare_kernel(const uint4* __restrict__ q, uint4* __restrict__ 
   }
   for (long long e = tid; e < static_cast<long long>(p.n_comb) * p.hist_bins; e += nthreads)
     p.hist[e] = 0u;
+  if (tid == 0) *p.grid_barrier = 0u;
   for (long long c = tid; c < p.n_comb; c += nthreads) {
     p.sel_prefix[c] = 0ull;
     p.sel_krem[c] = static_cast<uint32_t>(p.k_m[c]);
     p.sel_done[c] = 0u;
-    p.sel_ticket[c] = 0u;
     p.cand_count[c] = 0u;
   }
 }
@@ -464,16 +464,6 @@ __global__ void merge_stats_kernel(MergeParams p) {
   p.nlse2[prow] = -lse2;
   const int i = rg / p.group_size, j = rg % p.group_size;
   p.row_lse[i * p.n_q + g * p.group_size + j] = lse2 * 0.69314718055994530942f;
-}
-
-// A^C[t] = exp2(max_r log2 p_rt): decode the atomically-maximised value, one exp per position.
-__global__ void finalize_scores_kernel(const uint32_t* __restrict__ enc, float* __restrict__ scores,
-                                       float* __restrict__ user_scores, long long L) {
-  const long long t = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (t >= L) return;
-  const float a = exp2f(ordered_to_float(enc[t]));
-  scores[t] = a;
-  if (user_scores) user_scores[t] = a;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -528,13 +518,6 @@ cudaError_t launch_prepare(const void* q, void* qp, const PrepParams& p, int n_s
 cudaError_t launch_merge_stats(const MergeParams& p, cudaStream_t st) {
   const int n = p.n_groups * p.rb_rows;
   merge_stats_kernel<<<(n + 127) / 128, 128, 0, st>>>(p);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_finalize_scores(const uint32_t* enc, float* scores, float* user_scores,
-                                   long long L, cudaStream_t st) {
-  finalize_scores_kernel<<<static_cast<unsigned>((L + 255) / 256), 256, 0, st>>>(enc, scores,
-                                                                                user_scores, L);
   return cudaGetLastError();
 }
 

@@ -27,7 +27,7 @@ static constexpr int kMaxDynSmem = 232448;         // 227 KB per CTA on sm_100
 // Row statistics: how many of every 16 logit pairs take 2^x from the FMA-pipe polynomial
 // instead of the special-function unit (0 = none).  Balances the two pipes.
 #ifndef ILRE_ROW_STATS_POLY_PAIRS
-#define ILRE_ROW_STATS_POLY_PAIRS 6
+#define ILRE_ROW_STATS_POLY_PAIRS 4
 #endif
 static constexpr int kRowStatsPolyPairs = ILRE_ROW_STATS_POLY_PAIRS;
 
@@ -60,8 +60,8 @@ struct PrepParams {
   unsigned long long* sel_prefix;
   uint32_t* sel_krem;
   uint32_t* sel_done;
-  uint32_t* sel_ticket;
   uint32_t* cand_count;
+  uint32_t* grid_barrier;   // arrival counter of the selection kernel's grid barrier
 };
 
 struct MergeParams {
@@ -80,7 +80,5 @@ cudaError_t launch_row_stats(const CUtensorMap& tk, const CUtensorMap& tq, const
 cudaError_t launch_merge_stats(const MergeParams& p, cudaStream_t st);
 cudaError_t launch_scores(const CUtensorMap& tk, const CUtensorMap& tq, const QkParams& p,
                           cudaStream_t st);
-cudaError_t launch_finalize_scores(const uint32_t* enc, float* scores, float* user_scores,
-                                   long long L, cudaStream_t st);
 
 }  // namespace ilre

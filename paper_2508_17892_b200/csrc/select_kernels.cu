@@ -1,74 +1,42 @@
-// Algorithm 1 ("Context Allocation") on the device.
+// Algorithm 1 ("Context Allocation") on the device, as ONE cooperative kernel whose CTAs
+// meet at grid barriers between the phases:
 //
-//   pool_kernel        MaxPooling(size = stride = m) fused with the stride-1 window pooling
-//                      (average or max) of every (m, n) combination;
-//   select_pass_kernel radix select of the K_m largest 64-bit keys (pooled value, then lower
-//                      cell index first), 11/11/10 bits per pass, all combinations at once;
-//   gather_kernel      collects the selected keys;
-//   rank_sort_kernel   orders them (value descending, cell ascending);
-//   allocate_kernel    walks the combinations in loop order: maps cells back to tokens, skips
-//                      tokens already allocated, stops each combination at its quota B_c, then
-//                      writes the allocated positions in ascending order.
+//   A  A^C[t] = exp2(max_r log2 p_rt) from the scores pass' encoded maxima (Eq. 5);
+//   B  MaxPooling(size = stride = m) fused with the stride-1 window pooling (average or max)
+//      of every (m, n) combination, and the first radix histogram;
+//   C  radix select of the K_m largest 64-bit keys (pooled value, then lower cell index
+//      first), 11/11/10 bits per pass, all combinations at once; passes stop as soon as every
+//      combination's threshold is settled;
+//   D  gather of the selected keys;
+//   E  ranking (value descending, cell ascending) by counting, spread over the grid;
+//   F  one CTA walks the combinations in loop order: maps cells back to tokens, skips tokens
+//      already allocated, stops each combination at its quota B_c, then writes the allocated
+//      positions in ascending order.
+//
+// Work of phases B-D is cut into tiles of kSelTile cells of one combination; every CTA owns a
+// contiguous run of tiles, the same in every phase.
 #include "select_kernels.cuh"
 #include "sm100_ptx.cuh"
+
+// Build with -DILRE_SELECT_TRACE to have CTA 0 print the time spent in every phase.
+#ifdef ILRE_SELECT_TRACE
+#include <cstdio>
+#define SEL_TRACE(tag)                                                              \
+  do {                                                                              \
+    if (blockIdx.x == 0 && threadIdx.x == 0 && trace_n < 32) {                      \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(trace_t[trace_n]));          \
+      trace_tag[trace_n++] = tag;                                                   \
+    }                                                                               \
+  } while (0)
+#else
+#define SEL_TRACE(tag) do { } while (0)
+#endif
 
 namespace ilre {
 
 __device__ __forceinline__ unsigned long long make_key(float w, uint32_t cell) {
   return (static_cast<unsigned long long>(float_to_ordered(w)) << 32) | (0xFFFFFFFFu - cell);
 }
-
-// ---------------------------------------------------------------------------------------
-// pooling
-// ---------------------------------------------------------------------------------------
-static constexpr int kPoolTile = 1024;
-static constexpr int kPoolThreads = 256;
-
-__global__ void __launch_bounds__(kPoolThreads)
-pool_kernel(const ComboTable tbl, const SelectParams p) {
-  __shared__ float cells[kPoolTile + kMaxWin];
-  const int combo = blockIdx.y;
-  const int m = tbl.m[combo], n = tbl.n[combo], len = tbl.len[combo];
-  const int c0 = blockIdx.x * kPoolTile;
-  if (c0 >= len) return;
-  const long long Lp = p.L - p.n_sink;                     // scores without the sink part
-  const float* a = p.scores + p.n_sink;
-  const int lo = c0 - n / 2;
-  const int span = min(kPoolTile, len - c0) + n - 1;
-  const float pad = (p.win_op == 0) ? 0.f : -INFINITY;
-  for (int idx = threadIdx.x; idx < span; idx += kPoolThreads) {
-    const int u = lo + idx;
-    float v = pad;
-    if (u >= 0 && u < len) {
-      const long long t0 = static_cast<long long>(u) * m;
-      const long long t1 = min(t0 + m, Lp);
-      v = a[t0];
-      for (long long t = t0 + 1; t < t1; ++t) v = fmaxf(v, a[t]);
-    }
-    cells[idx] = v;
-  }
-  __syncthreads();
-  float* out = p.pooled + static_cast<long long>(combo) * p.pooled_stride;
-  const int n_out = min(kPoolTile, len - c0);
-  for (int i = threadIdx.x; i < n_out; i += kPoolThreads) {
-    float acc;
-    if (p.win_op == 0) {
-      acc = 0.f;
-      for (int j = 0; j < n; ++j) acc += cells[i + j];
-      acc = acc / static_cast<float>(n);
-    } else {
-      acc = cells[i];
-      for (int j = 1; j < n; ++j) acc = fmaxf(acc, cells[i + j]);
-    }
-    out[c0 + i] = acc;
-  }
-}
-
-// ---------------------------------------------------------------------------------------
-// radix select
-// ---------------------------------------------------------------------------------------
-static constexpr int kSelThreads = 512;
-static constexpr int kSelItemsPerThread = 16;
 
 __device__ __forceinline__ void pass_bits(int pass, int& shift, int& bits) {
   const int sh[kSelectPasses] = {53, 42, 32, 21, 10, 0};
@@ -77,152 +45,42 @@ __device__ __forceinline__ void pass_bits(int pass, int& shift, int& bits) {
   bits = bt[pass];
 }
 
-__global__ void __launch_bounds__(kSelThreads)
-select_pass_kernel(const ComboTable tbl, const SelectParams p, const int pass) {
-  __shared__ uint32_t sh_hist[kHistBins];
-  __shared__ uint32_t sh_warp[kSelThreads / 32];
-  __shared__ int sh_last;
-  const int combo = blockIdx.y;
-  if (p.sel_done[combo]) return;
-  const int len = tbl.len[combo];
-  int shift, bits;
-  pass_bits(pass, shift, bits);
-  const unsigned long long prefix = p.sel_prefix[combo];
-  const uint32_t mask = (1u << bits) - 1u;
-  for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) sh_hist[b] = 0u;
-  __syncthreads();
+struct SelShared {
+  uint32_t hist[kHistBins];
+  uint32_t scan[33];
+  int flag;
+  unsigned long long prefix[kMaxCombos];   // per combination: radix prefix found so far
+  uint32_t state[kMaxCombos];              // per combination: threshold settled / candidate count
+};
 
-  const float* w = p.pooled + static_cast<long long>(combo) * p.pooled_stride;
-  const int per_block = (len + gridDim.x - 1) / gridDim.x;
-  const int begin = blockIdx.x * per_block;
-  const int end = min(len, begin + per_block);
-  const int lane = threadIdx.x & 31;
-  for (int base = begin; base < end; base += kSelThreads) {
-    const int c = base + threadIdx.x;
-    uint32_t digit = 0xFFFFFFFFu;                          // sentinel: does not take part
-    if (c < end) {
-      const unsigned long long key = make_key(w[c], static_cast<uint32_t>(c));
-      if (pass == 0 || ((key ^ prefix) >> (shift + bits)) == 0ull)
-        digit = static_cast<uint32_t>(key >> shift) & mask;
-    }
-    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, digit);
-    if (digit != 0xFFFFFFFFu && lane == __ffs(peers) - 1) atomicAdd(&sh_hist[digit], __popc(peers));
-  }
-  __syncthreads();
-  uint32_t* gh = p.hist + static_cast<long long>(combo) * kHistBins;
-  for (int b = threadIdx.x; b < kHistBins; b += kSelThreads)
-    if (sh_hist[b]) atomicAdd(&gh[b], sh_hist[b]);
-  __threadfence();
+// Grid-wide barrier (all CTAs are co-resident: cooperative launch).  The arrival counter is
+// zero when the kernel starts and only grows: the k-th barrier completes when it reaches
+// k * gridDim.x.  The wait is bounded; a CTA that gives up records it and leaves the kernel.
+__device__ __forceinline__ bool grid_sync(const SelectParams& p, SelShared* sh, uint32_t& epoch) {
+  ++epoch;
   __syncthreads();
   if (threadIdx.x == 0) {
-    const uint32_t t = atomicAdd(&p.sel_ticket[combo], 1u);
-    sh_last = (t == gridDim.x - 1);
-  }
-  __syncthreads();
-  if (!sh_last) return;
-  __threadfence();
-
-  // Last block of this combination: locate the bin that holds the k-th largest key.
-  const uint32_t k_rem = p.sel_krem[combo];
-  uint32_t h[4];
-  uint32_t total = 0;
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    h[j] = __ldcg(&gh[kHistBins - 1 - (4 * threadIdx.x + j)]);   // bins in descending order
-    total += h[j];
-  }
-  uint32_t incl = total;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-    if (lane >= o) incl += v;
-  }
-  const int warp = threadIdx.x >> 5;
-  if (lane == 31) sh_warp[warp] = incl;
-  __syncthreads();
-  uint32_t warp_off = 0;
-  for (int wv = 0; wv < warp; ++wv) warp_off += sh_warp[wv];
-  const uint32_t excl = warp_off + incl - total;
-  if (excl < k_rem && k_rem <= excl + total) {
-    uint32_t cum = excl;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if (k_rem > cum && k_rem <= cum + h[j]) {
-        const uint32_t bin = kHistBins - 1 - (4 * threadIdx.x + j);
-        const uint32_t new_k = k_rem - cum;
-        p.sel_prefix[combo] = prefix | (static_cast<unsigned long long>(bin) << shift);
-        p.sel_krem[combo] = new_k;
-        p.sel_done[combo] = (h[j] == new_k || pass == kSelectPasses - 1) ? 1u : 0u;
+    int ok = 1;
+    const uint32_t target = epoch * gridDim.x;
+    __threadfence();
+    atomicAdd(p.barrier, 1u);
+    volatile uint32_t* arrivals = p.barrier;
+    const long long t0 = clock64();
+    for (uint32_t it = 1; *arrivals < target; ++it) {
+      if ((it & 0xFF) == 0 && clock64() - t0 > kWaitCycleLimit) {
+        atomicCAS(p.status, 0, kDevGridBarrier);
+        ok = 0;
+        break;
       }
-      cum += h[j];
     }
+    __threadfence();
+    sh->flag = ok;
   }
-  uint32_t grand = 0;
-  for (int wv = 0; wv < kSelThreads / 32; ++wv) grand += sh_warp[wv];
-  if (threadIdx.x == 0) {
-    if (k_rem > grand || k_rem == 0) p.sel_done[combo] = 1u;   // fewer keys than asked: take all
-    p.sel_ticket[combo] = 0u;
-  }
-  for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) gh[b] = 0u;
-}
-
-__global__ void __launch_bounds__(kSelThreads)
-gather_kernel(const ComboTable tbl, const SelectParams p) {
-  const int combo = blockIdx.y;
-  const int len = tbl.len[combo];
-  const unsigned long long threshold = p.sel_prefix[combo];
-  const float* w = p.pooled + static_cast<long long>(combo) * p.pooled_stride;
-  unsigned long long* cand = p.cand + static_cast<long long>(combo) * p.cand_stride;
-  const int per_block = (len + gridDim.x - 1) / gridDim.x;
-  const int begin = blockIdx.x * per_block;
-  const int end = min(len, begin + per_block);
-  for (int c = begin + threadIdx.x; c < end; c += kSelThreads) {
-    const unsigned long long key = make_key(w[c], static_cast<uint32_t>(c));
-    if (key >= threshold) {
-      const uint32_t pos = atomicAdd(&p.cand_count[combo], 1u);
-      if (pos < static_cast<uint32_t>(tbl.k_m[combo])) cand[pos] = key;
-    }
-  }
-}
-
-// ---------------------------------------------------------------------------------------
-// ranking: bitonic sort of <= kMaxKm keys, descending
-// ---------------------------------------------------------------------------------------
-static constexpr int kSortThreads = 1024;
-
-__global__ void __launch_bounds__(kSortThreads)
-rank_sort_kernel(const ComboTable tbl, const SelectParams p, const int pow2) {
-  extern __shared__ unsigned long long keys[];
-  const int combo = blockIdx.x;
-  const int n = min(static_cast<int>(min(p.cand_count[combo], static_cast<uint32_t>(kMaxKm))),
-                    tbl.k_m[combo]);
-  const unsigned long long* cand = p.cand + static_cast<long long>(combo) * p.cand_stride;
-  for (int i = threadIdx.x; i < pow2; i += kSortThreads) keys[i] = (i < n) ? cand[i] : 0ull;
   __syncthreads();
-  for (int k = 2; k <= pow2; k <<= 1) {
-    for (int j = k >> 1; j > 0; j >>= 1) {
-      for (int i = threadIdx.x; i < pow2; i += kSortThreads) {
-        const int x = i ^ j;
-        if (x > i) {
-          const unsigned long long a = keys[i], b = keys[x];
-          const bool descending_block = ((i & k) == 0);
-          if (descending_block ? (a < b) : (a > b)) { keys[i] = b; keys[x] = a; }
-        }
-      }
-      __syncthreads();
-    }
-  }
-  int* ranked = p.ranked + static_cast<long long>(combo) * p.cand_stride;
-  for (int i = threadIdx.x; i < n; i += kSortThreads)
-    ranked[i] = static_cast<int>(0xFFFFFFFFu - static_cast<uint32_t>(keys[i] & 0xFFFFFFFFull));
+  return sh->flag != 0;
 }
 
-// ---------------------------------------------------------------------------------------
-// allocation
-// ---------------------------------------------------------------------------------------
-static constexpr int kAllocThreads = 1024;
-
-// Exclusive prefix sum over the block; *total receives the block sum.
+// Exclusive prefix sum over the block of kSelThreads threads; *total receives the block sum.
 __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* sh_warp,
                                                          uint32_t* total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -251,118 +109,547 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s
   return sh_warp[warp] + incl - v;
 }
 
-__global__ void __launch_bounds__(kAllocThreads)
-allocate_kernel(const ComboTable tbl, const SelectParams p) {
-  __shared__ uint32_t sh_warp[33];
+// Adds one digit per thread (0xFFFFFFFF = none) to the shared histogram, one atomic per
+// distinct digit of the warp: plateaus of equal pooled values are the common case.
+__device__ __forceinline__ void hist_add(uint32_t* hist, uint32_t digit) {
+  if (!__any_sync(0xFFFFFFFFu, digit != 0xFFFFFFFFu)) return;
+  const uint32_t peers = __match_any_sync(0xFFFFFFFFu, digit);
+  if (digit != 0xFFFFFFFFu && (threadIdx.x & 31) == __ffs(peers) - 1)
+    atomicAdd(&hist[digit], __popc(peers));
+}
+
+__device__ __forceinline__ void hist_flush(uint32_t* sh_hist, uint32_t* gh) {
+  __syncthreads();
+  for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) {
+    const uint32_t v = sh_hist[b];
+    if (v) { atomicAdd(&gh[b], v); sh_hist[b] = 0u; }
+  }
+  __syncthreads();
+}
+
+__device__ __forceinline__ int combo_of_tile(const ComboTable& tbl, int tile) {
+  int c = 0;
+  while (c + 1 < tbl.n_comb && tile >= tbl.tile_begin[c + 1]) ++c;
+  return c;
+}
+
+static constexpr int kTilePer = kSelTile / kSelThreads;
+static constexpr int kScanGroup = 4;      // tiles whose loads are issued together
+
+// Pooled values of one tile, kTilePer per thread, all loads in flight together.
+__device__ __forceinline__ void fetch_tile(const ComboTable& tbl, const SelectParams& p, int tile,
+                                           const uint32_t* skip, float (&wv)[kTilePer]) {
+  const int combo = combo_of_tile(tbl, tile);
+  if (skip && skip[combo]) return;
+  const float* w = p.pooled + static_cast<long long>(combo) * p.pooled_stride;
+  const int c0 = (tile - tbl.tile_begin[combo]) * kSelTile;
+  const int c1 = min(tbl.len[combo], c0 + kSelTile);
+#pragma unroll
+  for (int k = 0; k < kTilePer; ++k) {
+    const int c = c0 + k * kSelThreads + threadIdx.x;
+    wv[k] = (c < c1) ? __ldcg(&w[c]) : 0.f;
+  }
+}
+
+// Phase B for one tile: pooled cells [c0, c0 + n_out) of `combo`, written to p.pooled; the
+// first-pass radix digit of every cell goes to the shared histogram.  `buf0`/`buf1` hold
+// kSelTile + kMaxWin floats each.
+__device__ __forceinline__ void pool_tile(const ComboTable& tbl, const SelectParams& p, int combo,
+                                          int c0, float* buf0, float* buf1, uint32_t* sh_hist) {
+  const int m = tbl.m[combo], n = tbl.n[combo], len = tbl.len[combo];
+  const long long Lp = p.L - p.n_sink;                     // scores without the sink part
+  const float* a = p.scores + p.n_sink;
+  const int lo = c0 - n / 2;
+  const int n_out = min(kSelTile, len - c0);
+  const int span = n_out + n - 1;
+  const float pad = (p.win_op == 0) ? 0.f : -INFINITY;
+  if (m == 1) {
+    constexpr int kLd = (kSelTile + kMaxWin + kSelThreads - 1) / kSelThreads;
+    float v[kLd];
+#pragma unroll
+    for (int k = 0; k < kLd; ++k) {
+      const int idx = k * kSelThreads + threadIdx.x, u = lo + idx;
+      v[k] = (idx < span && u >= 0 && u < len) ? __ldcg(a + u) : pad;
+    }
+#pragma unroll
+    for (int k = 0; k < kLd; ++k) {
+      const int idx = k * kSelThreads + threadIdx.x;
+      if (idx < span) buf0[idx] = v[k];
+    }
+  } else {
+    for (int idx = threadIdx.x; idx < span; idx += kSelThreads) {
+      const int u = lo + idx;
+      float v = pad;
+      if (u >= 0 && u < len) {
+        const long long t0 = static_cast<long long>(u) * m;
+        const long long t1 = min(t0 + m, Lp);
+        v = __ldcg(a + t0);
+        for (long long t = t0 + 1; t < t1; ++t) v = fmaxf(v, __ldcg(a + t));
+      }
+      buf0[idx] = v;
+    }
+  }
+  __syncthreads();
+  // Window maximum by doubling: after the step of width w, src[i] = max of cells [i, i + w);
+  // a window of n cells is then the maximum of two overlapping runs of width w <= n < 2w.
+  float* src = buf0;
+  int w = 1;
+  if (p.win_op != 0) {
+    float* dst = buf1;
+    while (2 * w <= n) {
+      const int cnt = span - 2 * w + 1;
+      for (int i = threadIdx.x; i < cnt; i += kSelThreads) dst[i] = fmaxf(src[i], src[i + w]);
+      __syncthreads();
+      float* t = src; src = dst; dst = t;
+      w *= 2;
+    }
+  }
+  float* out = p.pooled + static_cast<long long>(combo) * p.pooled_stride;
+  for (int base = 0; base < n_out; base += kSelThreads) {
+    const int i = base + threadIdx.x;
+    uint32_t digit = 0xFFFFFFFFu;
+    if (i < n_out) {
+      float acc;
+      if (p.win_op == 0) {
+        acc = 0.f;
+        for (int j = 0; j < n; ++j) acc += src[i + j];       // left to right, as the definition
+        acc = acc / static_cast<float>(n);
+      } else {
+        acc = fmaxf(src[i], src[i + n - w]);
+      }
+      out[c0 + i] = acc;
+      digit = static_cast<uint32_t>(make_key(acc, static_cast<uint32_t>(c0 + i)) >> 53);
+    }
+    hist_add(sh_hist, digit);
+  }
+  __syncthreads();
+}
+
+// The CTA that owns `combo` in this pass locates the bin holding the k-th largest key among
+// those that match the prefix so far, extends the prefix, and clears the histogram.
+__device__ __forceinline__ void bin_search(const SelectParams& p, int combo, int pass,
+                                           SelShared* sh) {
+  int shift, bits;
+  pass_bits(pass, shift, bits);
+  uint32_t* gh = p.hist + static_cast<long long>(combo) * kHistBins;
+  const unsigned long long prefix = __ldcg(&p.sel_prefix[combo]);
+  const uint32_t k_rem = __ldcg(&p.sel_krem[combo]);
+  constexpr int kPer = kHistBins / kSelThreads;
+  uint32_t h[kPer];
+  uint32_t total = 0;
+#pragma unroll
+  for (int j = 0; j < kPer; ++j) {
+    h[j] = __ldcg(&gh[kHistBins - 1 - (kPer * threadIdx.x + j)]);   // bins in descending order
+    total += h[j];
+  }
+  uint32_t grand;
+  const uint32_t excl = block_exclusive_scan(total, sh->scan, &grand);
+  if (excl < k_rem && k_rem <= excl + total) {
+    uint32_t cum = excl;
+#pragma unroll
+    for (int j = 0; j < kPer; ++j) {
+      if (k_rem > cum && k_rem <= cum + h[j]) {
+        const uint32_t bin = kHistBins - 1 - (kPer * threadIdx.x + j);
+        const uint32_t new_k = k_rem - cum;
+        p.sel_prefix[combo] = prefix | (static_cast<unsigned long long>(bin) << shift);
+        p.sel_krem[combo] = new_k;
+        p.sel_done[combo] = (h[j] == new_k || pass == kSelectPasses - 1) ? 1u : 0u;
+      }
+      cum += h[j];
+    }
+  }
+  if (threadIdx.x == 0 && (k_rem > grand || k_rem == 0))
+    p.sel_done[combo] = 1u;                                // fewer keys than asked: take all
+  for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) gh[b] = 0u;
+  __syncthreads();
+}
+
+// Phase E: ranks the candidates [32 * kb_begin, 32 * kb_end) of `combo` among all of its n
+// candidates by counting the keys above each (keys are distinct).  One warp per candidate,
+// its lanes split the comparison range; the candidates are staged in shared memory, at most
+// kRankChunk at a time (one staging serves all items when n fits).
+static constexpr int kRankChunk = 8192;
+
+__device__ __forceinline__ void rank_range(const SelectParams& p, int combo, int n, int kb_begin,
+                                           int kb_end, unsigned long long* chunk) {
+  const unsigned long long* cand = p.cand + static_cast<long long>(combo) * p.cand_stride;
+  int* ranked = p.ranked + static_cast<long long>(combo) * p.cand_stride;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const bool whole = n <= kRankChunk;
+  for (int kb = kb_begin; kb < kb_end; ++kb) {
+    const int mine = kb * kRankKeysPerItem + warp;
+    const unsigned long long key = (mine < n) ? __ldcg(&cand[mine]) : 0ull;
+    int above = 0;
+    for (int base = 0; base < n; base += kRankChunk) {
+      const int cnt = min(kRankChunk, n - base);
+      const int padded = (cnt + 63) & ~63;
+      if (!whole || kb == kb_begin) {
+        __syncthreads();
+        constexpr int kLd = kRankChunk / kSelThreads;       // all loads in flight together
+        unsigned long long v[kLd];
+#pragma unroll
+        for (int k = 0; k < kLd; ++k) {
+          const int i = k * kSelThreads + threadIdx.x;
+          v[k] = (i < cnt) ? __ldcg(&cand[base + i]) : 0ull;
+        }
+#pragma unroll
+        for (int k = 0; k < kLd; ++k) {
+          const int i = k * kSelThreads + threadIdx.x;
+          if (i < padded) chunk[i] = v[k];
+        }
+        __syncthreads();
+      }
+      const ulonglong2* pairs = reinterpret_cast<const ulonglong2*>(chunk);
+      const int rounds = padded >> 6;                       // 32 lanes x 2 keys per round
+#pragma unroll 4
+      for (int j = 0; j < rounds; ++j) {
+        const ulonglong2 two = pairs[32 * j + lane];
+        above += (two.x > key) ? 1 : 0;
+        above += (two.y > key) ? 1 : 0;
+      }
+    }
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) above += __shfl_xor_sync(0xFFFFFFFFu, above, o);
+    if (lane == 0 && mine < n)
+      ranked[above] = static_cast<int>(0xFFFFFFFFu - static_cast<uint32_t>(key & 0xFFFFFFFFull));
+  }
+}
+
+// Tokens of cell `cell` (size m) that are not allocated yet, as a bit mask (bit j = token j).
+__device__ __forceinline__ unsigned long long fresh_tokens(const uint32_t* bm, long long cell,
+                                                           int m, long long Lp, int n_sink) {
+  unsigned long long fresh = 0ull;
+  const long long t0 = cell * m;
+  for (int j = 0; j < m; ++j) {
+    const long long t = t0 + j;
+    if (t < Lp) {
+      const long long pos = n_sink + t;
+      const uint32_t word = *reinterpret_cast<const volatile uint32_t*>(&bm[pos >> 5]);
+      if (!((word >> (pos & 31)) & 1u)) fresh |= (1ull << j);
+    }
+  }
+  return fresh;
+}
+
+// Phase F (one CTA): quota walk over the ranked cells of every combination, then the
+// ascending list of allocated positions.  `bm` is the bitmap (shared or global memory),
+// `staged` room for kMaxKm cell ids in shared memory.  Every thread owns a run of consecutive
+// ranks; the cells of one combination are disjoint, so the new-token counts of all its cells
+// can be taken before any of them is marked.
+__device__ __forceinline__ void allocate(const ComboTable& tbl, const SelectParams& p,
+                                         uint32_t* bm, int* staged, SelShared* sh) {
   const long long Lp = p.L - p.n_sink;
+  for (int combo = threadIdx.x; combo < tbl.n_comb; combo += kSelThreads)
+    sh->state[combo] = __ldcg(&p.cand_count[combo]);
+  __syncthreads();
   for (int combo = 0; combo < tbl.n_comb; ++combo) {
     const int m = tbl.m[combo];
-    const int quota = tbl.quota[combo];
-    const int K = min(static_cast<int>(min(p.cand_count[combo], static_cast<uint32_t>(kMaxKm))),
+    const uint32_t quota = static_cast<uint32_t>(tbl.quota[combo]);
+    const int K = min(static_cast<int>(min(sh->state[combo], static_cast<uint32_t>(kMaxKm))),
                       tbl.k_m[combo]);
     const int* ranked = p.ranked + static_cast<long long>(combo) * p.cand_stride;
-    int taken = 0;                                            // uniform across the block
-    for (int base = 0; base < K && taken < quota; base += kAllocThreads) {
-      const int r = base + threadIdx.x;
-      unsigned long long fresh = 0ull;                        // bit j: token j of the cell is new
-      long long t0 = 0;
-      if (r < K) {
-        t0 = static_cast<long long>(ranked[r]) * m;
-        for (int j = 0; j < m; ++j) {
-          const long long t = t0 + j;
-          if (t < Lp) {
-            const long long pos = p.n_sink + t;
-            const uint32_t word = __ldcg(&p.bitmap[pos >> 5]);
-            if (!((word >> (pos & 31)) & 1u)) fresh |= (1ull << j);
-          }
-        }
+    for (int base = 0; base < K; base += 4 * kSelThreads) {   // coalesced, four loads in flight
+      int v[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int r = base + k * kSelThreads + threadIdx.x;
+        v[k] = (r < K) ? __ldcg(&ranked[r]) : 0;
       }
-      uint32_t total;
-      const uint32_t before = block_exclusive_scan(__popcll(fresh), sh_warp, &total);
-      const int room = quota - taken;
-      uint32_t ord = before;
-      while (fresh && ord < static_cast<uint32_t>(room)) {    // ascending position inside the cell
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int r = base + k * kSelThreads + threadIdx.x;
+        if (r < K) staged[r] = v[k];
+      }
+    }
+    __syncthreads();
+    const int per = (K + kSelThreads - 1) / kSelThreads;
+    const int r0 = min(K, static_cast<int>(threadIdx.x) * per), r1 = min(K, r0 + per);
+    uint32_t mine = 0;
+    for (int r = r0; r < r1; ++r) mine += __popcll(fresh_tokens(bm, staged[r], m, Lp, p.n_sink));
+    uint32_t total;
+    uint32_t ord = block_exclusive_scan(mine, sh->scan, &total);
+    for (int r = r0; r < r1 && ord < quota; ++r) {
+      const long long cell = staged[r];
+      unsigned long long fresh = fresh_tokens(bm, cell, m, Lp, p.n_sink);
+      while (fresh && ord < quota) {                         // ascending position inside the cell
         const int j = __ffsll(static_cast<long long>(fresh)) - 1;
         fresh &= fresh - 1;
-        const long long pos = p.n_sink + t0 + j;
-        atomicOr(&p.bitmap[pos >> 5], 1u << (pos & 31));
+        const long long pos = p.n_sink + cell * m + j;
+        atomicOr(&bm[pos >> 5], 1u << (pos & 31));
         ++ord;
       }
-      taken += min(static_cast<int>(total), room);
-      __syncthreads();                                        // bitmap updates visible to the block
     }
-    if (taken < quota && threadIdx.x == 0) atomicCAS(p.status, 0, kDevQuota);
-    __syncthreads();
+    if (total < quota && threadIdx.x == 0) atomicCAS(p.status, 0, kDevQuota);
+    __syncthreads();                                         // bitmap updates visible to the block
   }
 
-  // Ascending output: every thread owns a contiguous run of bitmap words.
+  // Ascending output.  Every warp owns a contiguous run of bitmap words and reads it 32
+  // consecutive words at a time (one per lane).
   const long long n_words = (p.L + 31) / 32;
-  const long long per_thread = (n_words + kAllocThreads - 1) / kAllocThreads;
-  const long long w0 = min(n_words, static_cast<long long>(threadIdx.x) * per_thread);
-  const long long w1 = min(n_words, w0 + per_thread);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long rounds = (n_words + kSelThreads - 1) / kSelThreads;       // per warp
+  const long long w_begin = static_cast<long long>(warp) * rounds * 32;
   uint32_t count = 0;
-  for (long long w = w0; w < w1; ++w) count += __popc(__ldcg(&p.bitmap[w]));
+  for (long long k = 0; k < rounds; ++k) {
+    const long long w = w_begin + k * 32 + lane;
+    if (w < n_words) count += __popc(*reinterpret_cast<volatile uint32_t*>(&bm[w]));
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) count += __shfl_xor_sync(0xFFFFFFFFu, count, o);
   uint32_t total;
-  uint32_t off = block_exclusive_scan(count, sh_warp, &total);
+  uint32_t off = block_exclusive_scan(lane == 0 ? count : 0u, sh->scan, &total);
+  off = __shfl_sync(0xFFFFFFFFu, off, 0);                   // first output slot of this warp
   const uint32_t cap = static_cast<uint32_t>(p.n_sink + p.budget);
-  for (long long w = w0; w < w1; ++w) {
-    uint32_t bits = __ldcg(&p.bitmap[w]);
+  for (long long k = 0; k < rounds; ++k) {
+    const long long w = w_begin + k * 32 + lane;
+    uint32_t bits = (w < n_words) ? *reinterpret_cast<volatile uint32_t*>(&bm[w]) : 0u;
+    uint32_t incl = __popc(bits);
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    uint32_t at = off + incl - __popc(bits);
     while (bits) {
       const int b = __ffs(bits) - 1;
       bits &= bits - 1;
-      if (off < cap) p.out_idx[off] = static_cast<int>(w * 32 + b);
-      ++off;
+      if (at < cap) p.out_idx[at] = static_cast<int>(w * 32 + b);
+      ++at;
     }
+    off += __shfl_sync(0xFFFFFFFFu, incl, 31);
   }
   if (threadIdx.x == 0 && total != cap) atomicCAS(p.status, 0, kDevQuota);
 }
 
+__global__ void __launch_bounds__(kSelThreads, 1)
+select_kernel(const ComboTable tbl, const SelectParams p) {
+  extern __shared__ __align__(16) uint8_t dyn_smem[];
+  __shared__ SelShared sh;
+  const int n_tiles = tbl.tile_begin[tbl.n_comb];
+  const int t_begin = static_cast<int>(static_cast<long long>(blockIdx.x) * n_tiles / gridDim.x);
+  const int t_end = static_cast<int>(static_cast<long long>(blockIdx.x + 1) * n_tiles / gridDim.x);
+  for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) sh.hist[b] = 0u;
+  uint32_t epoch = 0;
+#ifdef ILRE_SELECT_TRACE
+  __shared__ unsigned long long trace_t[32];
+  __shared__ const char* trace_tag[32];
+  int trace_n = 0;
+  SEL_TRACE("start");
+#endif
+
+  // ---- A: scores from the encoded maxima, one exp per position ----
+  {
+    const long long stride = static_cast<long long>(gridDim.x) * kSelThreads;
+    for (long long t = static_cast<long long>(blockIdx.x) * kSelThreads + threadIdx.x; t < p.L;
+         t += stride) {
+      const float a = exp2f(ordered_to_float(__ldcg(&p.enc[t])));
+      p.scores[t] = a;
+      if (p.user_scores) p.user_scores[t] = a;
+    }
+  }
+  if (!grid_sync(p, &sh, epoch)) return;
+  SEL_TRACE("scores");
+
+  // ---- B: pooling of every combination + first histogram ----
+  {
+    float* buf0 = reinterpret_cast<float*>(dyn_smem);
+    float* buf1 = buf0 + (kSelTile + kMaxWin);
+    int cur = -1;
+    for (int tile = t_begin; tile < t_end; ++tile) {
+      const int combo = combo_of_tile(tbl, tile);
+      if (combo != cur && cur >= 0)
+        hist_flush(sh.hist, p.hist + static_cast<long long>(cur) * kHistBins);
+      cur = combo;
+      pool_tile(tbl, p, combo, (tile - tbl.tile_begin[combo]) * kSelTile, buf0, buf1, sh.hist);
+    }
+    if (cur >= 0) hist_flush(sh.hist, p.hist + static_cast<long long>(cur) * kHistBins);
+  }
+  if (!grid_sync(p, &sh, epoch)) return;
+  SEL_TRACE("pool+hist0");
+
+  // ---- C: radix select ----
+  for (int pass = 0; pass < kSelectPasses; ++pass) {
+    if (pass > 0) {
+      int shift, bits;
+      pass_bits(pass, shift, bits);
+      const uint32_t mask = (1u << bits) - 1u;
+      for (int combo = threadIdx.x; combo < tbl.n_comb; combo += kSelThreads) {
+        sh.state[combo] = __ldcg(&p.sel_done[combo]);
+        sh.prefix[combo] = __ldcg(&p.sel_prefix[combo]);
+      }
+      __syncthreads();
+      int cur = -1;
+      for (int t0 = t_begin; t0 < t_end; t0 += kScanGroup) {
+        float wv[kScanGroup][kTilePer];
+#pragma unroll
+        for (int g = 0; g < kScanGroup; ++g)
+          if (t0 + g < t_end) fetch_tile(tbl, p, t0 + g, sh.state, wv[g]);
+#pragma unroll
+        for (int g = 0; g < kScanGroup; ++g) {
+          const int tile = t0 + g;
+          if (tile >= t_end) break;
+          const int combo = combo_of_tile(tbl, tile);
+          if (sh.state[combo]) continue;
+          if (combo != cur && cur >= 0)
+            hist_flush(sh.hist, p.hist + static_cast<long long>(cur) * kHistBins);
+          cur = combo;
+          const unsigned long long prefix = sh.prefix[combo];
+          const int c0 = (tile - tbl.tile_begin[combo]) * kSelTile;
+          const int c1 = min(tbl.len[combo], c0 + kSelTile);
+#pragma unroll
+          for (int k = 0; k < kTilePer; ++k) {
+            const int c = c0 + k * kSelThreads + threadIdx.x;
+            uint32_t digit = 0xFFFFFFFFu;                    // sentinel: does not take part
+            if (c < c1) {
+              const unsigned long long key = make_key(wv[g][k], static_cast<uint32_t>(c));
+              if (((key ^ prefix) >> (shift + bits)) == 0ull)
+                digit = static_cast<uint32_t>(key >> shift) & mask;
+            }
+            hist_add(sh.hist, digit);
+          }
+        }
+      }
+      if (cur >= 0) hist_flush(sh.hist, p.hist + static_cast<long long>(cur) * kHistBins);
+      if (!grid_sync(p, &sh, epoch)) return;
+      SEL_TRACE("histogram");
+    }
+    for (int combo = blockIdx.x; combo < tbl.n_comb; combo += gridDim.x)
+      if (__ldcg(&p.sel_done[combo]) == 0u) bin_search(p, combo, pass, &sh);
+    if (!grid_sync(p, &sh, epoch)) return;
+    SEL_TRACE("bin search");
+    int pending = 0;
+    for (int combo = threadIdx.x; combo < tbl.n_comb; combo += kSelThreads)
+      pending |= (__ldcg(&p.sel_done[combo]) == 0u);
+    if (!__syncthreads_or(pending)) break;                   // same data in every CTA
+  }
+
+  // ---- D: gather the keys at or above each combination's threshold ----
+  {
+    for (int combo = threadIdx.x; combo < tbl.n_comb; combo += kSelThreads)
+      sh.prefix[combo] = __ldcg(&p.sel_prefix[combo]);
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    for (int t0 = t_begin; t0 < t_end; t0 += kScanGroup) {
+      float wv[kScanGroup][kTilePer];
+#pragma unroll
+      for (int g = 0; g < kScanGroup; ++g)
+        if (t0 + g < t_end) fetch_tile(tbl, p, t0 + g, nullptr, wv[g]);
+#pragma unroll
+      for (int g = 0; g < kScanGroup; ++g) {
+        const int tile = t0 + g;
+        if (tile >= t_end) break;
+        const int combo = combo_of_tile(tbl, tile);
+        const unsigned long long threshold = sh.prefix[combo];
+        unsigned long long* cand = p.cand + static_cast<long long>(combo) * p.cand_stride;
+        const int c0 = (tile - tbl.tile_begin[combo]) * kSelTile;
+        const int c1 = min(tbl.len[combo], c0 + kSelTile);
+#pragma unroll
+        for (int k = 0; k < kTilePer; ++k) {
+          const int c = c0 + k * kSelThreads + threadIdx.x;
+          unsigned long long key = 0ull;
+          bool take = false;
+          if (c < c1) {
+            key = make_key(wv[g][k], static_cast<uint32_t>(c));
+            take = key >= threshold;
+          }
+          const uint32_t votes = __ballot_sync(0xFFFFFFFFu, take);
+          if (votes) {
+            uint32_t slot = 0;
+            if (lane == __ffs(votes) - 1) slot = atomicAdd(&p.cand_count[combo], __popc(votes));
+            slot = __shfl_sync(0xFFFFFFFFu, slot, __ffs(votes) - 1) +
+                   __popc(votes & ((1u << lane) - 1u));
+            if (take && slot < static_cast<uint32_t>(tbl.k_m[combo])) cand[slot] = key;
+          }
+        }
+      }
+    }
+  }
+  if (!grid_sync(p, &sh, epoch)) return;
+  SEL_TRACE("gather");
+
+  // ---- E: ranking ----
+  {
+    unsigned long long* chunk = reinterpret_cast<unsigned long long*>(dyn_smem);
+    for (int combo = threadIdx.x; combo < tbl.n_comb; combo += kSelThreads)
+      sh.state[combo] = min(min(__ldcg(&p.cand_count[combo]), static_cast<uint32_t>(kMaxKm)),
+                            static_cast<uint32_t>(tbl.k_m[combo]));
+    __syncthreads();
+    int n_items = 0;
+    for (int combo = 0; combo < tbl.n_comb; ++combo)
+      n_items += (static_cast<int>(sh.state[combo]) + kRankKeysPerItem - 1) / kRankKeysPerItem;
+    // every CTA takes a contiguous run of items, so that it stages few combinations
+    const int i_begin = static_cast<int>(static_cast<long long>(blockIdx.x) * n_items / gridDim.x);
+    const int i_end = static_cast<int>(static_cast<long long>(blockIdx.x + 1) * n_items / gridDim.x);
+    int item0 = 0;
+    for (int combo = 0; combo < tbl.n_comb; ++combo) {
+      const int n = static_cast<int>(sh.state[combo]);
+      const int items = (n + kRankKeysPerItem - 1) / kRankKeysPerItem;
+      const int lo = max(i_begin, item0) - item0, hi = min(i_end, item0 + items) - item0;
+      if (lo < hi) rank_range(p, combo, n, lo, hi, chunk);
+      item0 += items;
+    }
+  }
+  if (!grid_sync(p, &sh, epoch)) return;
+  SEL_TRACE("rank");
+
+  // ---- F: allocation and ascending output (one CTA) ----
+  if (blockIdx.x != 0) return;
+  uint32_t* bm = p.bitmap;
+  int* staged = reinterpret_cast<int*>(dyn_smem);
+  if (p.bitmap_in_smem) {
+    bm = reinterpret_cast<uint32_t*>(dyn_smem);
+    const long long n_words = (p.L + 31) / 32;
+    staged = reinterpret_cast<int*>(dyn_smem + ((n_words * 4 + 15) & ~15ll));
+    for (long long w = threadIdx.x; w < n_words; w += kSelThreads) {
+      const long long lo = w * 32;
+      uint32_t bits = 0;
+      if (p.n_sink > lo) bits = (p.n_sink - lo >= 32) ? 0xFFFFFFFFu : ((1u << (p.n_sink - lo)) - 1u);
+      bm[w] = bits;
+    }
+    __syncthreads();
+  }
+  allocate(tbl, p, bm, staged, &sh);
+  SEL_TRACE("allocate");
+#ifdef ILRE_SELECT_TRACE
+  if (threadIdx.x == 0)
+    for (int i = 1; i < trace_n; ++i)
+      printf("select phase %-12s %8.2f us\n", trace_tag[i], (trace_t[i] - trace_t[i - 1]) * 1e-3);
+#endif
+}
+
 // ---------------------------------------------------------------------------------------
-// launchers
+// host side
 // ---------------------------------------------------------------------------------------
-static int select_blocks(int max_len) {
-  int nb = (max_len + kSelThreads * kSelItemsPerThread - 1) / (kSelThreads * kSelItemsPerThread);
-  if (nb < 1) nb = 1;
-  if (nb > 256) nb = 256;
-  return nb;
+size_t select_smem_bytes(long long L, int* bitmap_in_smem) {
+  size_t bytes = 2 * static_cast<size_t>(kSelTile + kMaxWin) * sizeof(float);  // pooling tiles
+  const size_t rank_bytes = kRankChunk * sizeof(unsigned long long);           // ranking chunk
+  if (rank_bytes > bytes) bytes = rank_bytes;
+  const size_t staged_bytes = kMaxKm * sizeof(int);                            // ranked cells
+  const size_t bm_bytes = (static_cast<size_t>((L + 31) / 32) * sizeof(uint32_t) + 15) & ~size_t(15);
+  *bitmap_in_smem = bm_bytes <= static_cast<size_t>(kSelBitmapSmemBytes) ? 1 : 0;
+  const size_t alloc_bytes = staged_bytes + (*bitmap_in_smem ? bm_bytes : 0);
+  if (alloc_bytes > bytes) bytes = alloc_bytes;
+  return bytes;
 }
 
-cudaError_t launch_pool(const ComboTable& tbl, const SelectParams& p, int max_len,
-                        cudaStream_t st) {
-  dim3 grid((max_len + kPoolTile - 1) / kPoolTile, tbl.n_comb);
-  pool_kernel<<<grid, kPoolThreads, 0, st>>>(tbl, p);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_select_pass(const ComboTable& tbl, const SelectParams& p, int max_len, int pass,
-                               cudaStream_t st) {
-  dim3 grid(select_blocks(max_len), tbl.n_comb);
-  select_pass_kernel<<<grid, kSelThreads, 0, st>>>(tbl, p, pass);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_gather(const ComboTable& tbl, const SelectParams& p, int max_len,
-                          cudaStream_t st) {
-  dim3 grid(select_blocks(max_len), tbl.n_comb);
-  gather_kernel<<<grid, kSelThreads, 0, st>>>(tbl, p);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_rank_sort(const ComboTable& tbl, const SelectParams& p, int max_km,
-                             cudaStream_t st) {
-  int pow2 = 2;
-  while (pow2 < max_km) pow2 <<= 1;
-  const size_t smem = static_cast<size_t>(pow2) * sizeof(unsigned long long);
-  cudaError_t e = cudaFuncSetAttribute(rank_sort_kernel,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+cudaError_t select_max_grid(int n_sm, int* max_grid) {
+  cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kSelMaxDynSmemBytes);
   if (e != cudaSuccess) return e;
-  rank_sort_kernel<<<tbl.n_comb, kSortThreads, smem, st>>>(tbl, p, pow2);
-  return cudaGetLastError();
+  int per_sm = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, select_kernel, kSelThreads,
+                                                    kSelMaxDynSmemBytes);
+  if (e != cudaSuccess) return e;
+  if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+  *max_grid = n_sm;                      // one CTA per SM is plenty for these phases
+  return cudaSuccess;
 }
 
-cudaError_t launch_allocate(const ComboTable& tbl, const SelectParams& p, cudaStream_t st) {
-  allocate_kernel<<<1, kAllocThreads, 0, st>>>(tbl, p);
-  return cudaGetLastError();
+cudaError_t launch_select(const ComboTable& tbl, const SelectParams& p, int grid, size_t smem,
+                          cudaStream_t st) {
+  void* args[2] = {const_cast<ComboTable*>(&tbl), const_cast<SelectParams*>(&p)};
+  return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(select_kernel), dim3(grid),
+                                     dim3(kSelThreads), args, smem, st);
 }
 
 }  // namespace ilre

@@ -1,5 +1,5 @@
-// Parameters and launchers of the Algorithm 1 kernels: pooling, ranked top-K_m per
-// combination, quota allocation with de-duplication, ascending output.
+// Parameters and launcher of the Algorithm 1 kernel: pooling, ranked top-K_m per combination,
+// quota allocation with de-duplication, ascending output.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -10,8 +10,13 @@ static constexpr int kMaxCombos = 64;
 static constexpr int kHistBins = 2048;
 static constexpr int kMaxWin = 1024;        // largest stride-1 window size
 static constexpr int kMaxMaxSize = 64;      // largest strided max-pool size
-static constexpr int kMaxKm = 16384;        // largest K_m the in-block ranking sort holds
+static constexpr int kMaxKm = 16384;        // largest K_m (bounds the candidate lists)
 static constexpr int kSelectPasses = 6;     // 64-bit (value, index) key, 11/11/10 bits twice
+static constexpr int kSelThreads = 1024;    // threads per CTA of the selection kernel
+static constexpr int kSelTile = 4096;       // cells of one combination per work tile
+static constexpr int kRankKeysPerItem = kSelThreads / 32;   // candidates ranked per work item
+static constexpr int kSelBitmapSmemBytes = 136 * 1024;   // bitmap kept in shared memory up to this
+static constexpr int kSelMaxDynSmemBytes = kSelBitmapSmemBytes + kMaxKm * 4;
 
 // One entry per (m_i, n_j) combination, in Algorithm 1's loop order.
 struct ComboTable {
@@ -21,37 +26,40 @@ struct ComboTable {
   int len[kMaxCombos];     // number of cells = ceil((L - n_sink) / m)
   int k_m[kMaxCombos];     // candidates ranked for this combination
   int quota[kMaxCombos];   // B_c
+  int tile_begin[kMaxCombos + 1];   // first work tile of each combination (prefix sums)
 };
 
 struct SelectParams {
-  const float* scores;     // A^C [L]
+  const uint32_t* enc;     // [L] order-preserving uint of max_r log2 p_rt (scores pass output)
+  float* scores;           // A^C [L]
+  float* user_scores;      // optional copy of A^C for the caller, or null
   long long L;
   int n_sink;
   int win_op;              // 0 average, 1 max
   float* pooled;           // [n_comb][pooled_stride]
   long long pooled_stride;
-  uint32_t* hist;          // [n_comb][kHistBins]
+  uint32_t* hist;          // [n_comb][kHistBins], zero on entry and on exit
   unsigned long long* sel_prefix;
   uint32_t* sel_krem;
   uint32_t* sel_done;
-  uint32_t* sel_ticket;
   unsigned long long* cand;   // [n_comb][cand_stride] selected 64-bit keys
   int cand_stride;
   uint32_t* cand_count;
   int* ranked;             // [n_comb][cand_stride] cell ids in rank order
-  uint32_t* bitmap;        // [ceil(L/32)]
+  uint32_t* bitmap;        // [ceil(L/32)] in global memory, used when it does not fit shared memory
+  int bitmap_in_smem;
   int* out_idx;            // [n_sink + budget]
   int budget;
+  uint32_t* barrier;       // grid barrier arrival counter, zero when the kernel starts
   int* status;
 };
 
-cudaError_t launch_pool(const ComboTable& tbl, const SelectParams& p, int max_len, cudaStream_t st);
-cudaError_t launch_select_pass(const ComboTable& tbl, const SelectParams& p, int max_len, int pass,
-                               cudaStream_t st);
-cudaError_t launch_gather(const ComboTable& tbl, const SelectParams& p, int max_len,
+// Dynamic shared memory the kernel needs for a context of L positions.
+size_t select_smem_bytes(long long L, int* bitmap_in_smem);
+// Largest grid that is co-resident on the device (the kernel's CTAs wait on one another).
+cudaError_t select_max_grid(int n_sm, int* max_grid);
+// One cooperative launch: A^C from the encoded maxima, then all of Algorithm 1.
+cudaError_t launch_select(const ComboTable& tbl, const SelectParams& p, int grid, size_t smem,
                           cudaStream_t st);
-cudaError_t launch_rank_sort(const ComboTable& tbl, const SelectParams& p, int max_km,
-                             cudaStream_t st);
-cudaError_t launch_allocate(const ComboTable& tbl, const SelectParams& p, cudaStream_t st);
 
 }  // namespace ilre

@@ -11,7 +11,7 @@ namespace ilre {
 enum : int {
   kDevOk = 0,
   kDevWaitQFull = 1, kDevWaitKFull = 2, kDevWaitKEmpty = 3, kDevWaitAccFull = 4,
-  kDevWaitAccEmpty = 5, kDevSmemAlign = 6, kDevQuota = 16
+  kDevWaitAccEmpty = 5, kDevSmemAlign = 6, kDevGridBarrier = 7, kDevQuota = 16
 };
 
 // Spin budget of one wait, in SM clock cycles (about one second).
