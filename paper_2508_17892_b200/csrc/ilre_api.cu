@@ -330,7 +330,7 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
   long long rank_items = 0;
   for (int c = 0; c < tbl.n_comb; ++c)
     rank_items += (tbl.k_m[c] + kRankKeysPerItem - 1) / kRankKeysPerItem;
-  if (rank_items / 4 > want_grid) want_grid = rank_items / 4;
+  if (rank_items / 2 > want_grid) want_grid = rank_items / 2;
   if (want_grid < 1) want_grid = 1;
   if (want_grid > h->select_max_grid) want_grid = h->select_max_grid;
   const int select_grid = static_cast<int>(want_grid);

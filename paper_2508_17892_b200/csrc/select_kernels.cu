@@ -342,25 +342,37 @@ __device__ __forceinline__ void allocate(const ComboTable& tbl, const SelectPara
   for (int combo = threadIdx.x; combo < tbl.n_comb; combo += kSelThreads)
     sh->state[combo] = __ldcg(&p.cand_count[combo]);
   __syncthreads();
+  // The ranked cells of the next combination are fetched into registers while the current
+  // one is walked (kPre per thread cover K_m up to kPre * kSelThreads; the rest is loaded late).
+  constexpr int kPre = 5;
+  int pre[kPre];
+  auto candidates = [&](int combo) {
+    return min(static_cast<int>(min(sh->state[combo], static_cast<uint32_t>(kMaxKm))),
+               tbl.k_m[combo]);
+  };
+  auto prefetch = [&](int combo) {
+    const int K = candidates(combo);
+    const int* ranked = p.ranked + static_cast<long long>(combo) * p.cand_stride;
+#pragma unroll
+    for (int k = 0; k < kPre; ++k) {
+      const int r = k * kSelThreads + threadIdx.x;
+      pre[k] = (r < K) ? __ldcg(&ranked[r]) : 0;
+    }
+  };
+  if (tbl.n_comb > 0) prefetch(0);
   for (int combo = 0; combo < tbl.n_comb; ++combo) {
     const int m = tbl.m[combo];
     const uint32_t quota = static_cast<uint32_t>(tbl.quota[combo]);
-    const int K = min(static_cast<int>(min(sh->state[combo], static_cast<uint32_t>(kMaxKm))),
-                      tbl.k_m[combo]);
+    const int K = candidates(combo);
     const int* ranked = p.ranked + static_cast<long long>(combo) * p.cand_stride;
-    for (int base = 0; base < K; base += 4 * kSelThreads) {   // coalesced, four loads in flight
-      int v[4];
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const int r = base + k * kSelThreads + threadIdx.x;
-        v[k] = (r < K) ? __ldcg(&ranked[r]) : 0;
-      }
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const int r = base + k * kSelThreads + threadIdx.x;
-        if (r < K) staged[r] = v[k];
-      }
+    for (int k = 0; k < kPre; ++k) {
+      const int r = k * kSelThreads + threadIdx.x;
+      if (r < K) staged[r] = pre[k];
     }
+    for (int r = kPre * kSelThreads + threadIdx.x; r < K; r += kSelThreads)
+      staged[r] = __ldcg(&ranked[r]);
+    if (combo + 1 < tbl.n_comb) prefetch(combo + 1);
     __syncthreads();
     const int per = (K + kSelThreads - 1) / kSelThreads;
     const int r0 = min(K, static_cast<int>(threadIdx.x) * per), r1 = min(K, r0 + per);
