@@ -31,9 +31,9 @@ import numpy as np
 import torch
 
 # DRAM bytes per context position of the dominant kernel (row statistics), from one ncu
-# capture at L = 131072, q_len = 256: (270.6 MB read + 4.4 MB written) / 131072 keys.  Traffic
+# capture at L = 131072, q_len = 256: (270.57 MB read + 5.25 MB written, mean of two launches) / 131072 keys.  Traffic
 # grows in proportion to L (the query block is L2-resident), so it is scaled by L.
-ROW_STATS_DRAM_BYTES_PER_KEY = 2098.2
+ROW_STATS_DRAM_BYTES_PER_KEY = 2104.0
 METRIC = "key_cache_GBps_per_recall_L1M"
 UNIT = "GB/s"
 CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -287,6 +287,16 @@ def run_ours(args, world, rank, local):
                     kernel_ms=stages[dom], algorithmic_flops_per_launch=flops,
                     algorithmic_bytes_per_launch=k_bytes,
                     kernel_hbm_gbs=k_bytes / (stages[dom] * 1e-3) / 1e9)
+    # the row-statistics kernel also evaluates R * L exponentials; the special-function unit
+    # alone would do 16 per clock per SM
+    n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
+    sm_max_ghz = ((clocks or {}).get("sm_max_mhz") or 1965.0) / 1e3
+    exp_peak = 16.0 * n_sm * sm_max_ghz * 1e9
+    exp_rate = float(R) * w.L / (stages["row_stats"] * 1e-3)
+    roofline["row_stats_exponentials"] = dict(
+        bound="alu", achieved=exp_rate / 1e12, peak=exp_peak / 1e12, unit="Texp/s",
+        frac=exp_rate / exp_peak,
+        peak_source=f"16 ex2 per clock per SM x {n_sm} SMs x {sm_max_ghz:.3f} GHz")
     step_hbm_frac = (k_bytes / (ms_per_step * 1e-3) / 1e9) / peaks["hbm_gbs"]
     step_tensor_frac = (flops / (ms_per_step * 1e-3) / 1e12) / peaks["bf16_tflops_sustained"]
 
