@@ -140,7 +140,8 @@ def barrier():
 def workload_string(w) -> str:
     return (f"{w.name}: L={w.L}, q_len={w.q_len}, kv_heads={w.n_kv_heads}, "
             f"q_heads={w.n_q_heads}, d={w.d}, budget={w.budget}, "
-            f"windows={list(w.win_sizes)} (max), max_sizes={list(w.max_sizes)}")
+            f"windows={list(w.win_sizes)} ({'max' if w.win_op else 'avg'}), "
+            f"max_sizes={list(w.max_sizes)}, n_sink={w.n_sink}")
 
 
 def pick_workload(args):

@@ -44,6 +44,7 @@ struct ilre_recall {
   uint32_t* enc;
   float* scores;
   float* pooled;
+  float* maxpooled;
   uint32_t* hist;
   unsigned long long* sel_prefix;
   uint32_t* sel_krem;
@@ -114,7 +115,7 @@ bool dev_alloc(T** p, size_t count) {
 
 void free_all(ilre_recall* h) {
   cudaFree(h->qp); cudaFree(h->partial); cudaFree(h->nlse2); cudaFree(h->row_lse);
-  cudaFree(h->enc); cudaFree(h->scores); cudaFree(h->pooled); cudaFree(h->hist);
+  cudaFree(h->enc); cudaFree(h->scores); cudaFree(h->pooled); cudaFree(h->maxpooled); cudaFree(h->hist);
   cudaFree(h->sel_prefix); cudaFree(h->sel_krem); cudaFree(h->sel_done); cudaFree(h->grid_barrier);
   cudaFree(h->cand); cudaFree(h->cand_count); cudaFree(h->ranked); cudaFree(h->bitmap);
   cudaFree(h->status); cudaFree(h->stage_k); cudaFree(h->stage_q); cudaFree(h->stage_idx);
@@ -222,6 +223,7 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out) {
   ok = ok && dev_alloc(&h->enc, maxL);
   ok = ok && dev_alloc(&h->scores, maxL);
   ok = ok && dev_alloc(&h->pooled, ncomb * maxL);
+  ok = ok && dev_alloc(&h->maxpooled, ncomb * (maxL / 2 + 1));   // one array per distinct m > 1
   ok = ok && dev_alloc(&h->hist, ncomb * kHistBins);
   ok = ok && dev_alloc(&h->sel_prefix, ncomb);
   ok = ok && dev_alloc(&h->sel_krem, ncomb);
@@ -283,6 +285,21 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
       tbl.k_m[c] = static_cast<int>(km);
       tbl.quota[c] = budget / tbl.n_comb + (c < budget % tbl.n_comb ? 1 : 0);
       tbl.tile_begin[c + 1] = tbl.tile_begin[c] + static_cast<int>((len + kSelTile - 1) / kSelTile);
+      // the strided max-pool of size m is shared by all window sizes
+      tbl.src[c] = -1;
+      if (m > 1) {
+        int s = 0;
+        while (s < tbl.n_src && tbl.src_m[s] != m) ++s;
+        if (s == tbl.n_src) {
+          const int cells_per_tile = kSrcTileTokens / m;
+          tbl.src_m[s] = m;
+          tbl.src_len[s] = static_cast<int>(len);
+          tbl.src_tile_begin[s + 1] =
+              tbl.src_tile_begin[s] + static_cast<int>((len + cells_per_tile - 1) / cells_per_tile);
+          ++tbl.n_src;
+        }
+        tbl.src[c] = s;
+      }
     }
 
   CUtensorMap map_k, map_q;
@@ -318,6 +335,7 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
   sp.enc = h->enc; sp.scores = h->scores; sp.user_scores = out_scores_dev;
   sp.L = L; sp.n_sink = spec->n_sink; sp.win_op = spec->win_op;
   sp.pooled = h->pooled; sp.pooled_stride = h->cfg.max_L; sp.hist = h->hist;
+  sp.maxpooled = h->maxpooled; sp.maxpooled_stride = h->cfg.max_L / 2 + 1;
   sp.sel_prefix = h->sel_prefix; sp.sel_krem = h->sel_krem; sp.sel_done = h->sel_done;
   sp.cand = h->cand; sp.cand_stride = h->cand_stride;
   sp.cand_count = h->cand_count; sp.ranked = h->ranked; sp.bitmap = h->bitmap;

@@ -2,8 +2,8 @@
 // meet at grid barriers between the phases:
 //
 //   A  A^C[t] = exp2(max_r log2 p_rt) from the scores pass' encoded maxima (Eq. 5);
-//   B  MaxPooling(size = stride = m) fused with the stride-1 window pooling (average or max)
-//      of every (m, n) combination, and the first radix histogram;
+//   B  MaxPooling(size = stride = m), once per distinct m, then the stride-1 window pooling
+//      (average or max) of every (m, n) combination, and the first radix histogram;
 //   C  radix select of the K_m largest 64-bit keys (pooled value, then lower cell index
 //      first), 11/11/10 bits per pass, all combinations at once; passes stop as soon as every
 //      combination's threshold is settled;
@@ -127,10 +127,11 @@ __device__ __forceinline__ void hist_flush(uint32_t* sh_hist, uint32_t* gh) {
   __syncthreads();
 }
 
-__device__ __forceinline__ int combo_of_tile(const ComboTable& tbl, int tile) {
-  int c = 0;
-  while (c + 1 < tbl.n_comb && tile >= tbl.tile_begin[c + 1]) ++c;
-  return c;
+// Combination that owns `tile`.  Tiles are visited in increasing order, so the search resumes
+// from the previous answer (`cur`, 0 at first).
+__device__ __forceinline__ int combo_of_tile(const ComboTable& tbl, int tile, int& cur) {
+  while (cur + 1 < tbl.n_comb && tile >= tbl.tile_begin[cur + 1]) ++cur;
+  return cur;
 }
 
 static constexpr int kTilePer = kSelTile / kSelThreads;
@@ -138,8 +139,8 @@ static constexpr int kScanGroup = 4;      // tiles whose loads are issued togeth
 
 // Pooled values of one tile, kTilePer per thread, all loads in flight together.
 __device__ __forceinline__ void fetch_tile(const ComboTable& tbl, const SelectParams& p, int tile,
-                                           const uint32_t* skip, float (&wv)[kTilePer]) {
-  const int combo = combo_of_tile(tbl, tile);
+                                           int& cur, const uint32_t* skip, float (&wv)[kTilePer]) {
+  const int combo = combo_of_tile(tbl, tile, cur);
   if (skip && skip[combo]) return;
   const float* w = p.pooled + static_cast<long long>(combo) * p.pooled_stride;
   const int c0 = (tile - tbl.tile_begin[combo]) * kSelTile;
@@ -151,19 +152,53 @@ __device__ __forceinline__ void fetch_tile(const ComboTable& tbl, const SelectPa
   }
 }
 
-// Phase B for one tile: pooled cells [c0, c0 + n_out) of `combo`, written to p.pooled; the
-// first-pass radix digit of every cell goes to the shared histogram.  `buf0`/`buf1` hold
-// kSelTile + kMaxWin floats each.
+// Phase B1 for one tile of source `src`: cells of MaxPooling(size = stride = m), a shorter
+// last cell where m does not divide the length.  The tokens are read coalesced into `buf`
+// (kSrcTileTokens floats), all loads in flight together.
+__device__ __forceinline__ void maxpool_tile(const ComboTable& tbl, const SelectParams& p, int src,
+                                             int tile_in_src, float* buf) {
+  const int m = tbl.src_m[src], len = tbl.src_len[src];
+  const long long Lp = p.L - p.n_sink;
+  const float* a = p.scores + p.n_sink;
+  const int cells_per_tile = kSrcTileTokens / m;
+  const int c0 = tile_in_src * cells_per_tile;
+  const int n_cells = min(cells_per_tile, len - c0);
+  const long long t0 = static_cast<long long>(c0) * m;
+  const int n_tok = static_cast<int>(min(static_cast<long long>(n_cells) * m, Lp - t0));
+  constexpr int kLd = kSrcTileTokens / kSelThreads;
+  float v[kLd];
+#pragma unroll
+  for (int k = 0; k < kLd; ++k) {
+    const int i = k * kSelThreads + threadIdx.x;
+    v[k] = (i < n_tok) ? __ldcg(a + t0 + i) : -INFINITY;
+  }
+#pragma unroll
+  for (int k = 0; k < kLd; ++k) buf[k * kSelThreads + threadIdx.x] = v[k];
+  __syncthreads();
+  float* out = p.maxpooled + static_cast<long long>(src) * p.maxpooled_stride;
+  for (int c = threadIdx.x; c < n_cells; c += kSelThreads) {
+    float acc = buf[c * m];
+    for (int j = 1; j < m; ++j) acc = fmaxf(acc, buf[c * m + j]);
+    out[c0 + c] = acc;
+  }
+  __syncthreads();
+}
+
+// Phase B2 for one tile: pooled cells [c0, c0 + n_out) of `combo` from its max-pooled source
+// (the scores themselves for m = 1), written to p.pooled; the first-pass radix digit of every
+// cell goes to the shared histogram.  `buf0`/`buf1` hold kSelTile + kMaxWin floats each.
 __device__ __forceinline__ void pool_tile(const ComboTable& tbl, const SelectParams& p, int combo,
                                           int c0, float* buf0, float* buf1, uint32_t* sh_hist) {
-  const int m = tbl.m[combo], n = tbl.n[combo], len = tbl.len[combo];
-  const long long Lp = p.L - p.n_sink;                     // scores without the sink part
-  const float* a = p.scores + p.n_sink;
+  const int n = tbl.n[combo], len = tbl.len[combo];
+  const int source = tbl.src[combo];
+  const float* a = (source < 0)
+      ? p.scores + p.n_sink
+      : p.maxpooled + static_cast<long long>(source) * p.maxpooled_stride;
   const int lo = c0 - n / 2;
   const int n_out = min(kSelTile, len - c0);
   const int span = n_out + n - 1;
   const float pad = (p.win_op == 0) ? 0.f : -INFINITY;
-  if (m == 1) {
+  {
     constexpr int kLd = (kSelTile + kMaxWin + kSelThreads - 1) / kSelThreads;
     float v[kLd];
 #pragma unroll
@@ -175,18 +210,6 @@ __device__ __forceinline__ void pool_tile(const ComboTable& tbl, const SelectPar
     for (int k = 0; k < kLd; ++k) {
       const int idx = k * kSelThreads + threadIdx.x;
       if (idx < span) buf0[idx] = v[k];
-    }
-  } else {
-    for (int idx = threadIdx.x; idx < span; idx += kSelThreads) {
-      const int u = lo + idx;
-      float v = pad;
-      if (u >= 0 && u < len) {
-        const long long t0 = static_cast<long long>(u) * m;
-        const long long t1 = min(t0 + m, Lp);
-        v = __ldcg(a + t0);
-        for (long long t = t0 + 1; t < t1; ++t) v = fmaxf(v, __ldcg(a + t));
-      }
-      buf0[idx] = v;
     }
   }
   __syncthreads();
@@ -462,13 +485,28 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
   if (!grid_sync(p, &sh, epoch)) return;
   SEL_TRACE("scores");
 
-  // ---- B: pooling of every combination + first histogram ----
+  // ---- B1: strided max-pool arrays, one per distinct m > 1 ----
+  if (tbl.n_src > 0) {
+    float* buf = reinterpret_cast<float*>(dyn_smem);
+    const int n_st = tbl.src_tile_begin[tbl.n_src];
+    const int s_begin = static_cast<int>(static_cast<long long>(blockIdx.x) * n_st / gridDim.x);
+    const int s_end = static_cast<int>(static_cast<long long>(blockIdx.x + 1) * n_st / gridDim.x);
+    int src = 0;
+    for (int tile = s_begin; tile < s_end; ++tile) {
+      while (src + 1 < tbl.n_src && tile >= tbl.src_tile_begin[src + 1]) ++src;
+      maxpool_tile(tbl, p, src, tile - tbl.src_tile_begin[src], buf);
+    }
+    if (!grid_sync(p, &sh, epoch)) return;
+    SEL_TRACE("maxpool");
+  }
+
+  // ---- B2: window pooling of every combination + first histogram ----
   {
     float* buf0 = reinterpret_cast<float*>(dyn_smem);
     float* buf1 = buf0 + (kSelTile + kMaxWin);
-    int cur = -1;
+    int cur = -1, cursor = 0;
     for (int tile = t_begin; tile < t_end; ++tile) {
-      const int combo = combo_of_tile(tbl, tile);
+      const int combo = combo_of_tile(tbl, tile, cursor);
       if (combo != cur && cur >= 0)
         hist_flush(sh.hist, p.hist + static_cast<long long>(cur) * kHistBins);
       cur = combo;
@@ -490,17 +528,17 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
         sh.prefix[combo] = __ldcg(&p.sel_prefix[combo]);
       }
       __syncthreads();
-      int cur = -1;
+      int cur = -1, load_cursor = 0, cursor = 0;
       for (int t0 = t_begin; t0 < t_end; t0 += kScanGroup) {
         float wv[kScanGroup][kTilePer];
 #pragma unroll
         for (int g = 0; g < kScanGroup; ++g)
-          if (t0 + g < t_end) fetch_tile(tbl, p, t0 + g, sh.state, wv[g]);
+          if (t0 + g < t_end) fetch_tile(tbl, p, t0 + g, load_cursor, sh.state, wv[g]);
 #pragma unroll
         for (int g = 0; g < kScanGroup; ++g) {
           const int tile = t0 + g;
           if (tile >= t_end) break;
-          const int combo = combo_of_tile(tbl, tile);
+          const int combo = combo_of_tile(tbl, tile, cursor);
           if (sh.state[combo]) continue;
           if (combo != cur && cur >= 0)
             hist_flush(sh.hist, p.hist + static_cast<long long>(cur) * kHistBins);
@@ -541,16 +579,17 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
       sh.prefix[combo] = __ldcg(&p.sel_prefix[combo]);
     __syncthreads();
     const int lane = threadIdx.x & 31;
+    int load_cursor = 0, cursor = 0;
     for (int t0 = t_begin; t0 < t_end; t0 += kScanGroup) {
       float wv[kScanGroup][kTilePer];
 #pragma unroll
       for (int g = 0; g < kScanGroup; ++g)
-        if (t0 + g < t_end) fetch_tile(tbl, p, t0 + g, nullptr, wv[g]);
+        if (t0 + g < t_end) fetch_tile(tbl, p, t0 + g, load_cursor, nullptr, wv[g]);
 #pragma unroll
       for (int g = 0; g < kScanGroup; ++g) {
         const int tile = t0 + g;
         if (tile >= t_end) break;
-        const int combo = combo_of_tile(tbl, tile);
+        const int combo = combo_of_tile(tbl, tile, cursor);
         const unsigned long long threshold = sh.prefix[combo];
         unsigned long long* cand = p.cand + static_cast<long long>(combo) * p.cand_stride;
         const int c0 = (tile - tbl.tile_begin[combo]) * kSelTile;
@@ -634,6 +673,7 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
 // ---------------------------------------------------------------------------------------
 size_t select_smem_bytes(long long L, int* bitmap_in_smem) {
   size_t bytes = 2 * static_cast<size_t>(kSelTile + kMaxWin) * sizeof(float);  // pooling tiles
+  static_assert(kSrcTileTokens * sizeof(float) <= kRankChunk * sizeof(unsigned long long), "");
   const size_t rank_bytes = kRankChunk * sizeof(unsigned long long);           // ranking chunk
   if (rank_bytes > bytes) bytes = rank_bytes;
   const size_t staged_bytes = kMaxKm * sizeof(int);                            // ranked cells

@@ -14,6 +14,7 @@ static constexpr int kMaxKm = 16384;        // largest K_m (bounds the candidate
 static constexpr int kSelectPasses = 6;     // 64-bit (value, index) key, 11/11/10 bits twice
 static constexpr int kSelThreads = 1024;    // threads per CTA of the selection kernel
 static constexpr int kSelTile = 4096;       // cells of one combination per work tile
+static constexpr int kSrcTileTokens = 8192; // tokens per work tile of the strided max-pool
 static constexpr int kRankKeysPerItem = kSelThreads / 32;   // candidates ranked per work item
 static constexpr int kSelBitmapSmemBytes = 136 * 1024;   // bitmap kept in shared memory up to this
 static constexpr int kSelMaxDynSmemBytes = kSelBitmapSmemBytes + kMaxKm * 4;
@@ -27,6 +28,13 @@ struct ComboTable {
   int k_m[kMaxCombos];     // candidates ranked for this combination
   int quota[kMaxCombos];   // B_c
   int tile_begin[kMaxCombos + 1];   // first work tile of each combination (prefix sums)
+  // Distinct strided max-pool sizes m > 1 ("sources"): their pooled arrays are computed once
+  // and shared by every window size.  src[c] = source of combination c, -1 = the scores.
+  int n_src;
+  int src[kMaxCombos];
+  int src_m[kMaxCombos];
+  int src_len[kMaxCombos];
+  int src_tile_begin[kMaxCombos + 1];   // tiles of kSrcTileTokens / m cells each
 };
 
 struct SelectParams {
@@ -36,6 +44,8 @@ struct SelectParams {
   long long L;
   int n_sink;
   int win_op;              // 0 average, 1 max
+  float* maxpooled;        // [n_src][maxpooled_stride] strided max-pool of the scores
+  long long maxpooled_stride;
   float* pooled;           // [n_comb][pooled_stride]
   long long pooled_stride;
   uint32_t* hist;          // [n_comb][kHistBins], zero on entry and on exit

@@ -88,6 +88,18 @@ CONFIGS = {
 PAPER_DEFAULT_MAX_SIZES = (2, 4, 8)
 PAPER_DEFAULT_WIN_SIZES = tuple(range(1, 17))
 
+# Supplementary timing rows on the L = 1M cache (not benchmark configurations):
+#   a short query (4 * q_len = 64 rows per kv head: 64 flop per key byte, below the ridge, so
+#   the key scan is HBM-bound), and the benchmark configuration under Algorithm 1's default
+#   pooling spec.
+CONFIGS["probe_L1m_q16"] = RecallWorkload(
+    "probe_L1m_q16", seed=5, L=1048576, q_len=16, n_spans=128, span_len=(8, 256), budget=4096,
+    win_sizes=(1, 7, 15, 31, 63))
+CONFIGS["cfg5_L1m_paper_pool"] = RecallWorkload(
+    "cfg5_L1m_paper_pool", seed=4, L=1048576, q_len=256, n_spans=128, span_len=(8, 256),
+    budget=4096, max_sizes=PAPER_DEFAULT_MAX_SIZES, win_sizes=PAPER_DEFAULT_WIN_SIZES, win_op=0,
+    n_sink=4)
+
 
 def _rope_inplace(x: torch.Tensor, pos0: int) -> torch.Tensor:
     """Rotate x [n, H, d] (fp32) by RoPE at positions pos0 .. pos0+n-1 (rotate-half form)."""
