@@ -341,7 +341,9 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
   sp.cand_count = h->cand_count; sp.ranked = h->ranked; sp.bitmap = h->bitmap;
   sp.out_idx = out_idx_dev; sp.budget = budget; sp.barrier = h->grid_barrier;
   sp.status = h->status;
-  const size_t select_smem = select_smem_bytes(L, &sp.bitmap_in_smem);
+  int max_km = 1;
+  for (int c = 0; c < tbl.n_comb; ++c) max_km = tbl.k_m[c] > max_km ? tbl.k_m[c] : max_km;
+  const size_t select_smem = select_smem_bytes(L, max_km, &sp);
   // Grid of the selection kernel: enough CTAs for the scan tiles and for the ranking
   // (K_m^2 comparisons per combination), but no more, since every grid barrier pays for them.
   long long want_grid = tbl.tile_begin[tbl.n_comb];

@@ -338,20 +338,70 @@ __device__ __forceinline__ void rank_range(const SelectParams& p, int combo, int
   }
 }
 
+// Bitmap word access of the quota walk.  The bitmap lives in shared memory on the common path;
+// naming the address space spares the generic-address forms.
+template <bool kSmem>
+__device__ __forceinline__ uint32_t bitmap_word(const uint32_t* bm, int w) {
+  if constexpr (kSmem) {
+    uint32_t v;
+    asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(bm + w)) : "memory");
+    return v;
+  } else {
+    return *reinterpret_cast<const volatile uint32_t*>(bm + w);
+  }
+}
+template <bool kSmem>
+__device__ __forceinline__ void bitmap_set(uint32_t* bm, int w, uint32_t bits) {
+  if constexpr (kSmem) {
+    asm volatile("red.shared.or.b32 [%0], %1;" ::"r"(smem_u32(bm + w)), "r"(bits) : "memory");
+  } else {
+    atomicOr(bm + w, bits);
+  }
+}
+
 // Tokens of cell `cell` (size m) that are not allocated yet, as a bit mask (bit j = token j).
-__device__ __forceinline__ unsigned long long fresh_tokens(const uint32_t* bm, long long cell,
-                                                           int m, long long Lp, int n_sink) {
+// Positions fit 32 bits (L < 2^31).
+template <bool kSmem>
+__device__ __forceinline__ unsigned long long fresh_tokens(const uint32_t* bm, int cell, int m,
+                                                           int Lp, int n_sink) {
+  if (m == 1) {
+    const int pos = n_sink + cell;
+    return ((bitmap_word<kSmem>(bm, pos >> 5) >> (pos & 31)) & 1u) ^ 1u;
+  }
   unsigned long long fresh = 0ull;
-  const long long t0 = cell * m;
-  for (int j = 0; j < m; ++j) {
-    const long long t = t0 + j;
-    if (t < Lp) {
-      const long long pos = n_sink + t;
-      const uint32_t word = *reinterpret_cast<const volatile uint32_t*>(&bm[pos >> 5]);
-      if (!((word >> (pos & 31)) & 1u)) fresh |= (1ull << j);
-    }
+  const int t0 = cell * m;
+  const int cnt = min(m, Lp - t0);
+  for (int j = 0; j < cnt; ++j) {
+    const int pos = n_sink + t0 + j;
+    const uint32_t taken = (bitmap_word<kSmem>(bm, pos >> 5) >> (pos & 31)) & 1u;
+    fresh |= static_cast<unsigned long long>(taken ^ 1u) << j;
   }
   return fresh;
+}
+
+// Exclusive prefix sum over the block with a single barrier: every warp scans the 32 warp
+// totals itself.  `slot` alternates between calls (two buffers), which keeps a call's readers
+// apart from the next call's writers.
+__device__ __forceinline__ uint32_t block_exclusive_scan_1(uint32_t v, uint32_t (*tot)[32],
+                                                           int slot, uint32_t* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  if (lane == 31) tot[slot][warp] = incl;
+  __syncthreads();
+  const uint32_t w = tot[slot][lane];
+  uint32_t wi = w;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, wi, o);
+    if (lane >= o) wi += t;
+  }
+  *total = __shfl_sync(0xFFFFFFFFu, wi, 31);
+  return __shfl_sync(0xFFFFFFFFu, wi - w, warp) + incl - v;
 }
 
 // Phase F (one CTA): quota walk over the ranked cells of every combination, then the
@@ -359,64 +409,87 @@ __device__ __forceinline__ unsigned long long fresh_tokens(const uint32_t* bm, l
 // `staged` room for kMaxKm cell ids in shared memory.  Every thread owns a run of consecutive
 // ranks; the cells of one combination are disjoint, so the new-token counts of all its cells
 // can be taken before any of them is marked.
+#ifdef ILRE_SELECT_TRACE
+#define ALLOC_TRACE(tag) do { if (combo < 2) SEL_TRACE(tag); } while (0)
+#define ALLOC_TRACE_ARGS , unsigned long long* trace_t, const char** trace_tag, int& trace_n
+#define ALLOC_TRACE_PASS , trace_t, trace_tag, trace_n
+#else
+#define ALLOC_TRACE(tag) do { } while (0)
+#define ALLOC_TRACE_ARGS
+#define ALLOC_TRACE_PASS
+#endif
+template <bool kBitmapInSmem>
 __device__ __forceinline__ void allocate(const ComboTable& tbl, const SelectParams& p,
-                                         uint32_t* bm, int* staged, SelShared* sh) {
-  const long long Lp = p.L - p.n_sink;
+                                         uint8_t* dyn_smem, SelShared* sh ALLOC_TRACE_ARGS) {
+  // Two instantiations, so that the compiler knows the bitmap's address space on the common
+  // path (shared memory) instead of going through generic loads and atomics.
+  uint32_t* bm;
+  int* staged;
+  if constexpr (kBitmapInSmem) {
+    bm = reinterpret_cast<uint32_t*>(dyn_smem);
+    staged = reinterpret_cast<int*>(dyn_smem + ((((p.L + 31) / 32) * 4 + 15) & ~15ll));
+  } else {
+    bm = p.bitmap;
+    staged = reinterpret_cast<int*>(dyn_smem);
+  }
+  __shared__ uint32_t warp_totals[2][32];
+  const int Lp = static_cast<int>(p.L - p.n_sink);
   for (int combo = threadIdx.x; combo < tbl.n_comb; combo += kSelThreads)
     sh->state[combo] = __ldcg(&p.cand_count[combo]);
   __syncthreads();
-  // The ranked cells of the next combination are fetched into registers while the current
-  // one is walked (kPre per thread cover K_m up to kPre * kSelThreads; the rest is loaded late).
-  constexpr int kPre = 5;
-  int pre[kPre];
   auto candidates = [&](int combo) {
     return min(static_cast<int>(min(sh->state[combo], static_cast<uint32_t>(kMaxKm))),
                tbl.k_m[combo]);
   };
-  auto prefetch = [&](int combo) {
+  // The ranked cells of a combination are copied to shared memory asynchronously; with two
+  // staging buffers the copy of the next combination runs under the walk of the current one.
+  int* const stage_odd = p.stage_double ? staged + p.stage_capacity : staged;
+  auto issue_copy = [&](int combo) {
     const int K = candidates(combo);
     const int* ranked = p.ranked + static_cast<long long>(combo) * p.cand_stride;
-#pragma unroll
-    for (int k = 0; k < kPre; ++k) {
-      const int r = k * kSelThreads + threadIdx.x;
-      pre[k] = (r < K) ? __ldcg(&ranked[r]) : 0;
-    }
+    int* dst = (combo & 1) ? stage_odd : staged;
+    for (int r = threadIdx.x; r < K; r += kSelThreads)
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst + r)),
+                   "l"(ranked + r) : "memory");
+    asm volatile("cp.async.commit_group;" ::: "memory");
   };
-  if (tbl.n_comb > 0) prefetch(0);
+  if (tbl.n_comb > 0) issue_copy(0);
   for (int combo = 0; combo < tbl.n_comb; ++combo) {
     const int m = tbl.m[combo];
     const uint32_t quota = static_cast<uint32_t>(tbl.quota[combo]);
     const int K = candidates(combo);
-    const int* ranked = p.ranked + static_cast<long long>(combo) * p.cand_stride;
-#pragma unroll
-    for (int k = 0; k < kPre; ++k) {
-      const int r = k * kSelThreads + threadIdx.x;
-      if (r < K) staged[r] = pre[k];
-    }
-    for (int r = kPre * kSelThreads + threadIdx.x; r < K; r += kSelThreads)
-      staged[r] = __ldcg(&ranked[r]);
-    if (combo + 1 < tbl.n_comb) prefetch(combo + 1);
+    const int* cells = (combo & 1) ? stage_odd : staged;
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
+    if (p.stage_double && combo + 1 < tbl.n_comb) issue_copy(combo + 1);
+    ALLOC_TRACE("a:staged");
     const int per = (K + kSelThreads - 1) / kSelThreads;
     const int r0 = min(K, static_cast<int>(threadIdx.x) * per), r1 = min(K, r0 + per);
     uint32_t mine = 0;
-    for (int r = r0; r < r1; ++r) mine += __popcll(fresh_tokens(bm, staged[r], m, Lp, p.n_sink));
+    for (int r = r0; r < r1; ++r)
+      mine += __popcll(fresh_tokens<kBitmapInSmem>(bm, cells[r], m, Lp, p.n_sink));
     uint32_t total;
-    uint32_t ord = block_exclusive_scan(mine, sh->scan, &total);
+    uint32_t ord = block_exclusive_scan_1(mine, warp_totals, combo & 1, &total);
+    ALLOC_TRACE("a:counted");
     for (int r = r0; r < r1 && ord < quota; ++r) {
-      const long long cell = staged[r];
-      unsigned long long fresh = fresh_tokens(bm, cell, m, Lp, p.n_sink);
+      const int cell = cells[r];
+      unsigned long long fresh = fresh_tokens<kBitmapInSmem>(bm, cell, m, Lp, p.n_sink);
       while (fresh && ord < quota) {                         // ascending position inside the cell
         const int j = __ffsll(static_cast<long long>(fresh)) - 1;
         fresh &= fresh - 1;
-        const long long pos = p.n_sink + cell * m + j;
-        atomicOr(&bm[pos >> 5], 1u << (pos & 31));
+        const int pos = p.n_sink + cell * m + j;
+        bitmap_set<kBitmapInSmem>(bm, pos >> 5, 1u << (pos & 31));
         ++ord;
       }
     }
     if (total < quota && threadIdx.x == 0) atomicCAS(p.status, 0, kDevQuota);
     __syncthreads();                                         // bitmap updates visible to the block
+    if (!p.stage_double && combo + 1 < tbl.n_comb) issue_copy(combo + 1);
+    ALLOC_TRACE("a:marked");
   }
+#ifdef ILRE_SELECT_TRACE
+  SEL_TRACE("a:rest");
+#endif
 
   // Ascending output.  Every warp owns a contiguous run of bitmap words and reads it 32
   // consecutive words at a time (one per lane).
@@ -427,7 +500,7 @@ __device__ __forceinline__ void allocate(const ComboTable& tbl, const SelectPara
   uint32_t count = 0;
   for (long long k = 0; k < rounds; ++k) {
     const long long w = w_begin + k * 32 + lane;
-    if (w < n_words) count += __popc(*reinterpret_cast<volatile uint32_t*>(&bm[w]));
+    if (w < n_words) count += __popc(bitmap_word<kBitmapInSmem>(bm, static_cast<int>(w)));
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) count += __shfl_xor_sync(0xFFFFFFFFu, count, o);
@@ -437,7 +510,7 @@ __device__ __forceinline__ void allocate(const ComboTable& tbl, const SelectPara
   const uint32_t cap = static_cast<uint32_t>(p.n_sink + p.budget);
   for (long long k = 0; k < rounds; ++k) {
     const long long w = w_begin + k * 32 + lane;
-    uint32_t bits = (w < n_words) ? *reinterpret_cast<volatile uint32_t*>(&bm[w]) : 0u;
+    uint32_t bits = (w < n_words) ? bitmap_word<kBitmapInSmem>(bm, static_cast<int>(w)) : 0u;
     uint32_t incl = __popc(bits);
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -645,12 +718,9 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
 
   // ---- F: allocation and ascending output (one CTA) ----
   if (blockIdx.x != 0) return;
-  uint32_t* bm = p.bitmap;
-  int* staged = reinterpret_cast<int*>(dyn_smem);
   if (p.bitmap_in_smem) {
-    bm = reinterpret_cast<uint32_t*>(dyn_smem);
+    uint32_t* bm = reinterpret_cast<uint32_t*>(dyn_smem);
     const long long n_words = (p.L + 31) / 32;
-    staged = reinterpret_cast<int*>(dyn_smem + ((n_words * 4 + 15) & ~15ll));
     for (long long w = threadIdx.x; w < n_words; w += kSelThreads) {
       const long long lo = w * 32;
       uint32_t bits = 0;
@@ -658,8 +728,11 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
       bm[w] = bits;
     }
     __syncthreads();
+    SEL_TRACE("bitmap init");
+    allocate<true>(tbl, p, dyn_smem, &sh ALLOC_TRACE_PASS);
+  } else {
+    allocate<false>(tbl, p, dyn_smem, &sh ALLOC_TRACE_PASS);
   }
-  allocate(tbl, p, bm, staged, &sh);
   SEL_TRACE("allocate");
 #ifdef ILRE_SELECT_TRACE
   if (threadIdx.x == 0)
@@ -671,15 +744,19 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
 // ---------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------
-size_t select_smem_bytes(long long L, int* bitmap_in_smem) {
+size_t select_smem_bytes(long long L, int max_km, SelectParams* p) {
   size_t bytes = 2 * static_cast<size_t>(kSelTile + kMaxWin) * sizeof(float);  // pooling tiles
   static_assert(kSrcTileTokens * sizeof(float) <= kRankChunk * sizeof(unsigned long long), "");
   const size_t rank_bytes = kRankChunk * sizeof(unsigned long long);           // ranking chunk
   if (rank_bytes > bytes) bytes = rank_bytes;
-  const size_t staged_bytes = kMaxKm * sizeof(int);                            // ranked cells
+  // quota walk: bitmap (when it fits) + one or two staging buffers of max_km cell ids
+  const size_t cap = (static_cast<size_t>(max_km < 1 ? 1 : max_km) + 3) & ~size_t(3);
   const size_t bm_bytes = (static_cast<size_t>((L + 31) / 32) * sizeof(uint32_t) + 15) & ~size_t(15);
-  *bitmap_in_smem = bm_bytes <= static_cast<size_t>(kSelBitmapSmemBytes) ? 1 : 0;
-  const size_t alloc_bytes = staged_bytes + (*bitmap_in_smem ? bm_bytes : 0);
+  p->bitmap_in_smem = bm_bytes <= static_cast<size_t>(kSelBitmapSmemBytes) ? 1 : 0;
+  const size_t base = p->bitmap_in_smem ? bm_bytes : 0;
+  p->stage_capacity = static_cast<int>(cap);
+  p->stage_double = (base + 2 * cap * sizeof(int) <= static_cast<size_t>(kSelMaxDynSmemBytes)) ? 1 : 0;
+  const size_t alloc_bytes = base + (p->stage_double ? 2 : 1) * cap * sizeof(int);
   if (alloc_bytes > bytes) bytes = alloc_bytes;
   return bytes;
 }

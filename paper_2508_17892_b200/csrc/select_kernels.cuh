@@ -58,6 +58,8 @@ struct SelectParams {
   int* ranked;             // [n_comb][cand_stride] cell ids in rank order
   uint32_t* bitmap;        // [ceil(L/32)] in global memory, used when it does not fit shared memory
   int bitmap_in_smem;
+  int stage_capacity;      // cell ids per staging buffer of the quota walk (>= largest K_m)
+  int stage_double;        // two staging buffers fit shared memory
   int* out_idx;            // [n_sink + budget]
   int budget;
   uint32_t* barrier;       // grid barrier arrival counter, zero when the kernel starts
@@ -65,7 +67,8 @@ struct SelectParams {
 };
 
 // Dynamic shared memory the kernel needs for a context of L positions.
-size_t select_smem_bytes(long long L, int* bitmap_in_smem);
+// Also fills p->bitmap_in_smem, p->stage_capacity and p->stage_double.
+size_t select_smem_bytes(long long L, int max_km, SelectParams* p);
 // Largest grid that is co-resident on the device (the kernel's CTAs wait on one another).
 cudaError_t select_max_grid(int n_sm, int* max_grid);
 // One cooperative launch: A^C from the encoded maxima, then all of Algorithm 1.
