@@ -54,6 +54,8 @@ def _load():
         lib.ilre_oracle_allocate.argtypes = [c_f64p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
                                              c_i32p, ctypes.c_int, c_i32p, ctypes.c_int,
                                              ctypes.c_int, c_i32p, c_i32p, c_i32p, c_f64p, c_f64p]
+        lib.ilre_oracle_dca_rerope.argtypes = [c_u16p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
+                                               ctypes.c_int, ctypes.c_int, ctypes.c_double, c_f64p]
         _lib = lib
     return _lib
 
@@ -168,3 +170,22 @@ def recall(K, Q, budget: int, max_sizes: Sequence[int], win_sizes: Sequence[int]
     """The whole path: (ascending indices, A^C)."""
     a = scores(K, Q)
     return allocate(a, budget, max_sizes, win_sizes, win_op, n_sink), a
+
+
+def dca_rerope(K, chunk: int, n_sink: int = 0, theta: float = 500000.0) -> np.ndarray:
+    """Eq. 7: the cached keys re-rotated chunk by chunk (fp64, not rounded)."""
+    k = _u16(K)
+    L, n_kv, d = k.shape
+    out = np.empty((L, n_kv, d), dtype=np.float64)
+    rc = _load().ilre_oracle_dca_rerope(_p(k, ctypes.c_uint16), L, n_kv, d, chunk, n_sink,
+                                        float(theta), _p(out, ctypes.c_double))
+    if rc != 0:
+        raise RuntimeError(f"ilre_oracle_dca_rerope failed: {rc}")
+    return out
+
+
+def round_to_bf16(x: np.ndarray) -> np.ndarray:
+    """Round fp64 values to the nearest bf16 (ties to even); returns the uint16 patterns."""
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float64)).to(torch.bfloat16)
+    return t.contiguous().view(torch.int16).numpy().view(np.uint16)

@@ -35,6 +35,18 @@
  * special case (one size-1 max kernel, one average kernel) equals a plain top-B; a
  * hand-worked Algorithm 1 example; quota/unique/ascending invariants; needle recovery.
  * The paper prints no worked numerical example of this path, so none is pinned.
+ *
+ * Also here: Eq. 7, the re-rotation of the retrieval layer's cached keys under Dual Chunk
+ * Attention (ilre_oracle_dca_rerope), with these readings:
+ *   R13 chunks: chunk 1 holds the n_sink sink tokens plus `chunk` tokens, every later chunk
+ *       `chunk` tokens (the last one possibly fewer); N_C = ceil((L - n_sink) / chunk).
+ *   R14 D_i = (N_C - 1 - i) * chunk positions for i < N_C - 1, nothing for the last two chunks.
+ *   R15 R(D) is the RoPE rotation by D positions in the rotate-half layout: channel pair
+ *       (c, c + d/2) turns by the angle D * theta^(-2c/d).
+ * Pins (tests/test_oracle_dca.py): a hand-computed pair rotation; pair norms are kept; the
+ * last two chunks are untouched; rotating a key that carries RoPE at position p gives the
+ * key with RoPE at position p + D (against an independent RoPE routine); the logit identity
+ * q . R(D) k = (R(-D) q) . k; keys that differ only by whole chunks become equal.
  */
 #include <math.h>
 #include <stdint.h>
@@ -275,4 +287,37 @@ int ilre_oracle_allocate(const double *A, int64_t L, int n_sink, int budget,
     if (rc == 0 && w != (int64_t)n_sink + budget) rc = -3;
     free(in_I); free(P); free(W); free(rk);
     return rc;
+}
+
+
+/*
+ * Eq. 7: K~[t] = R(D_i) K[t] for every position t of chunk i < N_C - 1 (readings R13-R15).
+ * K is bf16 [L][n_kv][d]; out is double [L][n_kv][d] (exact rotation of the bf16 values,
+ * not rounded back).  Returns 0, or -1 on bad arguments.
+ */
+int ilre_oracle_dca_rerope(const uint16_t *K, int64_t L, int n_kv, int d, int chunk, int n_sink,
+                           double theta, double *out)
+{
+    if (!K || !out || L < 1 || n_kv < 1 || d < 2 || (d & 1) || chunk < 1 || n_sink < 0 ||
+        n_sink > L)
+        return -1;
+    const int half = d / 2;
+    const int64_t n_chunks = (L - n_sink + chunk - 1) / chunk;                     /* R13 */
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < L; ++t) {
+        int64_t i = (t < n_sink) ? 1 : 1 + (t - n_sink) / chunk;                  /* 1-based */
+        const double D = (i < n_chunks - 1) ? (double)((n_chunks - 1 - i) * chunk) : 0.0; /* R14 */
+        for (int g = 0; g < n_kv; ++g) {
+            const uint16_t *k = K + (t * n_kv + g) * d;
+            double *o = out + (t * n_kv + g) * d;
+            for (int c = 0; c < half; ++c) {
+                const double ang = D * pow(theta, -2.0 * (double)c / (double)d);  /* R15 */
+                const double cs = cos(ang), sn = sin(ang);
+                const double lo = bf16_to_double(k[c]), hi = bf16_to_double(k[c + half]);
+                o[c] = lo * cs - hi * sn;
+                o[c + half] = lo * sn + hi * cs;
+            }
+        }
+    }
+    return 0;
 }
