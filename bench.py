@@ -268,6 +268,31 @@ def run_ours(args, world, rank, local):
                    h2d_bytes_per_step=int(k_bytes + Q.numel() * 2),
                    d2h_bytes_per_step=int(idx_h.numel() * 4), steps=e2e_steps)
 
+    # Dual Chunk Attention re-rotation of the cache (Eq. 7), timed on its own: an HBM-bound
+    # streaming kernel, in place on a scratch copy of K
+    dca = None
+    if args.dca_chunk > 0 and rank == 0:
+        Kc = K.clone()
+        n_chunks = -(-(w.L - w.n_sink) // args.dca_chunk)
+        rotated = max(0, min(w.L, w.n_sink + (n_chunks - 2) * args.dca_chunk))
+        for _ in range(3):
+            eng.rerope_keys(Kc, args.dca_chunk, w.n_sink)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 20
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(reps):
+            eng.rerope_keys(Kc, args.dca_chunk, w.n_sink)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        moved = 2.0 * rotated * w.n_kv_heads * w.d * 2              # read + write
+        dca = dict(kernel="rerope_kernel", chunk=args.dca_chunk, ms=ms,
+                   algorithmic_bytes=moved, achieved=moved / (ms * 1e-3) / 1e9, unit="GB/s",
+                   bound="hbm", peak=measured_peaks()["hbm_gbs"],
+                   frac=moved / (ms * 1e-3) / 1e9 / measured_peaks()["hbm_gbs"])
+        del Kc
+
     elapsed_max, units = aggregate(elapsed_ms, float(k_bytes) * args.steps, dev)
     if rank != 0:
         return
@@ -318,7 +343,7 @@ def run_ours(args, world, rank, local):
                             parallelism="replicas only" if world > 1 else "single GPU"),
                 clocks=clocks, e2e=e2e, gpu_launches=launches, roofline=roofline,
                 cpu_baseline=cpu_baseline,
-                stages_ms=stages,
+                stages_ms=stages, dca_rerope=dca,
                 whole_step=dict(hbm_frac_one_read_of_K=step_hbm_frac,
                                 tensor_frac_one_qk=step_tensor_frac,
                                 hbm_frac_of_8TBps=(k_bytes / (ms_per_step * 1e-3) / 1e9) / 8000.0))
@@ -337,6 +362,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--L", type=int, default=0,
                     help="override the context length of --config (profiling on a small case)")
+    ap.add_argument("--dca-chunk", type=int, default=1024,
+                    help="also time the Eq. 7 key re-rotation with this chunk size (0 = skip)")
     ap.add_argument("--cpu-sample-keys", type=int, default=131072)
     ap.add_argument("--ref-sample-keys", type=int, default=4096)
     args = ap.parse_args()

@@ -107,6 +107,26 @@ int ilre_recall_run_host(ilre_recall_t* h,
                          void* cuda_stream);
 
 /*
+ * Dual Chunk Attention re-rotation of the retrieval layer's cached keys (Section 3.3, Eq. 7),
+ * to be applied before ilre_recall_run when DCA is on:
+ *   K~[t] = R(D_i) K[t]  for every position t of chunk i < N_C - 1,  D_i = (N_C - 1 - i) * chunk_size,
+ * where chunk 1 holds the n_sink sink tokens plus chunk_size tokens, every later chunk
+ * chunk_size tokens (the last possibly fewer), N_C = ceil((L - n_sink) / chunk_size), and R(D)
+ * is the RoPE rotation by D positions in the rotate-half layout (channel pair (c, c + 64) turns
+ * by D * rope_theta^(-2c/128)).  The last two chunks stay as they are.
+ *   k_cache_dev  bf16 [L][n_kv_heads][128], 16-byte aligned
+ *   k_out_dev    same shape; may be k_cache_dev itself (in place) or a separate buffer, in
+ *                which case the unrotated chunks are copied
+ * Arithmetic: fp32 from an angle table computed in double precision, one rounding to bf16
+ * (nearest even).  Asynchronous on cuda_stream.  At most 8192 + 2 chunks
+ * (ILRE_ERR_CAPACITY beyond).  The handle keeps the angle table between calls, so calls on
+ * one handle must not overlap.
+ */
+int ilre_recall_rerope_keys(ilre_recall_t* h, const void* k_cache_dev, void* k_out_dev,
+                            int64_t L, int32_t chunk_size, int32_t n_sink, double rope_theta,
+                            void* cuda_stream);
+
+/*
  * Row statistics of the last run (Eq. 4's softmax denominator): copies
  * lse[i * n_q_heads + h] = log(sum_t exp(s[h,i,t])) (natural log, fp32) for the q_len rows
  * of that run into out_lse_dev, asynchronously on cuda_stream.

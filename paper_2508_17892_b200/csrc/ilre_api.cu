@@ -10,6 +10,7 @@
 
 #include "../../include/ilre_recall.h"
 #include "qk_kernels.cuh"
+#include "rerope_kernels.cuh"
 #include "select_kernels.cuh"
 #include "sm100_ptx.cuh"
 
@@ -50,6 +51,9 @@ struct ilre_recall {
   uint32_t* sel_krem;
   uint32_t* sel_done;
   uint32_t* grid_barrier;
+  float2* rope_table;                   // (cos, sin) per (chunk distance, channel pair)
+  int rope_rows, rope_chunk;            // what the table currently holds
+  double rope_theta;
   unsigned long long* cand;
   uint32_t* cand_count;
   int* ranked;
@@ -116,7 +120,7 @@ bool dev_alloc(T** p, size_t count) {
 void free_all(ilre_recall* h) {
   cudaFree(h->qp); cudaFree(h->partial); cudaFree(h->nlse2); cudaFree(h->row_lse);
   cudaFree(h->enc); cudaFree(h->scores); cudaFree(h->pooled); cudaFree(h->maxpooled); cudaFree(h->hist);
-  cudaFree(h->sel_prefix); cudaFree(h->sel_krem); cudaFree(h->sel_done); cudaFree(h->grid_barrier);
+  cudaFree(h->sel_prefix); cudaFree(h->sel_krem); cudaFree(h->sel_done); cudaFree(h->grid_barrier); cudaFree(h->rope_table);
   cudaFree(h->cand); cudaFree(h->cand_count); cudaFree(h->ranked); cudaFree(h->bitmap);
   cudaFree(h->status); cudaFree(h->stage_k); cudaFree(h->stage_q); cudaFree(h->stage_idx);
   for (int r = 0; r < kProfRing; ++r)
@@ -229,6 +233,7 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out) {
   ok = ok && dev_alloc(&h->sel_krem, ncomb);
   ok = ok && dev_alloc(&h->sel_done, ncomb);
   ok = ok && dev_alloc(&h->grid_barrier, 1);
+  ok = ok && dev_alloc(&h->rope_table, static_cast<size_t>(kRopeTableRows) * kRopeHalfDim);
   ok = ok && dev_alloc(&h->cand, ncomb * h->cand_stride);
   ok = ok && dev_alloc(&h->cand_count, ncomb);
   ok = ok && dev_alloc(&h->ranked, ncomb * h->cand_stride);
@@ -404,6 +409,41 @@ int ilre_recall_run_host(ilre_recall_t* h, const void* k_cache_host, int64_t L,
     ILRE_CUDA(cudaMemcpyAsync(out_scores_host, h->scores, static_cast<size_t>(L) * sizeof(float),
                               cudaMemcpyDeviceToHost, st));
   ILRE_CUDA(cudaStreamSynchronize(st));
+  return ILRE_OK;
+}
+
+int ilre_recall_rerope_keys(ilre_recall_t* h, const void* k_cache_dev, void* k_out_dev, int64_t L,
+                            int32_t chunk_size, int32_t n_sink, double rope_theta,
+                            void* cuda_stream) {
+  if (!h || !k_cache_dev || !k_out_dev || L < 1 || chunk_size < 1 || n_sink < 0 || n_sink > L ||
+      !(rope_theta > 1.0))
+    return ILRE_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(k_cache_dev) & 15u) || (reinterpret_cast<uintptr_t>(k_out_dev) & 15u))
+    return ILRE_ERR_ALIGNMENT;
+  const long long n_chunks = (L - n_sink + chunk_size - 1) / chunk_size;
+  const long long n_rows = n_chunks - 2;               // distinct non-zero distances D_i
+  if (n_rows > kRopeTableRows) return ILRE_ERR_CAPACITY;
+  if (n_rows < 1 && k_out_dev == k_cache_dev) return ILRE_OK;    // nothing moves
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return ILRE_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  h->last_stream = st;
+  int launches = 0;
+  // The table depends on (chunk, theta) only; rows beyond what an earlier call built are
+  // the reason to rebuild.  Rebuilding is stream-ordered before the rotation.
+  if (n_rows > 0 && (h->rope_chunk != chunk_size || h->rope_theta != rope_theta ||
+                     h->rope_rows < n_rows)) {
+    ILRE_CUDA(launch_rope_table(h->rope_table, static_cast<int>(n_rows), chunk_size, rope_theta, st));
+    h->rope_chunk = chunk_size; h->rope_theta = rope_theta; h->rope_rows = static_cast<int>(n_rows);
+    ++launches;
+  }
+  ReropeParams rp;
+  rp.k_in = static_cast<const uint4*>(k_cache_dev);
+  rp.k_out = static_cast<uint4*>(k_out_dev);
+  rp.L = L; rp.n_kv = h->cfg.n_kv_heads; rp.chunk = chunk_size; rp.n_sink = n_sink;
+  rp.n_chunks = n_chunks; rp.table = h->rope_table;
+  ILRE_CUDA(launch_rerope(rp, h->n_sm, st)); ++launches;
+  h->last_launches = launches;
   return ILRE_OK;
 }
 

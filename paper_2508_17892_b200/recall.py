@@ -18,7 +18,8 @@ LIB_PATH = os.path.join(_HERE, "libilre_recall.so")
 STAGE_NAMES = ("prepare", "row_stats", "merge_stats", "scores", "select")
 
 EXPORTED_SYMBOLS = (
-    "ilre_recall_create", "ilre_recall_run", "ilre_recall_run_host", "ilre_recall_copy_row_lse",
+    "ilre_recall_create", "ilre_recall_run", "ilre_recall_run_host", "ilre_recall_rerope_keys",
+    "ilre_recall_copy_row_lse",
     "ilre_recall_status", "ilre_recall_set_profiling", "ilre_recall_stage_times",
     "ilre_recall_last_launch_count", "ilre_recall_destroy", "ilre_strerror",
     "ilre_topk_positions_noalloc",
@@ -64,6 +65,7 @@ def load_library() -> ctypes.CDLL:
     lib.ilre_recall_create.argtypes = [ctypes.POINTER(IlreConfig), ctypes.POINTER(vp)]
     lib.ilre_recall_run.argtypes = [vp, vp, i64, vp, i32, i32, ctypes.POINTER(IlrePoolSpec), vp, vp, vp]
     lib.ilre_recall_run_host.argtypes = lib.ilre_recall_run.argtypes
+    lib.ilre_recall_rerope_keys.argtypes = [vp, vp, vp, i64, i32, i32, ctypes.c_double, vp]
     lib.ilre_recall_copy_row_lse.argtypes = [vp, vp, i32, vp]
     lib.ilre_recall_status.argtypes = [vp]
     lib.ilre_recall_set_profiling.argtypes = [vp, i32]
@@ -179,6 +181,24 @@ class IlreRecall:
         if rc != 0:
             raise IlreError(rc, "ilre_recall_run_host")
         return out_idx, out_scores
+
+    def rerope_keys(self, K: torch.Tensor, chunk_size: int, n_sink: int = 0,
+                    rope_theta: float = 500000.0, out: Optional[torch.Tensor] = None,
+                    stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        """Eq. 7 (Dual Chunk Attention): re-rotate the cached keys chunk by chunk.  In place
+        unless ``out`` is given.  Returns the tensor that holds the result."""
+        dst = K if out is None else out
+        for t in (K, dst):
+            assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+            assert t.shape[1:] == (self.cfg.n_kv_heads, self.cfg.head_dim)
+        assert dst.shape == K.shape
+        st = stream if stream is not None else torch.cuda.current_stream(self.device)
+        rc = self._lib.ilre_recall_rerope_keys(self._h, K.data_ptr(), dst.data_ptr(), K.shape[0],
+                                               chunk_size, n_sink, float(rope_theta),
+                                               st.cuda_stream)
+        if rc != 0:
+            raise IlreError(rc, "ilre_recall_rerope_keys")
+        return dst
 
     # -- diagnostics -------------------------------------------------------------------
     def row_lse(self, q_len: int, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:

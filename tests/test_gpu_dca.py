@@ -1,0 +1,112 @@
+"""GPU parity of the Dual Chunk Attention key re-rotation (Eq. 7) against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import parity
+from workloads import make_inputs, small_workload
+
+pytestmark = pytest.mark.gpu
+
+# One bf16 rounding of an fp32 result: half a unit in the last place is at most 2^-8 of the
+# value (8 significant bits).  Before it, the fp32 rotation carries an absolute error of a few
+# 2^-24 of the INPUT magnitudes (two products, one sum, an fp32 table entry), which matters
+# where the two products cancel: inputs here stay below 16, hence 16 * 4 * 2^-24 ~ 4e-6.
+REL_TOL = 2.0 ** -8 * (1 + 1e-3)
+ABS_TOL = 4e-6
+
+
+def _engine(n_kv=8, n_q=32, max_L=70000):
+    from paper_2508_17892_b200 import IlreRecall
+    return IlreRecall(max_L=max_L, max_q_len=64, max_budget=512, n_kv_heads=n_kv, n_q_heads=n_q)
+
+
+def _as_f64(t: torch.Tensor) -> np.ndarray:
+    return t.cpu().to(torch.float64).numpy()
+
+
+CASES = [
+    # L, n_kv, chunk, n_sink
+    (4096, 8, 1024, 0),
+    (5000, 8, 1024, 4),          # ragged last chunk, sink in the first chunk
+    (777, 2, 64, 4),
+    (300, 8, 100, 0),            # N_C = 3: only the first chunk turns
+    (200, 8, 100, 0),            # N_C = 2: nothing turns
+    (65, 1, 1, 3),               # chunk of one position
+    (65552, 8, 8, 0),            # 8194 chunks: exactly the capacity of the angle table
+]
+
+
+@pytest.mark.parametrize("case", CASES, ids=lambda c: f"L{c[0]}_kv{c[1]}_c{c[2]}_s{c[3]}")
+def test_rerope_matches_oracle(case):
+    L, n_kv, chunk, n_sink = case
+    g = torch.Generator().manual_seed(L + chunk)
+    K = (torch.randn(L, n_kv, 128, generator=g) * 2.0).to(torch.bfloat16)
+    want = oracle.dca_rerope(K, chunk, n_sink)
+    eng = _engine(n_kv=n_kv, n_q=n_kv * 4, max_L=max(L, 4096))
+    Kd = K.cuda()
+    out = torch.empty_like(Kd)
+    eng.rerope_keys(Kd, chunk, n_sink, out=out)            # separate output
+    inplace = Kd.clone()
+    eng.rerope_keys(inplace, chunk, n_sink)                # in place
+    torch.cuda.synchronize()
+    eng.check_status()
+    assert torch.equal(out, inplace)
+    assert torch.equal(Kd.cpu(), K)                        # the input of the first call is intact
+    got = _as_f64(out)
+    err = np.abs(got - want)
+    assert np.all(err <= REL_TOL * np.abs(want) + ABS_TOL), float((err / (np.abs(want) + 1e-30)).max())
+    # almost every element is the correctly rounded value of the exact rotation
+    exact = oracle.round_to_bf16(want)
+    same = out.cpu().view(torch.int16).numpy().view(np.uint16) == exact
+    assert same.mean() > 0.999, same.mean()
+    # the last two chunks are bit-identical to the input
+    n_chunks = -(-(L - n_sink) // chunk)
+    keep_from = n_sink + max(n_chunks - 2, 0) * chunk
+    assert torch.equal(out[keep_from:].cpu(), K[keep_from:])
+    eng.close()
+
+
+def test_too_many_chunks_is_refused():
+    from paper_2508_17892_b200 import IlreError
+    eng = _engine(max_L=70000)
+    K = torch.zeros(66000, 8, 128, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(IlreError) as e:
+        eng.rerope_keys(K, 4)                              # 16500 chunks > 8192 + 2
+    assert e.value.code == -3
+    with pytest.raises(IlreError) as e:
+        eng.rerope_keys(K, 0)
+    assert e.value.code == -1
+    eng.close()
+
+
+def test_recall_on_rerotated_keys_matches_oracle():
+    # Eq. 7 followed by the recall: the oracle runs on the oracle's own re-rotated keys (rounded
+    # to bf16, as a cache holds them); the device output may differ from that rounding in rare
+    # elements by one unit in the last place, so its scores are checked at the score tolerance.
+    w = small_workload(6000, 16, seed=11, n_spans=3, span_len=(16, 32), budget=256,
+                       win_sizes=(1, 7, 15), win_op=1)
+    x = make_inputs(w)
+    chunk, n_sink = 1024, 0
+    ref_keys = torch.from_numpy(oracle.round_to_bf16(oracle.dca_rerope(x.K, chunk, n_sink))
+                                .view(np.int16)).view(torch.bfloat16).reshape(x.K.shape)
+    from paper_2508_17892_b200 import IlreRecall
+    eng = IlreRecall(max_L=w.L, max_q_len=w.q_len, max_budget=w.budget)
+    Kd = x.K.cuda()
+    eng.rerope_keys(Kd, chunk, n_sink)
+    idx, sc = eng.run(Kd, x.Q.cuda(), w.budget, w.max_sizes, w.win_sizes, w.win_op, w.n_sink,
+                      want_scores=True)
+    torch.cuda.synchronize()
+    eng.check_status()
+    # exact parity of the recall itself on the device's own re-rotated keys
+    parity.check_recall(Kd.cpu(), x.Q, w, idx.cpu().numpy(), sc.cpu().numpy())
+    # and against the all-oracle pipeline: a key that differs by one bf16 unit moves a logit by
+    # at most |q_c| * 2^-8 |k_c| / sqrt(d), far below what separates planted spans from the rest
+    ref_idx, ref_scores = oracle.recall(ref_keys, x.Q, w.budget, w.max_sizes, w.win_sizes, w.win_op,
+                                        w.n_sink)
+    rel = np.abs(sc.cpu().numpy() - ref_scores) / ref_scores
+    assert np.quantile(rel, 0.999) < 2e-3 and rel.max() < 0.05
+    planted = set(x.planted_positions().tolist())
+    assert len(planted & set(idx.cpu().tolist())) == len(planted & set(ref_idx.tolist()))
+    eng.close()
