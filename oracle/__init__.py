@@ -189,3 +189,32 @@ def round_to_bf16(x: np.ndarray) -> np.ndarray:
     import torch
     t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float64)).to(torch.bfloat16)
     return t.contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def key_fill(X, W, pos0: int, theta: float = 500000.0, bias=None) -> np.ndarray:
+    """Eq. 1 + Eq. 3 for the keys of the retrieval layer: K = PE(X W_K^T (+ b)), fp64.
+
+    X: bf16 [n_tok, d_model] hidden states of the tokens at positions pos0 .. pos0 + n_tok - 1;
+    W: bf16 [n_kv * d_h, d_model] (one row per output channel); bias: optional bf16
+    [n_kv * d_h].  PE is RoPE in the rotate-half layout of the cache (pair (c, c + d_h/2) of
+    every head turns by pos * theta^(-2c/d_h)), d_h = 128.  Returns fp64 [n_tok, n_kv, 128],
+    not rounded.  The matrix product is numpy's fp64 matmul (a library step)."""
+    import torch
+    x = X.to(torch.float64).numpy() if hasattr(X, "numpy") else np.asarray(X, dtype=np.float64)
+    w = W.to(torch.float64).numpy() if hasattr(W, "numpy") else np.asarray(W, dtype=np.float64)
+    d_h = 128
+    n_tok, n_out = x.shape[0], w.shape[0]
+    assert n_out % d_h == 0 and x.shape[1] == w.shape[1]
+    y = x @ w.T
+    if bias is not None:
+        b = bias.to(torch.float64).numpy() if hasattr(bias, "numpy") else np.asarray(bias)
+        y = y + b[None, :]
+    y = y.reshape(n_tok, n_out // d_h, d_h)
+    half = d_h // 2
+    inv_freq = np.power(float(theta), -2.0 * np.arange(half, dtype=np.float64) / d_h)
+    ang = (pos0 + np.arange(n_tok, dtype=np.float64))[:, None] * inv_freq[None, :]
+    cs, sn = np.cos(ang)[:, None, :], np.sin(ang)[:, None, :]
+    out = np.empty_like(y)
+    out[..., :half] = y[..., :half] * cs - y[..., half:] * sn
+    out[..., half:] = y[..., :half] * sn + y[..., half:] * cs
+    return out
