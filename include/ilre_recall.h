@@ -107,6 +107,27 @@ int ilre_recall_run_host(ilre_recall_t* h,
                          void* cuda_stream);
 
 /*
+ * Key-cache fill of the retrieval layer (Section 3.3: "calculate the key states for the context
+ * ... fill the cache with chunked key states"; Eq. 1 with the positional encoding of Eq. 3):
+ *   K[pos0 + t, g, :] = R(pos0 + t) (x[t, :] . W_K[g*128 : (g+1)*128, :]^T + b[g*128 : (g+1)*128])
+ * for t = 0 .. n_tok-1 and every kv head g, where R(p) is RoPE at position p in the
+ * rotate-half layout (pair (c, c + 64) turns by p * rope_theta^(-2c/128)).  One call fills the
+ * rows [pos0, pos0 + n_tok) of the cache, e.g. one prefill chunk.
+ *   x_dev        bf16 [n_tok][d_model] hidden states entering the key projection
+ *   w_k_dev      bf16 [n_kv_heads * 128][d_model], one row per output channel
+ *   bias_dev     bf16 [n_kv_heads * 128] or NULL
+ *   k_cache_dev  bf16 [L][n_kv_heads][128]; rows outside [pos0, pos0 + n_tok) are not touched
+ * d_model must be a multiple of 64 (ILRE_ERR_UNSUPPORTED), pos0 + n_tok <= L <= max_L
+ * (ILRE_ERR_CAPACITY), all three tensors 16-byte aligned.  bf16 x bf16 products accumulate in
+ * fp32 on the tensor cores; bias, rotation in fp32 from angle tables built in double precision;
+ * one rounding to bf16.  Asynchronous on cuda_stream; bounded waits report through
+ * ilre_recall_status.
+ */
+int ilre_recall_fill_keys(ilre_recall_t* h, const void* x_dev, int64_t n_tok, int32_t d_model,
+                          const void* w_k_dev, const void* bias_dev, int64_t pos0,
+                          double rope_theta, void* k_cache_dev, int64_t L, void* cuda_stream);
+
+/*
  * Dual Chunk Attention re-rotation of the retrieval layer's cached keys (Section 3.3, Eq. 7),
  * to be applied before ilre_recall_run when DCA is on:
  *   K~[t] = R(D_i) K[t]  for every position t of chunk i < N_C - 1,  D_i = (N_C - 1 - i) * chunk_size,

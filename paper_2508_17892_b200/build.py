@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ_DIR = os.path.join(HERE, "_build")
 LIB_PATH = os.path.join(HERE, "libilre_recall.so")
-SOURCES = ["ilre_api.cu", "qk_kernels.cu", "select_kernels.cu", "rerope_kernels.cu",
+SOURCES = ["ilre_api.cu", "qk_kernels.cu", "select_kernels.cu", "rerope_kernels.cu", "fill_kernels.cu",
            "topk_noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]

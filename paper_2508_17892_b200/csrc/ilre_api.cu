@@ -9,6 +9,7 @@
 #include <new>
 
 #include "../../include/ilre_recall.h"
+#include "fill_kernels.cuh"
 #include "qk_kernels.cuh"
 #include "rerope_kernels.cuh"
 #include "select_kernels.cuh"
@@ -54,6 +55,10 @@ struct ilre_recall {
   float2* rope_table;                   // (cos, sin) per (chunk distance, channel pair)
   int rope_rows, rope_chunk;            // what the table currently holds
   double rope_theta;
+  float2* pos_lo;                       // RoPE angle tables of the key-cache fill
+  float2* pos_hi;
+  int pos_hi_rows;
+  double pos_theta;                     // theta the tables were built for (0 = none)
   unsigned long long* cand;
   uint32_t* cand_count;
   int* ranked;
@@ -120,7 +125,7 @@ bool dev_alloc(T** p, size_t count) {
 void free_all(ilre_recall* h) {
   cudaFree(h->qp); cudaFree(h->partial); cudaFree(h->nlse2); cudaFree(h->row_lse);
   cudaFree(h->enc); cudaFree(h->scores); cudaFree(h->pooled); cudaFree(h->maxpooled); cudaFree(h->hist);
-  cudaFree(h->sel_prefix); cudaFree(h->sel_krem); cudaFree(h->sel_done); cudaFree(h->grid_barrier); cudaFree(h->rope_table);
+  cudaFree(h->sel_prefix); cudaFree(h->sel_krem); cudaFree(h->sel_done); cudaFree(h->grid_barrier); cudaFree(h->rope_table); cudaFree(h->pos_lo); cudaFree(h->pos_hi);
   cudaFree(h->cand); cudaFree(h->cand_count); cudaFree(h->ranked); cudaFree(h->bitmap);
   cudaFree(h->status); cudaFree(h->stage_k); cudaFree(h->stage_q); cudaFree(h->stage_idx);
   for (int r = 0; r < kProfRing; ++r)
@@ -129,10 +134,10 @@ void free_all(ilre_recall* h) {
 }
 
 bool encode_2d(EncodeTiledFn fn, CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows,
-               uint64_t row_pitch_bytes) {
+               uint64_t row_pitch_bytes, uint32_t box_rows = kTileKeys) {
   const cuuint64_t gdim[2] = {inner, rows};
   const cuuint64_t gstride[1] = {row_pitch_bytes};
-  const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(kTileKeys)};
+  const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(box_rows)};
   const cuuint32_t estride[2] = {1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box,
             estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -234,6 +239,9 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out) {
   ok = ok && dev_alloc(&h->sel_done, ncomb);
   ok = ok && dev_alloc(&h->grid_barrier, 1);
   ok = ok && dev_alloc(&h->rope_table, static_cast<size_t>(kRopeTableRows) * kRopeHalfDim);
+  h->pos_hi_rows = static_cast<int>(cfg->max_L / kRopeLoRows + 2);
+  ok = ok && dev_alloc(&h->pos_lo, static_cast<size_t>(kRopeLoRows) * 64);
+  ok = ok && dev_alloc(&h->pos_hi, static_cast<size_t>(h->pos_hi_rows) * 64);
   ok = ok && dev_alloc(&h->cand, ncomb * h->cand_stride);
   ok = ok && dev_alloc(&h->cand_count, ncomb);
   ok = ok && dev_alloc(&h->ranked, ncomb * h->cand_stride);
@@ -409,6 +417,53 @@ int ilre_recall_run_host(ilre_recall_t* h, const void* k_cache_host, int64_t L,
     ILRE_CUDA(cudaMemcpyAsync(out_scores_host, h->scores, static_cast<size_t>(L) * sizeof(float),
                               cudaMemcpyDeviceToHost, st));
   ILRE_CUDA(cudaStreamSynchronize(st));
+  return ILRE_OK;
+}
+
+int ilre_recall_fill_keys(ilre_recall_t* h, const void* x_dev, int64_t n_tok, int32_t d_model,
+                          const void* w_k_dev, const void* bias_dev, int64_t pos0,
+                          double rope_theta, void* k_cache_dev, int64_t L, void* cuda_stream) {
+  if (!h || !x_dev || !w_k_dev || !k_cache_dev || n_tok < 0 || d_model < 1 || pos0 < 0 || L < 1 ||
+      !(rope_theta > 1.0))
+    return ILRE_ERR_INVALID_ARG;
+  if (d_model % kFillBlockK != 0) return ILRE_ERR_UNSUPPORTED;
+  if (L > h->cfg.max_L || pos0 + n_tok > L || n_tok > 2147483647LL - 256) return ILRE_ERR_CAPACITY;
+  if ((reinterpret_cast<uintptr_t>(x_dev) & 15u) || (reinterpret_cast<uintptr_t>(w_k_dev) & 15u) ||
+      (reinterpret_cast<uintptr_t>(k_cache_dev) & 15u))
+    return ILRE_ERR_ALIGNMENT;
+  if (n_tok == 0) return ILRE_OK;
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return ILRE_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  h->last_stream = st;
+  int launches = 0;
+  if (h->pos_theta != rope_theta) {                    // tables depend on theta only
+    ILRE_CUDA(launch_rope_pos_tables(h->pos_lo, h->pos_hi, h->pos_hi_rows, rope_theta, st));
+    h->pos_theta = rope_theta;
+    ++launches;
+  }
+  const int n_out = h->cfg.n_kv_heads * kHeadDim;
+  const long long m_tiles = (n_tok + kFillTileM - 1) / kFillTileM;
+  // two heads per tile when that still gives every SM a tile, one head per tile otherwise
+  const int tile_n = (n_out % 256 == 0 && m_tiles * (n_out / 256) >= h->n_sm) ? 256 : 128;
+  const long long n_tiles = m_tiles * (n_out / tile_n);
+  CUtensorMap map_x, map_w;
+  if (!encode_2d(h->encode, &map_x, x_dev, static_cast<uint64_t>(d_model),
+                 static_cast<uint64_t>(n_tok), static_cast<uint64_t>(d_model) * 2, kFillTileM))
+    return ILRE_ERR_CUDA;
+  if (!encode_2d(h->encode, &map_w, w_k_dev, static_cast<uint64_t>(d_model),
+                 static_cast<uint64_t>(n_out), static_cast<uint64_t>(d_model) * 2, tile_n))
+    return ILRE_ERR_CUDA;
+  FillParams fp;
+  fp.n_tok = n_tok; fp.d_model = d_model; fp.n_kv = h->cfg.n_kv_heads; fp.pos0 = pos0;
+  fp.bias = static_cast<const uint16_t*>(bias_dev);
+  fp.rope_lo = h->pos_lo; fp.rope_hi = h->pos_hi;
+  fp.k_cache = static_cast<uint16_t*>(k_cache_dev);
+  fp.stages = fill_max_stages(tile_n);
+  fp.status = h->status;
+  const int grid = static_cast<int>(n_tiles < h->n_sm ? n_tiles : h->n_sm);
+  ILRE_CUDA(launch_fill(map_x, map_w, fp, tile_n, grid, st)); ++launches;
+  h->last_launches = launches;
   return ILRE_OK;
 }
 

@@ -18,7 +18,8 @@ LIB_PATH = os.path.join(_HERE, "libilre_recall.so")
 STAGE_NAMES = ("prepare", "row_stats", "merge_stats", "scores", "select")
 
 EXPORTED_SYMBOLS = (
-    "ilre_recall_create", "ilre_recall_run", "ilre_recall_run_host", "ilre_recall_rerope_keys",
+    "ilre_recall_create", "ilre_recall_run", "ilre_recall_run_host", "ilre_recall_fill_keys",
+    "ilre_recall_rerope_keys",
     "ilre_recall_copy_row_lse",
     "ilre_recall_status", "ilre_recall_set_profiling", "ilre_recall_stage_times",
     "ilre_recall_last_launch_count", "ilre_recall_destroy", "ilre_strerror",
@@ -65,6 +66,7 @@ def load_library() -> ctypes.CDLL:
     lib.ilre_recall_create.argtypes = [ctypes.POINTER(IlreConfig), ctypes.POINTER(vp)]
     lib.ilre_recall_run.argtypes = [vp, vp, i64, vp, i32, i32, ctypes.POINTER(IlrePoolSpec), vp, vp, vp]
     lib.ilre_recall_run_host.argtypes = lib.ilre_recall_run.argtypes
+    lib.ilre_recall_fill_keys.argtypes = [vp, vp, i64, i32, vp, vp, i64, ctypes.c_double, vp, i64, vp]
     lib.ilre_recall_rerope_keys.argtypes = [vp, vp, vp, i64, i32, i32, ctypes.c_double, vp]
     lib.ilre_recall_copy_row_lse.argtypes = [vp, vp, i32, vp]
     lib.ilre_recall_status.argtypes = [vp]
@@ -181,6 +183,23 @@ class IlreRecall:
         if rc != 0:
             raise IlreError(rc, "ilre_recall_run_host")
         return out_idx, out_scores
+
+    def fill_keys(self, X: torch.Tensor, W_k: torch.Tensor, K_cache: torch.Tensor, pos0: int,
+                  bias: Optional[torch.Tensor] = None, rope_theta: float = 500000.0,
+                  stream: Optional[torch.cuda.Stream] = None) -> None:
+        """Key projection + RoPE of the tokens X (positions pos0 ..) written into K_cache."""
+        for t in (X, W_k, K_cache) + ((bias,) if bias is not None else ()):
+            assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+        assert X.dim() == 2 and W_k.shape == (self.cfg.n_kv_heads * self.cfg.head_dim, X.shape[1])
+        assert K_cache.shape[1:] == (self.cfg.n_kv_heads, self.cfg.head_dim)
+        assert bias is None or bias.shape == (W_k.shape[0],)
+        st = stream if stream is not None else torch.cuda.current_stream(self.device)
+        rc = self._lib.ilre_recall_fill_keys(
+            self._h, X.data_ptr(), X.shape[0], X.shape[1], W_k.data_ptr(),
+            bias.data_ptr() if bias is not None else None, pos0, float(rope_theta),
+            K_cache.data_ptr(), K_cache.shape[0], st.cuda_stream)
+        if rc != 0:
+            raise IlreError(rc, "ilre_recall_fill_keys")
 
     def rerope_keys(self, K: torch.Tensor, chunk_size: int, n_sink: int = 0,
                     rope_theta: float = 500000.0, out: Optional[torch.Tensor] = None,
