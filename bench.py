@@ -293,6 +293,48 @@ def run_ours(args, world, rank, local):
                    frac=moved / (ms * 1e-3) / 1e9 / measured_peaks()["hbm_gbs"])
         del Kc
 
+    # Key-cache fill (key projection + RoPE into the cache), timed on its own: a tensor-bound
+    # GEMM.  Llama-3.1-8B shape (d_model 4096), activations and weights drawn on the device.
+    fill = None
+    if args.fill_tokens > 0 and rank == 0:
+        gen = torch.Generator(device=dev).manual_seed(1234)
+        d_model = 4096
+        n_fill = min(args.fill_tokens, w.L)
+        Xf = torch.randn(n_fill, d_model, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        Wf = (torch.randn(w.n_kv_heads * w.d, d_model, generator=gen, device=dev) / 64).to(torch.bfloat16)
+        Kf = torch.empty(n_fill, w.n_kv_heads, w.d, dtype=torch.bfloat16, device=dev)
+
+        def timed(fn, reps):
+            for _ in range(3):
+                fn()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record()
+            for _ in range(reps):
+                fn()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / reps
+
+        ms_all = timed(lambda: eng.fill_keys(Xf, Wf, Kf, 0), 5)
+        chunk = min(1024, n_fill)
+        n_chunks = n_fill // chunk
+
+        def by_chunks():
+            for c in range(n_chunks):
+                eng.fill_keys(Xf[c * chunk:(c + 1) * chunk], Wf, Kf, c * chunk)
+
+        ms_chunks = timed(by_chunks, 2) / max(n_chunks, 1)
+        fl_all = 2.0 * n_fill * d_model * w.n_kv_heads * w.d
+        fl_chunk = 2.0 * chunk * d_model * w.n_kv_heads * w.d
+        pk = measured_peaks()["bf16_tflops_sustained"]
+        fill = dict(kernel="fill_kernel", d_model=d_model, tokens=n_fill, bound="tensor",
+                    unit="TFLOP/s", peak=pk, ms=ms_all, achieved=fl_all / (ms_all * 1e-3) / 1e12,
+                    frac=fl_all / (ms_all * 1e-3) / 1e12 / pk,
+                    per_chunk=dict(tokens=chunk, ms=ms_chunks,
+                                   achieved=fl_chunk / (ms_chunks * 1e-3) / 1e12))
+        del Xf, Wf, Kf
+
     elapsed_max, units = aggregate(elapsed_ms, float(k_bytes) * args.steps, dev)
     if rank != 0:
         return
@@ -343,7 +385,7 @@ def run_ours(args, world, rank, local):
                             parallelism="replicas only" if world > 1 else "single GPU"),
                 clocks=clocks, e2e=e2e, gpu_launches=launches, roofline=roofline,
                 cpu_baseline=cpu_baseline,
-                stages_ms=stages, dca_rerope=dca,
+                stages_ms=stages, dca_rerope=dca, key_fill=fill,
                 whole_step=dict(hbm_frac_one_read_of_K=step_hbm_frac,
                                 tensor_frac_one_qk=step_tensor_frac,
                                 hbm_frac_of_8TBps=(k_bytes / (ms_per_step * 1e-3) / 1e9) / 8000.0))
@@ -364,6 +406,8 @@ def main():
                     help="override the context length of --config (profiling on a small case)")
     ap.add_argument("--dca-chunk", type=int, default=1024,
                     help="also time the Eq. 7 key re-rotation with this chunk size (0 = skip)")
+    ap.add_argument("--fill-tokens", type=int, default=1048576,
+                    help="also time the key-cache fill over this many tokens (0 = skip)")
     ap.add_argument("--cpu-sample-keys", type=int, default=131072)
     ap.add_argument("--ref-sample-keys", type=int, default=4096)
     args = ap.parse_args()
