@@ -110,6 +110,30 @@ def test_ragged_shapes_match_oracle(case):
     eng.close()
 
 
+BIG = [
+    # L, q_len, budget, max_sizes, win_sizes, win_op, n_sink -- paths of the selection kernel
+    # that the benchmark shapes do not reach
+    (40000, 4, 9000, (1,), (1, 5), 1, 0),          # K_m > 8192: ranking staged in two chunks
+    (60000, 2, 16382, (1,), (1,), 0, 0),           # largest budget: one staging buffer only
+    (1200000, 1, 4096, (1,), (1, 15), 1, 4),       # bitmap too large for shared memory
+    (1100000, 1, 2000, (2, 64), (1, 3), 0, 3),     # strided max-pool sources at 1M, m = 64
+]
+
+
+@pytest.mark.parametrize("case", BIG, ids=lambda c: f"L{c[0]}_q{c[1]}_B{c[2]}_m{len(c[3])}")
+def test_selection_kernel_edge_paths(case):
+    L, q_len, budget, max_sizes, win_sizes, win_op, n_sink = case
+    w = small_workload(L, q_len, seed=L % 1000 + budget, n_spans=4, span_len=(16, 64),
+                       budget=budget, max_sizes=max_sizes, win_sizes=win_sizes, win_op=win_op,
+                       n_sink=n_sink)
+    x = make_inputs(w)
+    eng = _engine(w)
+    idx, sc = _run(eng, x)
+    rep = parity.check_recall(x.K, x.Q, w, idx, sc)
+    print(case, rep)
+    eng.close()
+
+
 def test_handle_reuse_and_determinism(cases):
     # one handle, different shapes back to back, and bit-identical repeats
     big = make_inputs(CONFIGS["cfg2_L32k"])
