@@ -148,6 +148,16 @@ int ilre_recall_rerope_keys(ilre_recall_t* h, const void* k_cache_dev, void* k_o
                             void* cuda_stream);
 
 /*
+ * The compressed prompt (Algorithm 1's last line, C~ = C[I], and Section 3.3's last step):
+ *   out[i] = input_ids[idx[i]] for i < n_idx, then the n_query ids of the query part.
+ * All pointers are int32 arrays on the current device; idx is what ilre_recall_run returned.
+ * A position outside [0, L) yields -1.  No handle; asynchronous on cuda_stream.
+ */
+int ilre_gather_input_ids(const int32_t* input_ids_dev, int64_t L, const int32_t* idx_dev,
+                          int32_t n_idx, const int32_t* query_ids_dev, int32_t n_query,
+                          int32_t* out_ids_dev, void* cuda_stream);
+
+/*
  * Row statistics of the last run (Eq. 4's softmax denominator): copies
  * lse[i * n_q_heads + h] = log(sum_t exp(s[h,i,t])) (natural log, fp32) for the q_len rows
  * of that run into out_lse_dev, asynchronously on cuda_stream.

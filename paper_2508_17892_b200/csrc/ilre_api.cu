@@ -502,6 +502,17 @@ int ilre_recall_rerope_keys(ilre_recall_t* h, const void* k_cache_dev, void* k_o
   return ILRE_OK;
 }
 
+int ilre_gather_input_ids(const int32_t* input_ids_dev, int64_t L, const int32_t* idx_dev,
+                          int32_t n_idx, const int32_t* query_ids_dev, int32_t n_query,
+                          int32_t* out_ids_dev, void* cuda_stream) {
+  if (L < 1 || n_idx < 0 || n_query < 0 || !out_ids_dev || (n_idx > 0 && (!input_ids_dev || !idx_dev)) ||
+      (n_query > 0 && !query_ids_dev))
+    return ILRE_ERR_INVALID_ARG;
+  ILRE_CUDA(launch_gather_ids(input_ids_dev, L, idx_dev, n_idx, query_ids_dev, n_query, out_ids_dev,
+                              static_cast<cudaStream_t>(cuda_stream)));
+  return ILRE_OK;
+}
+
 int ilre_recall_copy_row_lse(ilre_recall_t* h, float* out_lse_dev, int32_t q_len,
                              void* cuda_stream) {
   if (!h || !out_lse_dev || q_len < 1 || q_len > h->cfg.max_q_len) return ILRE_ERR_INVALID_ARG;

@@ -86,6 +86,30 @@ rerope_kernel(const ReropeParams p) {
   }
 }
 
+// Algorithm 1's last step and the hand-over to the inference engine: the compressed prompt is
+// the input ids at the chosen positions followed by the ids of the query part.
+__global__ void gather_ids_kernel(const int32_t* __restrict__ ids, long long L,
+                                  const int32_t* __restrict__ idx, int n_idx,
+                                  const int32_t* __restrict__ query_ids, int n_query,
+                                  int32_t* __restrict__ out) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n_idx) {
+    const int pos = idx[i];
+    out[i] = (pos >= 0 && pos < L) ? ids[pos] : -1;      // -1 marks a position outside the context
+  } else if (i < n_idx + n_query) {
+    out[i] = query_ids[i - n_idx];
+  }
+}
+
+cudaError_t launch_gather_ids(const int32_t* ids, long long L, const int32_t* idx, int n_idx,
+                              const int32_t* query_ids, int n_query, int32_t* out,
+                              cudaStream_t st) {
+  const int n = n_idx + n_query;
+  if (n < 1) return cudaSuccess;
+  gather_ids_kernel<<<(n + 255) / 256, 256, 0, st>>>(ids, L, idx, n_idx, query_ids, n_query, out);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_rope_table(float2* table, int n_rows, int chunk, double theta,
                               cudaStream_t st) {
   if (n_rows < 1) return cudaSuccess;

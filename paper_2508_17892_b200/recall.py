@@ -19,7 +19,7 @@ STAGE_NAMES = ("prepare", "row_stats", "merge_stats", "scores", "select")
 
 EXPORTED_SYMBOLS = (
     "ilre_recall_create", "ilre_recall_run", "ilre_recall_run_host", "ilre_recall_fill_keys",
-    "ilre_recall_rerope_keys",
+    "ilre_recall_rerope_keys", "ilre_gather_input_ids",
     "ilre_recall_copy_row_lse",
     "ilre_recall_status", "ilre_recall_set_profiling", "ilre_recall_stage_times",
     "ilre_recall_last_launch_count", "ilre_recall_destroy", "ilre_strerror",
@@ -68,6 +68,7 @@ def load_library() -> ctypes.CDLL:
     lib.ilre_recall_run_host.argtypes = lib.ilre_recall_run.argtypes
     lib.ilre_recall_fill_keys.argtypes = [vp, vp, i64, i32, vp, vp, i64, ctypes.c_double, vp, i64, vp]
     lib.ilre_recall_rerope_keys.argtypes = [vp, vp, vp, i64, i32, i32, ctypes.c_double, vp]
+    lib.ilre_gather_input_ids.argtypes = [vp, i64, vp, i32, vp, i32, vp, vp]
     lib.ilre_recall_copy_row_lse.argtypes = [vp, vp, i32, vp]
     lib.ilre_recall_status.argtypes = [vp]
     lib.ilre_recall_set_profiling.argtypes = [vp, i32]
@@ -93,6 +94,22 @@ def _spec(max_sizes: Sequence[int], win_sizes: Sequence[int], win_op: int, n_sin
     ws = (ctypes.c_int32 * len(win_sizes))(*win_sizes)
     spec = IlrePoolSpec(len(max_sizes), ms, len(win_sizes), ws, win_op, 0, n_sink)
     return spec, (ms, ws)
+
+
+def gather_input_ids(input_ids: torch.Tensor, idx: torch.Tensor, query_ids: torch.Tensor,
+                     stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Compressed prompt: input_ids at the recalled positions, then the query's ids (int32)."""
+    for t in (input_ids, idx, query_ids):
+        assert t.is_cuda and t.dtype == torch.int32 and t.is_contiguous() and t.dim() == 1
+    out = torch.empty(idx.numel() + query_ids.numel(), dtype=torch.int32, device=input_ids.device)
+    st = stream if stream is not None else torch.cuda.current_stream(input_ids.device)
+    with torch.cuda.device(input_ids.device):
+        rc = load_library().ilre_gather_input_ids(input_ids.data_ptr(), input_ids.numel(),
+                                                  idx.data_ptr(), idx.numel(), query_ids.data_ptr(),
+                                                  query_ids.numel(), out.data_ptr(), st.cuda_stream)
+    if rc != 0:
+        raise IlreError(rc, "ilre_gather_input_ids")
+    return out
 
 
 def topk_positions_noalloc(scores: torch.Tensor, k: int,

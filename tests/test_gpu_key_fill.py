@@ -112,3 +112,17 @@ def test_fill_argument_errors():
     assert e.value.code == -3
     assert eng.status() == 0
     eng.close()
+
+
+def test_gather_input_ids_is_plain_indexing():
+    from paper_2508_17892_b200 import gather_input_ids
+    g = torch.Generator().manual_seed(0)
+    ids = torch.randint(0, 128000, (5000,), generator=g, dtype=torch.int32)
+    idx = torch.sort(torch.randperm(5000, generator=g)[:700]).values.to(torch.int32)
+    query = torch.randint(0, 128000, (37,), generator=g, dtype=torch.int32)
+    out = gather_input_ids(ids.cuda(), idx.cuda(), query.cuda())
+    want = np.concatenate([ids.numpy()[idx.numpy()], query.numpy()])     # C~ = C[I], then the query
+    np.testing.assert_array_equal(out.cpu().numpy(), want)
+    bad = torch.tensor([0, 4999, 5000, -1], dtype=torch.int32)
+    out = gather_input_ids(ids.cuda(), bad.cuda(), query[:0].cuda())
+    np.testing.assert_array_equal(out.cpu().numpy(), [ids[0].item(), ids[4999].item(), -1, -1])
