@@ -218,3 +218,32 @@ def key_fill(X, W, pos0: int, theta: float = 500000.0, bias=None) -> np.ndarray:
     out[..., :half] = y[..., :half] * cs - y[..., half:] * sn
     out[..., half:] = y[..., :half] * sn + y[..., half:] * cs
     return out
+
+
+def chunk_attention(Q, K, V, n_prefix: int) -> np.ndarray:
+    """Streaming chunked prefill attention of one chunk (Eq. 2 with the Lambda-shaped mask), fp64.
+
+    Q: bf16 [c, n_q, d] queries of the chunk's tokens; K, V: bf16 [n_prefix + c, n_kv, d], the
+    cached sink and sliding-window keys/values (the first n_prefix rows, visible to every query)
+    followed by the chunk's own, which are visible causally: query j sees rows
+    0 .. n_prefix + j.  Query head h reads kv head h // (n_q // n_kv).  Returns the attention
+    output fp64 [c, n_q, d].  Written as plain loops over heads with a library softmax-free
+    definition: exp, sum, divide."""
+    import torch
+    q = Q.to(torch.float64).numpy()
+    k = K.to(torch.float64).numpy()
+    v = V.to(torch.float64).numpy()
+    c, n_q, d = q.shape
+    n_kv = k.shape[1]
+    group = n_q // n_kv
+    assert k.shape[0] == n_prefix + c and v.shape == k.shape
+    out = np.empty((c, n_q, d), dtype=np.float64)
+    for h in range(n_q):
+        g = h // group
+        s = (q[:, h, :] @ k[:, g, :].T) / np.sqrt(d)                     # [c, n_prefix + c]
+        for j in range(c):
+            row = s[j, : n_prefix + j + 1]
+            p = np.exp(row - row.max())
+            p /= p.sum()
+            out[j, h, :] = p @ v[: n_prefix + j + 1, g, :]
+    return out
