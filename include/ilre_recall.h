@@ -107,6 +107,27 @@ int ilre_recall_run_host(ilre_recall_t* h,
                          void* cuda_stream);
 
 /*
+ * Streaming chunked prefill attention of one chunk in a layer before the retrieval layer
+ * (Section 3.1, Eq. 2 with the Lambda-shaped mask; Section 3.3: "only cache the sink and sliding
+ * part of the key states and value states"):
+ *   out[j, h, :] = sum_k softmax_k(q[j, h, :] . k[k, kv(h), :] / sqrt(128)) v[k, kv(h), :],
+ *   k = 0 .. n_prefix + j,
+ * where the first n_prefix rows of k/v are the cached sink and sliding-window tokens, visible to
+ * every query, and the following chunk_len rows the chunk's own, visible causally.  The caller
+ * keeps the cache (sink S, window W) and lays the rows out in that order.
+ *   q_dev    bf16 [chunk_len][n_q_heads][128]             (RoPE applied)
+ *   k_dev    bf16 [n_prefix + chunk_len][n_kv_heads][128] (RoPE applied)
+ *   v_dev    bf16 [n_prefix + chunk_len][n_kv_heads][128]
+ *   out_dev  bf16 [chunk_len][n_q_heads][128]
+ * All 16-byte aligned.  Products on the tensor cores with fp32 accumulation; the probabilities
+ * are rounded to bf16 before they multiply the values (as the output is).  Asynchronous on
+ * cuda_stream; bounded waits report through ilre_recall_status.
+ */
+int ilre_recall_chunk_attention(ilre_recall_t* h, const void* q_dev, const void* k_dev,
+                                const void* v_dev, int32_t chunk_len, int32_t n_prefix,
+                                void* out_dev, void* cuda_stream);
+
+/*
  * Key-cache fill of the retrieval layer (Section 3.3: "calculate the key states for the context
  * ... fill the cache with chunked key states"; Eq. 1 with the positional encoding of Eq. 3):
  *   K[pos0 + t, g, :] = R(pos0 + t) (x[t, :] . W_K[g*128 : (g+1)*128, :]^T + b[g*128 : (g+1)*128])

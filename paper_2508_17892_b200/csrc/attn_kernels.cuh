@@ -1,0 +1,27 @@
+// Streaming chunked prefill attention of one chunk (Eq. 2 with the Lambda-shaped mask): the
+// layers before the retrieval layer attend to the cached sink + sliding-window keys/values and,
+// causally, to the chunk's own.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ilre {
+
+static constexpr int kAttnThreads = 192;     // warp 0 TMA, warp 1 MMA, warps 2..5 softmax
+
+struct AttnParams {
+  int c;             // query tokens of the chunk
+  int n_prefix;      // rows of K/V visible to every query (sink + sliding window)
+  int n_q, n_kv;     // query heads, kv heads
+  float c2;          // log2(e) / sqrt(d)
+  uint16_t* out;     // bf16 [c][n_q][128]
+  int* status;
+};
+
+size_t attn_smem_bytes();
+// grid = (ceil(c / 128), n_q)
+cudaError_t launch_chunk_attention(const CUtensorMap& map_q, const CUtensorMap& map_k,
+                                   const CUtensorMap& map_v, const AttnParams& p, cudaStream_t st);
+
+}  // namespace ilre

@@ -9,6 +9,7 @@
 #include <new>
 
 #include "../../include/ilre_recall.h"
+#include "attn_kernels.cuh"
 #include "fill_kernels.cuh"
 #include "qk_kernels.cuh"
 #include "rerope_kernels.cuh"
@@ -417,6 +418,36 @@ int ilre_recall_run_host(ilre_recall_t* h, const void* k_cache_host, int64_t L,
     ILRE_CUDA(cudaMemcpyAsync(out_scores_host, h->scores, static_cast<size_t>(L) * sizeof(float),
                               cudaMemcpyDeviceToHost, st));
   ILRE_CUDA(cudaStreamSynchronize(st));
+  return ILRE_OK;
+}
+
+int ilre_recall_chunk_attention(ilre_recall_t* h, const void* q_dev, const void* k_dev,
+                                const void* v_dev, int32_t chunk_len, int32_t n_prefix,
+                                void* out_dev, void* cuda_stream) {
+  if (!h || !q_dev || !k_dev || !v_dev || !out_dev || chunk_len < 1 || n_prefix < 0)
+    return ILRE_ERR_INVALID_ARG;
+  if (static_cast<long long>(chunk_len) + n_prefix > 2147483647LL - 256) return ILRE_ERR_CAPACITY;
+  if ((reinterpret_cast<uintptr_t>(q_dev) & 15u) || (reinterpret_cast<uintptr_t>(k_dev) & 15u) ||
+      (reinterpret_cast<uintptr_t>(v_dev) & 15u) || (reinterpret_cast<uintptr_t>(out_dev) & 15u))
+    return ILRE_ERR_ALIGNMENT;
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return ILRE_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  h->last_stream = st;
+  const uint64_t n_rows = static_cast<uint64_t>(n_prefix) + chunk_len;
+  const uint64_t q_inner = static_cast<uint64_t>(h->cfg.n_q_heads) * kHeadDim;
+  const uint64_t kv_inner = static_cast<uint64_t>(h->cfg.n_kv_heads) * kHeadDim;
+  CUtensorMap map_q, map_k, map_v;
+  if (!encode_2d(h->encode, &map_q, q_dev, q_inner, chunk_len, q_inner * 2, 128) ||
+      !encode_2d(h->encode, &map_k, k_dev, kv_inner, n_rows, kv_inner * 2, 128) ||
+      !encode_2d(h->encode, &map_v, v_dev, kv_inner, n_rows, kv_inner * 2, 128))
+    return ILRE_ERR_CUDA;
+  AttnParams ap;
+  ap.c = chunk_len; ap.n_prefix = n_prefix; ap.n_q = h->cfg.n_q_heads; ap.n_kv = h->cfg.n_kv_heads;
+  ap.c2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(kHeadDim)));
+  ap.out = static_cast<uint16_t*>(out_dev); ap.status = h->status;
+  ILRE_CUDA(launch_chunk_attention(map_q, map_k, map_v, ap, st));
+  h->last_launches = 1;
   return ILRE_OK;
 }
 

@@ -19,7 +19,7 @@ STAGE_NAMES = ("prepare", "row_stats", "merge_stats", "scores", "select")
 
 EXPORTED_SYMBOLS = (
     "ilre_recall_create", "ilre_recall_run", "ilre_recall_run_host", "ilre_recall_fill_keys",
-    "ilre_recall_rerope_keys", "ilre_gather_input_ids",
+    "ilre_recall_chunk_attention", "ilre_recall_rerope_keys", "ilre_gather_input_ids",
     "ilre_recall_copy_row_lse",
     "ilre_recall_status", "ilre_recall_set_profiling", "ilre_recall_stage_times",
     "ilre_recall_last_launch_count", "ilre_recall_destroy", "ilre_strerror",
@@ -66,6 +66,7 @@ def load_library() -> ctypes.CDLL:
     lib.ilre_recall_create.argtypes = [ctypes.POINTER(IlreConfig), ctypes.POINTER(vp)]
     lib.ilre_recall_run.argtypes = [vp, vp, i64, vp, i32, i32, ctypes.POINTER(IlrePoolSpec), vp, vp, vp]
     lib.ilre_recall_run_host.argtypes = lib.ilre_recall_run.argtypes
+    lib.ilre_recall_chunk_attention.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp]
     lib.ilre_recall_fill_keys.argtypes = [vp, vp, i64, i32, vp, vp, i64, ctypes.c_double, vp, i64, vp]
     lib.ilre_recall_rerope_keys.argtypes = [vp, vp, vp, i64, i32, i32, ctypes.c_double, vp]
     lib.ilre_gather_input_ids.argtypes = [vp, i64, vp, i32, vp, i32, vp, vp]
@@ -200,6 +201,22 @@ class IlreRecall:
         if rc != 0:
             raise IlreError(rc, "ilre_recall_run_host")
         return out_idx, out_scores
+
+    def chunk_attention(self, Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, n_prefix: int,
+                        stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        """Attention of one prefill chunk over n_prefix cached rows plus, causally, its own."""
+        for t in (Q, K, V):
+            assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous() and t.dim() == 3
+        c = Q.shape[0]
+        assert Q.shape[1:] == (self.cfg.n_q_heads, self.cfg.head_dim)
+        assert K.shape == (n_prefix + c, self.cfg.n_kv_heads, self.cfg.head_dim) and V.shape == K.shape
+        out = torch.empty_like(Q)
+        st = stream if stream is not None else torch.cuda.current_stream(self.device)
+        rc = self._lib.ilre_recall_chunk_attention(self._h, Q.data_ptr(), K.data_ptr(), V.data_ptr(),
+                                                   c, n_prefix, out.data_ptr(), st.cuda_stream)
+        if rc != 0:
+            raise IlreError(rc, "ilre_recall_chunk_attention")
+        return out
 
     def fill_keys(self, X: torch.Tensor, W_k: torch.Tensor, K_cache: torch.Tensor, pos0: int,
                   bias: Optional[torch.Tensor] = None, rope_theta: float = 500000.0,
