@@ -335,6 +335,34 @@ def run_ours(args, world, rank, local):
                                    achieved=fl_chunk / (ms_chunks * 1e-3) / 1e12))
         del Xf, Wf, Kf
 
+    # Streaming chunked prefill attention of one chunk (paper defaults: chunk 1024, sink 4 +
+    # window 512), timed on its own
+    attn = None
+    if args.attn_chunk > 0 and rank == 0:
+        gen = torch.Generator(device=dev).manual_seed(4321)
+        c_len, n_pre = args.attn_chunk, 516
+        Qa = torch.randn(c_len, w.n_q_heads, w.d, generator=gen, device=dev).to(torch.bfloat16)
+        Ka = torch.randn(n_pre + c_len, w.n_kv_heads, w.d, generator=gen, device=dev).to(torch.bfloat16)
+        Va = torch.randn(n_pre + c_len, w.n_kv_heads, w.d, generator=gen, device=dev).to(torch.bfloat16)
+        for _ in range(3):
+            eng.chunk_attention(Qa, Ka, Va, n_pre)
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 50
+        torch.cuda.synchronize()
+        a0.record()
+        for _ in range(reps):
+            eng.chunk_attention(Qa, Ka, Va, n_pre)
+        a1.record()
+        torch.cuda.synchronize()
+        ms = a0.elapsed_time(a1) / reps
+        pairs = c_len * n_pre + c_len * (c_len + 1) / 2.0               # visible (query, key) pairs
+        fl = pairs * w.n_q_heads * 4.0 * w.d                             # QK^T and PV
+        pk = measured_peaks()["bf16_tflops"]
+        attn = dict(kernel="chunk_attention_kernel", chunk=c_len, n_prefix=n_pre, ms=ms,
+                    algorithmic_flops=fl, achieved=fl / (ms * 1e-3) / 1e12, unit="TFLOP/s",
+                    bound="tensor", peak=pk, frac=fl / (ms * 1e-3) / 1e12 / pk)
+        del Qa, Ka, Va
+
     elapsed_max, units = aggregate(elapsed_ms, float(k_bytes) * args.steps, dev)
     if rank != 0:
         return
@@ -385,7 +413,7 @@ def run_ours(args, world, rank, local):
                             parallelism="replicas only" if world > 1 else "single GPU"),
                 clocks=clocks, e2e=e2e, gpu_launches=launches, roofline=roofline,
                 cpu_baseline=cpu_baseline,
-                stages_ms=stages, dca_rerope=dca, key_fill=fill,
+                stages_ms=stages, dca_rerope=dca, key_fill=fill, chunk_attention=attn,
                 whole_step=dict(hbm_frac_one_read_of_K=step_hbm_frac,
                                 tensor_frac_one_qk=step_tensor_frac,
                                 hbm_frac_of_8TBps=(k_bytes / (ms_per_step * 1e-3) / 1e9) / 8000.0))
@@ -406,6 +434,8 @@ def main():
                     help="override the context length of --config (profiling on a small case)")
     ap.add_argument("--dca-chunk", type=int, default=1024,
                     help="also time the Eq. 7 key re-rotation with this chunk size (0 = skip)")
+    ap.add_argument("--attn-chunk", type=int, default=1024,
+                    help="also time the chunked prefill attention of one chunk (0 = skip)")
     ap.add_argument("--fill-tokens", type=int, default=1048576,
                     help="also time the key-cache fill over this many tokens (0 = skip)")
     ap.add_argument("--cpu-sample-keys", type=int, default=131072)

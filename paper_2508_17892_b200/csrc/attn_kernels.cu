@@ -5,9 +5,11 @@
 //
 // One CTA per (128 query tokens, query head).  Both contractions run on the tensor cores:
 // S = Q K^T into tensor memory, and O += P V with P written to shared memory as bf16 by the
-// softmax warps.  Two sweeps over the (at most a dozen) key tiles: the first takes the row
-// statistics, the second forms normalised probabilities, so that O accumulates in tensor memory
-// without rescaling.  Key/value tiles come through one TMA ring.
+// softmax warps.  One sweep over the key tiles with an online softmax: probabilities are taken
+// against a per-row reference maximum, O accumulates in tensor memory and is rescaled there
+// only when a row's maximum has run ahead of its reference by more than 2^8 (rare after the
+// first tiles); the row sums divide the output at the end.  Key and value tiles come through
+// one TMA ring.  Heavier CTAs (later query tiles see more keys) are launched first.
 #include <cuda_bf16.h>
 
 #include "attn_kernels.cuh"
@@ -18,7 +20,8 @@ namespace ilre {
 static constexpr int kAttnStages = 4;
 static constexpr int kAttnTileBytes = 128 * 128 * 2;       // one 128 x 128 bf16 tile
 static constexpr int kAttnTailBytes = 256;
-static constexpr int kAttnSoftmaxWarps = 4;
+static constexpr int kAttnSoftmaxWarps = 8;          // two per TMEM lane quadrant: 64 columns each
+static constexpr int kAttnXchgBytes = 3 * 1024;      // tile maxima [2][2][128] + row sums [128]
 
 struct AttnTail {
   uint64_t q_full;
@@ -54,10 +57,12 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
   const uint32_t p_s = ring_s + kAttnStages * kAttnTileBytes;
   uint8_t* p_ptr = smem + (1 + kAttnStages) * kAttnTileBytes;
   AttnTail* tail = reinterpret_cast<AttnTail*>(smem + (2 + kAttnStages) * kAttnTileBytes);
+  float* xchg_max = reinterpret_cast<float*>(smem + (2 + kAttnStages) * kAttnTileBytes + kAttnTailBytes);
+  float* xchg_sum = xchg_max + 512;
   volatile int* abort_flag = &tail->abort_flag;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  const int j0 = blockIdx.x * 128;                      // first query token of this CTA
+  const int j0 = (gridDim.x - 1 - blockIdx.x) * 128;    // first query token; heavy tiles first
   const int h = blockIdx.y, g = h / (p.n_q / p.n_kv);
   const int last_q = min(j0 + 128, p.c) - 1;
   const int n_tiles = (p.n_prefix + last_q) / 128 + 1;   // key tiles that hold a visible key
@@ -93,23 +98,22 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
   const uint32_t tmem_o = tmem_base + 256;
   const bool run = (*abort_flag == 0);
 
-  // Ring items: sweep 1 = K_0 .. K_{T-1}; sweep 2 = K_0, V_0, K_1, V_1, ...
+  // Ring items: K_0, V_0, K_1, V_1, ...
   if (warp == 0) {
     if (lane == 0 && run) {
       const uint32_t qf = smem_u32(&tail->q_full);
       mbar_arrive_expect_tx(qf, kAttnTileBytes);
       tma_load_2d(q_s, &map_q, h * 128, j0, qf);
       tma_load_2d(q_s + 16384, &map_q, h * 128 + 64, j0, qf);
-      const int n_items = 3 * n_tiles;
+      const int n_items = 2 * n_tiles;
       for (int it = 0; it < n_items; ++it) {
         const int s = it % kAttnStages;
         const uint32_t use = static_cast<uint32_t>(it / kAttnStages);
         if (!mbar_wait(smem_u32(&tail->kv_empty[s]), (use & 1u) ^ 1u, abort_flag, p.status,
                        kDevWaitKEmpty))
           break;
-        const bool is_v = it >= n_tiles && ((it - n_tiles) & 1);
-        const int t = it < n_tiles ? it : (it - n_tiles) >> 1;
-        const CUtensorMap* map = is_v ? &map_v : &map_k;
+        const CUtensorMap* map = (it & 1) ? &map_v : &map_k;
+        const int t = it >> 1;
         const uint32_t bar = smem_u32(&tail->kv_full[s]);
         mbar_arrive_expect_tx(bar, kAttnTileBytes);
         tma_load_2d(ring_s + s * kAttnTileBytes, map, g * 128, t * 128, bar);
@@ -145,12 +149,11 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
         ++u;
         return true;
       };
-      for (int t = 0; t < n_tiles && ok; ++t) ok = issue_s(t);                 // sweep 1
-      if (ok) ok = issue_s(n_tiles);                                           // S of tile 0, sweep 2
+      if (ok) ok = issue_s(0);                                                 // S of tile 0
       for (int t = 0; t < n_tiles && ok; ++t) {
-        if (t + 1 < n_tiles) ok = issue_s(n_tiles + 2 * (t + 1));
+        if (t + 1 < n_tiles) ok = issue_s(2 * (t + 1));                        // S of the next tile
         if (!ok) break;
-        const int item = n_tiles + 2 * t + 1;                                  // V_t
+        const int item = 2 * t + 1;                                            // V_t
         const int s = item % kAttnStages;
         ok = mbar_wait(smem_u32(&tail->p_full), static_cast<uint32_t>(t) & 1u, abort_flag, p.status,
                        kDevWaitAccFull) &&
@@ -172,106 +175,130 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
       if (ok) umma_commit(smem_u32(&tail->o_full));
     }
   } else {
-    const int quad = warp & 3;
+    // Eight softmax warps: warp w reads TMEM lane quadrant w % 4; the two warps of a quadrant
+    // split the 128 columns (keys of S, channels of O) in halves.  A thread therefore owns
+    // half a query row; the two halves meet through shared memory once per tile (maximum).
+    // Every warp runs all iterations, also after a wait was abandoned, so that the named
+    // barrier below always gets its 256 threads.
+    const int quad = warp & 3, half = (warp - 2) >> 2;
     const int row = quad * 32 + lane;
     const int qj = j0 + row;
     const int limit = p.n_prefix + qj;                   // last visible key row of this query
-    const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+    const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + half * 64;
     const float c2 = p.c2;
     bool ok = run;
     uint32_t u = 0;
-    // ---- sweep 1: row maximum and sum of exponentials ----
-    float m = -1e30f, z = 0.f;
-    for (int t = 0; t < n_tiles && ok; ++t, ++u) {
+    // Online softmax: `ref` is the row's reference maximum (raw logits), `l` this thread's
+    // share of the sum of 2^((s - ref) c2) over the keys seen so far.
+    constexpr float kRefSlack = 8.f;                     // log2 units
+    float ref = -INFINITY, l = 0.f;
+    for (int t = 0; t < n_tiles; ++t, ++u) {
       const uint32_t b = u & 1u, use = u >> 1;
-      ok = mbar_wait(smem_u32(&tail->s_full[b]), use & 1u, abort_flag, p.status, kDevWaitAccFull);
-      if (!ok) break;
-      tc_fence_after();
+      if (ok)
+        ok = mbar_wait(smem_u32(&tail->s_full[b]), use & 1u, abort_flag, p.status, kDevWaitAccFull);
+      // tile maximum of the visible logits
+      float cm = -INFINITY;
+      if (ok) {
+        tc_fence_after();
 #pragma unroll 1
-      for (int q4 = 0; q4 < 4; ++q4) {
-        float v[32];
-        tmem_ld32(lane_base + b * 128 + q4 * 32, v);
-        tmem_ld_wait();
-        const int k0 = t * 128 + q4 * 32;
-        float cm = -INFINITY;
+        for (int q2 = 0; q2 < 2; ++q2) {
+          float v[32];
+          tmem_ld32(lane_base + b * 128 + q2 * 32, v);
+          tmem_ld_wait();
+          const int k0 = t * 128 + half * 64 + q2 * 32;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          if (k0 + i > limit) v[i] = -INFINITY;
-          cm = fmaxf(cm, v[i]);
+          for (int i = 0; i < 32; ++i)
+            if (k0 + i <= limit) cm = fmaxf(cm, v[i]);
         }
-        const float m_new = fmaxf(m, cm);
-        const float nm = -m_new * c2;
-        float sum = 0.f;
-#pragma unroll
-        for (int i = 0; i < 32; ++i) sum += ex2_approx(fmaf(v[i], c2, nm));
-        z = fmaf(z, ex2_approx((m - m_new) * c2), sum);
-        m = m_new;
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&tail->s_empty[b]));
-    }
-    const float nl = -(m * c2 + log2f(z));               // -lse in log2 units
-    // ---- sweep 2: normalised probabilities as the bf16 A operand of O += P V ----
-    for (int t = 0; t < n_tiles && ok; ++t, ++u) {
-      const uint32_t b = u & 1u, use = u >> 1;
-      ok = mbar_wait(smem_u32(&tail->s_full[b]), use & 1u, abort_flag, p.status, kDevWaitAccFull);
-      if (!ok) break;
-      tc_fence_after();
-      uint32_t packed[64];
+      xchg_max[((t & 1) * 2 + half) * 128 + row] = cm;
+      asm volatile("bar.sync 1, %0;" ::"r"(kAttnSoftmaxWarps * 32) : "memory");
+      cm = fmaxf(cm, xchg_max[((t & 1) * 2 + (half ^ 1)) * 128 + row]);
+      if (!ok) continue;
+      // move the reference only when the maximum has run ahead of it
+      float scale = 1.f;
+      if ((cm - ref) * c2 > kRefSlack || ref == -INFINITY) {
+        scale = (ref == -INFINITY) ? 0.f : ex2_approx((ref - cm) * c2);
+        ref = (cm == -INFINITY) ? ref : cm;
+      }
+      const float nr = (ref == -INFINITY) ? 0.f : -ref * c2;
+      uint32_t packed[32];
+      float sum = 0.f;
 #pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) {
+      for (int q2 = 0; q2 < 2; ++q2) {
         float v[32];
-        tmem_ld32(lane_base + b * 128 + q4 * 32, v);
+        tmem_ld32(lane_base + b * 128 + q2 * 32, v);
         tmem_ld_wait();
-        const int k0 = t * 128 + q4 * 32;
+        const int k0 = t * 128 + half * 64 + q2 * 32;
 #pragma unroll
         for (int i = 0; i < 32; i += 2) {
-          const float p0 = (k0 + i <= limit) ? ex2_approx(fmaf(v[i], c2, nl)) : 0.f;
-          const float p1 = (k0 + i + 1 <= limit) ? ex2_approx(fmaf(v[i + 1], c2, nl)) : 0.f;
+          const float p0 = (k0 + i <= limit) ? ex2_approx(fmaf(v[i], c2, nr)) : 0.f;
+          const float p1 = (k0 + i + 1 <= limit) ? ex2_approx(fmaf(v[i + 1], c2, nr)) : 0.f;
+          sum += p0 + p1;
           const __nv_bfloat162 pr = __floats2bfloat162_rn(p0, p1);
-          packed[q4 * 16 + (i >> 1)] = *reinterpret_cast<const uint32_t*>(&pr);
+          packed[q2 * 16 + (i >> 1)] = *reinterpret_cast<const uint32_t*>(&pr);
         }
       }
+      l = fmaf(l, scale, sum);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&tail->s_empty[b]));
-      // the previous tile's P must have been consumed by its MMAs
+      // the previous tile's P must have been consumed (and O updated) by its MMAs
       ok = mbar_wait(smem_u32(&tail->p_empty), (static_cast<uint32_t>(t) & 1u) ^ 1u, abort_flag,
                      p.status, kDevWaitAccEmpty);
-      if (!ok) break;
-      // P[row][key]: two halves of 64 keys, rows of 128 bytes, 16-byte groups XOR-swizzled by
-      // the row index (the layout TMA's 128-byte swizzle produces for the other operands)
+      if (!ok) continue;
+      if (t > 0 && __any_sync(0xFFFFFFFFu, scale != 1.f)) {
+        // rescale this warp's share of O (32 rows x 64 channels) to the new references
+        tc_fence_after();
+#pragma unroll 1
+        for (int q2 = 0; q2 < 2; ++q2) {
+          float o[32];
+          tmem_ld32(lane_base + 256 + q2 * 32, o);
+          tmem_ld_wait();
 #pragma unroll
-      for (int grp = 0; grp < 16; ++grp) {
-        const int half = grp >> 3, c16 = grp & 7;
+          for (int i = 0; i < 32; ++i) o[i] *= scale;
+          tmem_st32(lane_base + 256 + q2 * 32, o);
+        }
+        tmem_st_wait();
+        tc_fence_before();
+      }
+      // P[row][key]: two halves of 64 keys (one per warp of the quadrant), rows of 128 bytes,
+      // 16-byte groups XOR-swizzled by the row index (the layout TMA's 128-byte swizzle
+      // produces for the other operands)
+#pragma unroll
+      for (int c16 = 0; c16 < 8; ++c16) {
         uint4* dst = reinterpret_cast<uint4*>(p_ptr + half * 16384 + row * 128 +
                                               ((c16 ^ (row & 7)) << 4));
-        *dst = make_uint4(packed[grp * 4], packed[grp * 4 + 1], packed[grp * 4 + 2],
-                          packed[grp * 4 + 3]);
+        *dst = make_uint4(packed[c16 * 4], packed[c16 * 4 + 1], packed[c16 * 4 + 2],
+                          packed[c16 * 4 + 3]);
       }
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&tail->p_full));
     }
-    // ---- output ----
+    // ---- output: O / (sum of both halves), this thread's 64 channels ----
+    if (half == 1) xchg_sum[row] = l;
+    asm volatile("bar.sync 1, %0;" ::"r"(kAttnSoftmaxWarps * 32) : "memory");
+    if (half == 0) xchg_sum[row] += l;
+    asm volatile("bar.sync 1, %0;" ::"r"(kAttnSoftmaxWarps * 32) : "memory");
     if (ok) ok = mbar_wait(smem_u32(&tail->o_full), 0, abort_flag, p.status, kDevWaitAccFull);
     if (ok) {
       tc_fence_after();
-      uint16_t* dst = p.out + (static_cast<size_t>(qj) * p.n_q + h) * 128;
+      uint16_t* dst = p.out + (static_cast<size_t>(qj) * p.n_q + h) * 128 + half * 64;
+      const float inv_l = 1.f / xchg_sum[row];
 #pragma unroll 1
-      for (int q4 = 0; q4 < 4; ++q4) {
+      for (int q2 = 0; q2 < 2; ++q2) {
         float v[32];
-        tmem_ld32(lane_base + 256 + q4 * 32, v);
+        tmem_ld32(lane_base + 256 + q2 * 32, v);
         tmem_ld_wait();
         if (qj < p.c) {
           uint32_t w[16];
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
-            const __nv_bfloat162 pr = __floats2bfloat162_rn(v[i], v[i + 1]);
+            const __nv_bfloat162 pr = __floats2bfloat162_rn(v[i] * inv_l, v[i + 1] * inv_l);
             w[i >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
           }
-          uint4* d4 = reinterpret_cast<uint4*>(dst + q4 * 32);
+          uint4* d4 = reinterpret_cast<uint4*>(dst + q2 * 32);
 #pragma unroll
           for (int q = 0; q < 4; ++q) d4[q] = make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
         }
@@ -287,7 +314,7 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
 }
 
 size_t attn_smem_bytes() {
-  return static_cast<size_t>(2 + kAttnStages) * kAttnTileBytes + kAttnTailBytes;
+  return static_cast<size_t>(2 + kAttnStages) * kAttnTileBytes + kAttnTailBytes + kAttnXchgBytes;
 }
 
 cudaError_t launch_chunk_attention(const CUtensorMap& map_q, const CUtensorMap& map_k,

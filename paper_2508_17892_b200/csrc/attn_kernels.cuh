@@ -8,7 +8,7 @@
 
 namespace ilre {
 
-static constexpr int kAttnThreads = 192;     // warp 0 TMA, warp 1 MMA, warps 2..5 softmax
+static constexpr int kAttnThreads = 320;     // warp 0 TMA, warp 1 MMA, warps 2..9 softmax
 
 struct AttnParams {
   int c;             // query tokens of the chunk
