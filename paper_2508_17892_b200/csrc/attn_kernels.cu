@@ -3,13 +3,15 @@
 // where the first n_prefix rows of K/V are the cached sink and sliding-window tokens (visible
 // to every query of the chunk) and the remaining c rows the chunk's own (visible causally).
 //
-// One CTA per (128 query tokens, query head).  Both contractions run on the tensor cores:
-// S = Q K^T into tensor memory, and O += P V with P written to shared memory as bf16 by the
-// softmax warps.  One sweep over the key tiles with an online softmax: probabilities are taken
-// against a per-row reference maximum, O accumulates in tensor memory and is rescaled there
-// only when a row's maximum has run ahead of its reference by more than 2^8 (rare after the
-// first tiles); the row sums divide the output at the end.  Key and value tiles come through
-// one TMA ring.  Heavier CTAs (later query tiles see more keys) are launched first.
+// One CTA per (128 query tokens, pair of query heads that share a kv head).  Both contractions
+// run on the tensor cores: S = Q K^T into tensor memory, and O += P V with P written to shared
+// memory as bf16 by the softmax warps (eight per head).  The two heads are two independent streams over the
+// same key/value tiles (one TMA ring feeds both): while the softmax warpgroup of one stream
+// works on its S tile, the tensor cores serve the other stream.  One sweep over the key tiles
+// with an online softmax: probabilities are taken against a per-row reference maximum, O
+// accumulates in tensor memory and is rescaled there only when a row's maximum has run ahead
+// of its reference by more than 2^8 (rare after the first tiles); the row sums divide the
+// output at the end.  Heavier CTAs (later query tiles see more keys) are launched first.
 #include <cuda_bf16.h>
 
 #include "attn_kernels.cuh"
@@ -17,20 +19,20 @@
 
 namespace ilre {
 
-static constexpr int kAttnStages = 4;
+static constexpr int kAttnStages = 3;
 static constexpr int kAttnTileBytes = 128 * 128 * 2;       // one 128 x 128 bf16 tile
 static constexpr int kAttnTailBytes = 256;
-static constexpr int kAttnSoftmaxWarps = 8;          // two per TMEM lane quadrant: 64 columns each
-static constexpr int kAttnXchgBytes = 3 * 1024;      // tile maxima [2][2][128] + row sums [128]
+static constexpr int kAttnSoftmaxWarps = 8;                // per stream: two per TMEM lane quadrant
+static constexpr int kAttnXchgBytes = 2 * 1024;            // per stream: [2 halves][128 rows] floats
 
 struct AttnTail {
   uint64_t q_full;
   uint64_t kv_full[kAttnStages];
   uint64_t kv_empty[kAttnStages];
-  uint64_t s_full[2];
+  uint64_t s_full[2];          // per stream
   uint64_t s_empty[2];
-  uint64_t p_full;
-  uint64_t p_empty;
+  uint64_t p_full[2];
+  uint64_t p_empty[2];
   uint64_t o_full;
   uint32_t tmem_base;
   int abort_flag;
@@ -52,18 +54,19 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
                        const __grid_constant__ CUtensorMap map_v, const AttnParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t smem_base = smem_u32(smem);
-  const uint32_t q_s = smem_base;
-  const uint32_t ring_s = q_s + kAttnTileBytes;
-  const uint32_t p_s = ring_s + kAttnStages * kAttnTileBytes;
-  uint8_t* p_ptr = smem + (1 + kAttnStages) * kAttnTileBytes;
-  AttnTail* tail = reinterpret_cast<AttnTail*>(smem + (2 + kAttnStages) * kAttnTileBytes);
-  float* xchg_max = reinterpret_cast<float*>(smem + (2 + kAttnStages) * kAttnTileBytes + kAttnTailBytes);
-  float* xchg_sum = xchg_max + 512;
+  const uint32_t q_s = smem_base;                                        // 2 tiles
+  const uint32_t ring_s = q_s + 2 * kAttnTileBytes;
+  const uint32_t p_s = ring_s + kAttnStages * kAttnTileBytes;           // 2 tiles
+  uint8_t* p_ptr = smem + (2 + kAttnStages) * kAttnTileBytes;
+  AttnTail* tail = reinterpret_cast<AttnTail*>(smem + (4 + kAttnStages) * kAttnTileBytes);
+  float* xchg_all = reinterpret_cast<float*>(smem + (4 + kAttnStages) * kAttnTileBytes + kAttnTailBytes);
   volatile int* abort_flag = &tail->abort_flag;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   const int j0 = (gridDim.x - 1 - blockIdx.x) * 128;    // first query token; heavy tiles first
-  const int h = blockIdx.y, g = h / (p.n_q / p.n_kv);
+  const int n_streams = p.pair ? 2 : 1;
+  const int h0 = p.pair ? 2 * blockIdx.y : blockIdx.y;  // head of stream 0; stream 1 = h0 + 1
+  const int g = h0 / (p.n_q / p.n_kv);
   const int last_q = min(j0 + 128, p.c) - 1;
   const int n_tiles = (p.n_prefix + last_q) / 128 + 1;   // key tiles that hold a visible key
 
@@ -78,12 +81,12 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
       mbar_init(smem_u32(&tail->kv_full[s]), 1);
       mbar_init(smem_u32(&tail->kv_empty[s]), 1);
     }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(smem_u32(&tail->s_full[b]), 1);
-      mbar_init(smem_u32(&tail->s_empty[b]), kAttnSoftmaxWarps);
+    for (int x = 0; x < 2; ++x) {
+      mbar_init(smem_u32(&tail->s_full[x]), 1);
+      mbar_init(smem_u32(&tail->s_empty[x]), kAttnSoftmaxWarps);
+      mbar_init(smem_u32(&tail->p_full[x]), kAttnSoftmaxWarps);
+      mbar_init(smem_u32(&tail->p_empty[x]), 1);
     }
-    mbar_init(smem_u32(&tail->p_full), kAttnSoftmaxWarps);
-    mbar_init(smem_u32(&tail->p_empty), 1);
     mbar_init(smem_u32(&tail->o_full), 1);
     fence_mbar_init();
   }
@@ -95,16 +98,18 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tail->tmem_base;
-  const uint32_t tmem_o = tmem_base + 256;
   const bool run = (*abort_flag == 0);
 
-  // Ring items: K_0, V_0, K_1, V_1, ...
+  // TMEM columns: S of stream x at 128 x, O of stream x at 256 + 128 x.
+  // Ring items: K_0, V_0, K_1, V_1, ... each used by both streams.
   if (warp == 0) {
     if (lane == 0 && run) {
       const uint32_t qf = smem_u32(&tail->q_full);
-      mbar_arrive_expect_tx(qf, kAttnTileBytes);
-      tma_load_2d(q_s, &map_q, h * 128, j0, qf);
-      tma_load_2d(q_s + 16384, &map_q, h * 128 + 64, j0, qf);
+      mbar_arrive_expect_tx(qf, n_streams * kAttnTileBytes);
+      for (int x = 0; x < n_streams; ++x) {
+        tma_load_2d(q_s + x * kAttnTileBytes, &map_q, (h0 + x) * 128, j0, qf);
+        tma_load_2d(q_s + x * kAttnTileBytes + 16384, &map_q, (h0 + x) * 128 + 64, j0, qf);
+      }
       const int n_items = 2 * n_tiles;
       for (int it = 0; it < n_items; ++it) {
         const int s = it % kAttnStages;
@@ -126,76 +131,89 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
       constexpr uint32_t idesc_o = umma_idesc_bf16(128, 128) | (1u << 16);   // B = V: channels contiguous
       bool ok = mbar_wait(smem_u32(&tail->q_full), 0, abort_flag, p.status, kDevWaitQFull);
       tc_fence_after();
-      uint32_t u = 0;                                     // S accumulators issued so far
-      auto issue_s = [&](int item) -> bool {
-        const uint32_t b = u & 1u, use = u >> 1;
-        if (!mbar_wait(smem_u32(&tail->s_empty[b]), (use & 1u) ^ 1u, abort_flag, p.status,
-                       kDevWaitAccEmpty))
-          return false;
-        const int s = item % kAttnStages;
-        if (!mbar_wait(smem_u32(&tail->kv_full[s]), static_cast<uint32_t>(item / kAttnStages) & 1u,
-                       abort_flag, p.status, kDevWaitKFull))
-          return false;
-        tc_fence_after();
-        const uint32_t k_s = ring_s + s * kAttnTileBytes;
-#pragma unroll
-        for (int kb = 0; kb < 2; ++kb)
-#pragma unroll
-          for (int ks = 0; ks < 4; ++ks)
-            umma_bf16(tmem_base + b * 128, umma_desc_sw128(q_s + kb * 16384 + ks * 32),
-                      umma_desc_sw128(k_s + kb * 16384 + ks * 32), idesc_s, (kb | ks) != 0);
-        umma_commit(smem_u32(&tail->kv_empty[s]));
-        umma_commit(smem_u32(&tail->s_full[b]));
-        ++u;
-        return true;
+      auto ring_wait = [&](int item) -> bool {
+        return mbar_wait(smem_u32(&tail->kv_full[item % kAttnStages]),
+                         static_cast<uint32_t>(item / kAttnStages) & 1u, abort_flag, p.status,
+                         kDevWaitKFull);
       };
-      if (ok) ok = issue_s(0);                                                 // S of tile 0
-      for (int t = 0; t < n_tiles && ok; ++t) {
-        if (t + 1 < n_tiles) ok = issue_s(2 * (t + 1));                        // S of the next tile
-        if (!ok) break;
-        const int item = 2 * t + 1;                                            // V_t
-        const int s = item % kAttnStages;
-        ok = mbar_wait(smem_u32(&tail->p_full), static_cast<uint32_t>(t) & 1u, abort_flag, p.status,
-                       kDevWaitAccFull) &&
-             mbar_wait(smem_u32(&tail->kv_full[s]), static_cast<uint32_t>(item / kAttnStages) & 1u,
-                       abort_flag, p.status, kDevWaitKFull);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t v_s = ring_s + s * kAttnTileBytes;
+      auto issue_s = [&](int x, int t) {                  // S_x = Q_x K_t^T
+        const uint32_t k_s = ring_s + ((2 * t) % kAttnStages) * kAttnTileBytes;
+        const uint32_t qx = q_s + x * kAttnTileBytes;
 #pragma unroll
         for (int kb = 0; kb < 2; ++kb)
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks)
-            umma_bf16(tmem_o, umma_desc_sw128(p_s + kb * 16384 + ks * 32),
-                      umma_desc_sw128_mn(v_s + (kb * 64 + ks * 16) * 128, 16384, 1024), idesc_o,
-                      (t | kb | ks) != 0);
-        umma_commit(smem_u32(&tail->kv_empty[s]));
-        umma_commit(smem_u32(&tail->p_empty));
+            umma_bf16(tmem_base + x * 128, umma_desc_sw128(qx + kb * 16384 + ks * 32),
+                      umma_desc_sw128(k_s + kb * 16384 + ks * 32), idesc_s, (kb | ks) != 0);
+        umma_commit(smem_u32(&tail->s_full[x]));
+      };
+      if (ok) ok = ring_wait(0);
+      if (ok) {
+        tc_fence_after();
+        for (int x = 0; x < n_streams; ++x) issue_s(x, 0);
+        umma_commit(smem_u32(&tail->kv_empty[0]));
+      }
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        const int v_item = 2 * t + 1, k_item = 2 * t + 2;
+        const uint32_t v_s = ring_s + (v_item % kAttnStages) * kAttnTileBytes;
+        for (int x = 0; x < n_streams && ok; ++x) {
+          // O_x += P_x V_t
+          ok = mbar_wait(smem_u32(&tail->p_full[x]), static_cast<uint32_t>(t) & 1u, abort_flag,
+                         p.status, kDevWaitAccFull);
+          if (ok && x == 0) ok = ring_wait(v_item);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t px = p_s + x * kAttnTileBytes;
+#pragma unroll
+          for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+              umma_bf16(tmem_base + 256 + x * 128, umma_desc_sw128(px + kb * 16384 + ks * 32),
+                        umma_desc_sw128_mn(v_s + (kb * 64 + ks * 16) * 128, 16384, 1024), idesc_o,
+                        (t | kb | ks) != 0);
+          umma_commit(smem_u32(&tail->p_empty[x]));
+          if (x == n_streams - 1) umma_commit(smem_u32(&tail->kv_empty[v_item % kAttnStages]));
+          // S_x of the next tile: its softmax warps have read S_x(t) before they wrote P_x(t)
+          if (t + 1 < n_tiles) {
+            ok = mbar_wait(smem_u32(&tail->s_empty[x]), static_cast<uint32_t>(t) & 1u, abort_flag,
+                           p.status, kDevWaitAccEmpty);
+            if (ok && x == 0) ok = ring_wait(k_item);
+            if (!ok) break;
+            tc_fence_after();
+            issue_s(x, t + 1);
+            if (x == n_streams - 1) umma_commit(smem_u32(&tail->kv_empty[k_item % kAttnStages]));
+          }
+        }
       }
       if (ok) umma_commit(smem_u32(&tail->o_full));
     }
-  } else {
-    // Eight softmax warps: warp w reads TMEM lane quadrant w % 4; the two warps of a quadrant
-    // split the 128 columns (keys of S, channels of O) in halves.  A thread therefore owns
-    // half a query row; the two halves meet through shared memory once per tile (maximum).
-    // Every warp runs all iterations, also after a wait was abandoned, so that the named
-    // barrier below always gets its 256 threads.
-    const int quad = warp & 3, half = (warp - 2) >> 2;
+  } else if ((warp - 2) / kAttnSoftmaxWarps < n_streams) {
+    // Softmax warps of stream x: warp w reads TMEM lane quadrant w % 4; the two warps of a
+    // quadrant split the 128 columns (keys of S, channels of O) in halves, so a thread owns
+    // half a query row; the halves meet through shared memory once per tile (the maximum).
+    // Every warp runs all iterations, also after a wait was abandoned, so that the stream's
+    // named barrier always gets its 256 threads.
+    const int x = (warp - 2) / kAttnSoftmaxWarps;
+    const int quad = warp & 3, half = ((warp - 2) % kAttnSoftmaxWarps) >> 2;
     const int row = quad * 32 + lane;
     const int qj = j0 + row;
+    const int h = h0 + x;
     const int limit = p.n_prefix + qj;                   // last visible key row of this query
     const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + half * 64;
+    const uint32_t s_tm = lane_base + x * 128, o_tm = lane_base + 256 + x * 128;
+    uint8_t* p_mine = p_ptr + x * kAttnTileBytes + half * 16384;
+    float* xchg = xchg_all + x * 256;                    // [2][128]
+    const int bar_id = 1 + x;
     const float c2 = p.c2;
     bool ok = run;
-    uint32_t u = 0;
     // Online softmax: `ref` is the row's reference maximum (raw logits), `l` this thread's
     // share of the sum of 2^((s - ref) c2) over the keys seen so far.
     constexpr float kRefSlack = 8.f;                     // log2 units
     float ref = -INFINITY, l = 0.f;
-    for (int t = 0; t < n_tiles; ++t, ++u) {
-      const uint32_t b = u & 1u, use = u >> 1;
+    for (int t = 0; t < n_tiles; ++t) {
       if (ok)
-        ok = mbar_wait(smem_u32(&tail->s_full[b]), use & 1u, abort_flag, p.status, kDevWaitAccFull);
+        ok = mbar_wait(smem_u32(&tail->s_full[x]), static_cast<uint32_t>(t) & 1u, abort_flag,
+                       p.status, kDevWaitAccFull);
       // tile maximum of the visible logits
       float cm = -INFINITY;
       if (ok) {
@@ -203,7 +221,7 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
 #pragma unroll 1
         for (int q2 = 0; q2 < 2; ++q2) {
           float v[32];
-          tmem_ld32(lane_base + b * 128 + q2 * 32, v);
+          tmem_ld32(s_tm + q2 * 32, v);
           tmem_ld_wait();
           const int k0 = t * 128 + half * 64 + q2 * 32;
 #pragma unroll
@@ -211,9 +229,10 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
             if (k0 + i <= limit) cm = fmaxf(cm, v[i]);
         }
       }
-      xchg_max[((t & 1) * 2 + half) * 128 + row] = cm;
-      asm volatile("bar.sync 1, %0;" ::"r"(kAttnSoftmaxWarps * 32) : "memory");
-      cm = fmaxf(cm, xchg_max[((t & 1) * 2 + (half ^ 1)) * 128 + row]);
+      xchg[half * 128 + row] = cm;
+      asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(kAttnSoftmaxWarps * 32) : "memory");
+      cm = fmaxf(cm, xchg[(half ^ 1) * 128 + row]);
+      asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(kAttnSoftmaxWarps * 32) : "memory");
       if (!ok) continue;
       // move the reference only when the maximum has run ahead of it
       float scale = 1.f;
@@ -227,7 +246,7 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
 #pragma unroll
       for (int q2 = 0; q2 < 2; ++q2) {
         float v[32];
-        tmem_ld32(lane_base + b * 128 + q2 * 32, v);
+        tmem_ld32(s_tm + q2 * 32, v);
         tmem_ld_wait();
         const int k0 = t * 128 + half * 64 + q2 * 32;
 #pragma unroll
@@ -242,9 +261,9 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
       l = fmaf(l, scale, sum);
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&tail->s_empty[b]));
+      if (lane == 0) mbar_arrive(smem_u32(&tail->s_empty[x]));
       // the previous tile's P must have been consumed (and O updated) by its MMAs
-      ok = mbar_wait(smem_u32(&tail->p_empty), (static_cast<uint32_t>(t) & 1u) ^ 1u, abort_flag,
+      ok = mbar_wait(smem_u32(&tail->p_empty[x]), (static_cast<uint32_t>(t) & 1u) ^ 1u, abort_flag,
                      p.status, kDevWaitAccEmpty);
       if (!ok) continue;
       if (t > 0 && __any_sync(0xFFFFFFFFu, scale != 1.f)) {
@@ -253,43 +272,40 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
 #pragma unroll 1
         for (int q2 = 0; q2 < 2; ++q2) {
           float o[32];
-          tmem_ld32(lane_base + 256 + q2 * 32, o);
+          tmem_ld32(o_tm + q2 * 32, o);
           tmem_ld_wait();
 #pragma unroll
           for (int i = 0; i < 32; ++i) o[i] *= scale;
-          tmem_st32(lane_base + 256 + q2 * 32, o);
+          tmem_st32(o_tm + q2 * 32, o);
         }
         tmem_st_wait();
         tc_fence_before();
       }
-      // P[row][key]: two halves of 64 keys (one per warp of the quadrant), rows of 128 bytes,
-      // 16-byte groups XOR-swizzled by the row index (the layout TMA's 128-byte swizzle
-      // produces for the other operands)
+      // P[row][key]: one half of 64 keys per warp of the quadrant, rows of 128 bytes, 16-byte
+      // groups XOR-swizzled by the row index (the layout TMA's 128-byte swizzle produces for
+      // the other operands)
 #pragma unroll
       for (int c16 = 0; c16 < 8; ++c16) {
-        uint4* dst = reinterpret_cast<uint4*>(p_ptr + half * 16384 + row * 128 +
-                                              ((c16 ^ (row & 7)) << 4));
+        uint4* dst = reinterpret_cast<uint4*>(p_mine + row * 128 + ((c16 ^ (row & 7)) << 4));
         *dst = make_uint4(packed[c16 * 4], packed[c16 * 4 + 1], packed[c16 * 4 + 2],
                           packed[c16 * 4 + 3]);
       }
       fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&tail->p_full));
+      if (lane == 0) mbar_arrive(smem_u32(&tail->p_full[x]));
     }
     // ---- output: O / (sum of both halves), this thread's 64 channels ----
-    if (half == 1) xchg_sum[row] = l;
-    asm volatile("bar.sync 1, %0;" ::"r"(kAttnSoftmaxWarps * 32) : "memory");
-    if (half == 0) xchg_sum[row] += l;
-    asm volatile("bar.sync 1, %0;" ::"r"(kAttnSoftmaxWarps * 32) : "memory");
+    xchg[half * 128 + row] = l;
+    asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(kAttnSoftmaxWarps * 32) : "memory");
+    const float inv_l = 1.f / (l + xchg[(half ^ 1) * 128 + row]);
     if (ok) ok = mbar_wait(smem_u32(&tail->o_full), 0, abort_flag, p.status, kDevWaitAccFull);
     if (ok) {
       tc_fence_after();
       uint16_t* dst = p.out + (static_cast<size_t>(qj) * p.n_q + h) * 128 + half * 64;
-      const float inv_l = 1.f / xchg_sum[row];
 #pragma unroll 1
       for (int q2 = 0; q2 < 2; ++q2) {
         float v[32];
-        tmem_ld32(lane_base + 256 + q2 * 32, v);
+        tmem_ld32(o_tm + q2 * 32, v);
         tmem_ld_wait();
         if (qj < p.c) {
           uint32_t w[16];
@@ -314,7 +330,7 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
 }
 
 size_t attn_smem_bytes() {
-  return static_cast<size_t>(2 + kAttnStages) * kAttnTileBytes + kAttnTailBytes + kAttnXchgBytes;
+  return static_cast<size_t>(4 + kAttnStages) * kAttnTileBytes + kAttnTailBytes + kAttnXchgBytes;
 }
 
 cudaError_t launch_chunk_attention(const CUtensorMap& map_q, const CUtensorMap& map_k,
@@ -324,7 +340,7 @@ cudaError_t launch_chunk_attention(const CUtensorMap& map_q, const CUtensorMap& 
                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(smem));
   if (e != cudaSuccess) return e;
-  dim3 grid((p.c + 127) / 128, p.n_q);
+  dim3 grid((p.c + 127) / 128, p.pair ? p.n_q / 2 : p.n_q);
   chunk_attention_kernel<<<grid, kAttnThreads, smem, st>>>(map_q, map_k, map_v, p);
   return cudaGetLastError();
 }

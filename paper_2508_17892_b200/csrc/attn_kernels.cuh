@@ -8,19 +8,20 @@
 
 namespace ilre {
 
-static constexpr int kAttnThreads = 320;     // warp 0 TMA, warp 1 MMA, warps 2..9 softmax
+static constexpr int kAttnThreads = 576;     // warp 0 TMA, warp 1 MMA, warps 2..9 / 10..17 softmax
 
 struct AttnParams {
   int c;             // query tokens of the chunk
   int n_prefix;      // rows of K/V visible to every query (sink + sliding window)
   int n_q, n_kv;     // query heads, kv heads
+  int pair;          // 1: a CTA serves two query heads of one kv head; 0: one head
   float c2;          // log2(e) / sqrt(d)
   uint16_t* out;     // bf16 [c][n_q][128]
   int* status;
 };
 
 size_t attn_smem_bytes();
-// grid = (ceil(c / 128), n_q)
+// grid = (ceil(c / 128), n_q / 2 or n_q)
 cudaError_t launch_chunk_attention(const CUtensorMap& map_q, const CUtensorMap& map_k,
                                    const CUtensorMap& map_v, const AttnParams& p, cudaStream_t st);
 
