@@ -287,6 +287,7 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
   std::memset(&tbl, 0, sizeof(tbl));
   const long long Lp = L - spec->n_sink;
   tbl.n_comb = (budget > 0) ? spec->n_max * spec->n_win : 0;
+  long long allocated_before = 0;
   for (int i = 0, c = 0; i < spec->n_max && tbl.n_comb; ++i)
     for (int j = 0; j < spec->n_win; ++j, ++c) {
       const int m = spec->max_sizes[i];
@@ -296,8 +297,17 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
       tbl.m[c] = m;
       tbl.n[c] = spec->win_sizes[j];
       tbl.len[c] = static_cast<int>(len);
-      tbl.k_m[c] = static_cast<int>(km);
       tbl.quota[c] = budget / tbl.n_comb + (c < budget % tbl.n_comb ? 1 : 0);
+      // Algorithm 1 ranks K_m cells, but the quota walk of this combination cannot go further
+      // than quota cells that bring a new token plus the cells made up entirely of tokens the
+      // earlier combinations took (at most allocated / m full cells and the partial tail
+      // cell).  Ranking only that many gives the same walk and, for all but the last
+      // combinations, far fewer candidates to select and order.
+      long long reach = tbl.quota[c] + allocated_before / m + ((Lp % m) != 0 ? 1 : 0);
+      if (reach < 1) reach = 1;
+      if (km > reach) km = reach;
+      tbl.k_m[c] = static_cast<int>(km);
+      allocated_before += tbl.quota[c];
       tbl.tile_begin[c + 1] = tbl.tile_begin[c] + static_cast<int>((len + kSelTile - 1) / kSelTile);
       // the strided max-pool of size m is shared by all window sizes
       tbl.src[c] = -1;

@@ -1,7 +1,8 @@
 // Eq. 7: K~^{C_i} = R(D_i) K^{C_i} for the chunks i < N_C - 1 of the retrieval layer's key
 // cache, D_i = (N_C - 1 - i) * chunk positions, so that every cached key sits within two
 // chunks of the query.  A streaming kernel bound by HBM: every byte of the rotated part of
-// the cache is read once and written once.
+// the cache is read once and written once.  The file also holds the small gather that turns
+// the recalled positions into the compressed prompt.
 #include <cuda_bf16.h>
 
 #include "rerope_kernels.cuh"

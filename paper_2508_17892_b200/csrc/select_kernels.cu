@@ -409,18 +409,9 @@ __device__ __forceinline__ uint32_t block_exclusive_scan_1(uint32_t v, uint32_t 
 // `staged` room for kMaxKm cell ids in shared memory.  Every thread owns a run of consecutive
 // ranks; the cells of one combination are disjoint, so the new-token counts of all its cells
 // can be taken before any of them is marked.
-#ifdef ILRE_SELECT_TRACE
-#define ALLOC_TRACE(tag) do { if (combo < 2) SEL_TRACE(tag); } while (0)
-#define ALLOC_TRACE_ARGS , unsigned long long* trace_t, const char** trace_tag, int& trace_n
-#define ALLOC_TRACE_PASS , trace_t, trace_tag, trace_n
-#else
-#define ALLOC_TRACE(tag) do { } while (0)
-#define ALLOC_TRACE_ARGS
-#define ALLOC_TRACE_PASS
-#endif
 template <bool kBitmapInSmem>
 __device__ __forceinline__ void allocate(const ComboTable& tbl, const SelectParams& p,
-                                         uint8_t* dyn_smem, SelShared* sh ALLOC_TRACE_ARGS) {
+                                         uint8_t* dyn_smem, SelShared* sh) {
   // Two instantiations, so that the compiler knows the bitmap's address space on the common
   // path (shared memory) instead of going through generic loads and atomics.
   uint32_t* bm;
@@ -462,7 +453,6 @@ __device__ __forceinline__ void allocate(const ComboTable& tbl, const SelectPara
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
     if (p.stage_double && combo + 1 < tbl.n_comb) issue_copy(combo + 1);
-    ALLOC_TRACE("a:staged");
     const int per = (K + kSelThreads - 1) / kSelThreads;
     const int r0 = min(K, static_cast<int>(threadIdx.x) * per), r1 = min(K, r0 + per);
     uint32_t mine = 0;
@@ -470,7 +460,6 @@ __device__ __forceinline__ void allocate(const ComboTable& tbl, const SelectPara
       mine += __popcll(fresh_tokens<kBitmapInSmem>(bm, cells[r], m, Lp, p.n_sink));
     uint32_t total;
     uint32_t ord = block_exclusive_scan_1(mine, warp_totals, combo & 1, &total);
-    ALLOC_TRACE("a:counted");
     for (int r = r0; r < r1 && ord < quota; ++r) {
       const int cell = cells[r];
       unsigned long long fresh = fresh_tokens<kBitmapInSmem>(bm, cell, m, Lp, p.n_sink);
@@ -485,11 +474,7 @@ __device__ __forceinline__ void allocate(const ComboTable& tbl, const SelectPara
     if (total < quota && threadIdx.x == 0) atomicCAS(p.status, 0, kDevQuota);
     __syncthreads();                                         // bitmap updates visible to the block
     if (!p.stage_double && combo + 1 < tbl.n_comb) issue_copy(combo + 1);
-    ALLOC_TRACE("a:marked");
   }
-#ifdef ILRE_SELECT_TRACE
-  SEL_TRACE("a:rest");
-#endif
 
   // Ascending output.  Every warp owns a contiguous run of bitmap words and reads it 32
   // consecutive words at a time (one per lane).
@@ -729,9 +714,9 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
     }
     __syncthreads();
     SEL_TRACE("bitmap init");
-    allocate<true>(tbl, p, dyn_smem, &sh ALLOC_TRACE_PASS);
+    allocate<true>(tbl, p, dyn_smem, &sh);
   } else {
-    allocate<false>(tbl, p, dyn_smem, &sh ALLOC_TRACE_PASS);
+    allocate<false>(tbl, p, dyn_smem, &sh);
   }
   SEL_TRACE("allocate");
 #ifdef ILRE_SELECT_TRACE
