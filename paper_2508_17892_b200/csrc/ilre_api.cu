@@ -49,9 +49,7 @@ struct ilre_recall {
   float* pooled;
   float* maxpooled;
   uint32_t* hist;
-  unsigned long long* sel_prefix;
-  uint32_t* sel_krem;
-  uint32_t* sel_done;
+  int* tile_ties;
   uint32_t* grid_barrier;
   float2* rope_table;                   // (cos, sin) per (chunk distance, channel pair)
   int rope_rows, rope_chunk;            // what the table currently holds
@@ -126,7 +124,7 @@ bool dev_alloc(T** p, size_t count) {
 void free_all(ilre_recall* h) {
   cudaFree(h->qp); cudaFree(h->partial); cudaFree(h->nlse2); cudaFree(h->row_lse);
   cudaFree(h->enc); cudaFree(h->scores); cudaFree(h->pooled); cudaFree(h->maxpooled); cudaFree(h->hist);
-  cudaFree(h->sel_prefix); cudaFree(h->sel_krem); cudaFree(h->sel_done); cudaFree(h->grid_barrier); cudaFree(h->rope_table); cudaFree(h->pos_lo); cudaFree(h->pos_hi);
+  cudaFree(h->tile_ties); cudaFree(h->grid_barrier); cudaFree(h->rope_table); cudaFree(h->pos_lo); cudaFree(h->pos_hi);
   cudaFree(h->cand); cudaFree(h->cand_count); cudaFree(h->ranked); cudaFree(h->bitmap);
   cudaFree(h->status); cudaFree(h->stage_k); cudaFree(h->stage_q); cudaFree(h->stage_idx);
   for (int r = 0; r < kProfRing; ++r)
@@ -234,10 +232,8 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out) {
   ok = ok && dev_alloc(&h->scores, maxL);
   ok = ok && dev_alloc(&h->pooled, ncomb * maxL);
   ok = ok && dev_alloc(&h->maxpooled, ncomb * (maxL / 2 + 1));   // one array per distinct m > 1
-  ok = ok && dev_alloc(&h->hist, ncomb * kHistBins);
-  ok = ok && dev_alloc(&h->sel_prefix, ncomb);
-  ok = ok && dev_alloc(&h->sel_krem, ncomb);
-  ok = ok && dev_alloc(&h->sel_done, ncomb);
+  ok = ok && dev_alloc(&h->hist, static_cast<size_t>(kSelectPasses) * kMaxCombos * kHistBins);
+  ok = ok && dev_alloc(&h->tile_ties, ncomb * (maxL / kSelTile + 1));
   ok = ok && dev_alloc(&h->grid_barrier, 1);
   ok = ok && dev_alloc(&h->rope_table, static_cast<size_t>(kRopeTableRows) * kRopeHalfDim);
   h->pos_hi_rows = static_cast<int>(cfg->max_L / kRopeLoRows + 2);
@@ -343,10 +339,9 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
   std::memset(&pp, 0, sizeof(pp));
   pp.n_kv = h->cfg.n_kv_heads; pp.n_q = h->cfg.n_q_heads; pp.group_size = g.group_size;
   pp.q_len = q_len; pp.n_rb = g.n_rb; pp.rb_rows = g.rb_rows; pp.L = L; pp.n_sink = spec->n_sink;
-  pp.enc = h->enc; pp.bitmap = h->bitmap; pp.hist = h->hist; pp.hist_bins = kHistBins;
+  pp.enc = h->enc; pp.bitmap = h->bitmap; pp.hist = h->hist;
   pp.n_comb = tbl.n_comb;
-  for (int c = 0; c < tbl.n_comb; ++c) pp.k_m[c] = tbl.k_m[c];
-  pp.sel_prefix = h->sel_prefix; pp.sel_krem = h->sel_krem; pp.sel_done = h->sel_done;
+  pp.hist_words = static_cast<long long>(kSelectPasses) * tbl.n_comb * kHistBins;
   pp.cand_count = h->cand_count; pp.grid_barrier = h->grid_barrier;
 
   MergeParams mp;
@@ -360,7 +355,7 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
   sp.L = L; sp.n_sink = spec->n_sink; sp.win_op = spec->win_op;
   sp.pooled = h->pooled; sp.pooled_stride = h->cfg.max_L; sp.hist = h->hist;
   sp.maxpooled = h->maxpooled; sp.maxpooled_stride = h->cfg.max_L / 2 + 1;
-  sp.sel_prefix = h->sel_prefix; sp.sel_krem = h->sel_krem; sp.sel_done = h->sel_done;
+  sp.tile_ties = h->tile_ties;
   sp.cand = h->cand; sp.cand_stride = h->cand_stride;
   sp.cand_count = h->cand_count; sp.ranked = h->ranked; sp.bitmap = h->bitmap;
   sp.out_idx = out_idx_dev; sp.budget = budget; sp.barrier = h->grid_barrier;

@@ -431,13 +431,9 @@ __global__ void prepare_kernel(const uint4* __restrict__ q, uint4* __restrict__ 
     if (p.n_sink > lo) bits = (p.n_sink - lo >= 32) ? 0xFFFFFFFFu : ((1u << (p.n_sink - lo)) - 1u);
     p.bitmap[w] = bits;
   }
-  for (long long e = tid; e < static_cast<long long>(p.n_comb) * p.hist_bins; e += nthreads)
-    p.hist[e] = 0u;
+  for (long long e = tid; e < p.hist_words; e += nthreads) p.hist[e] = 0u;
   if (tid == 0) *p.grid_barrier = 0u;
   for (long long c = tid; c < p.n_comb; c += nthreads) {
-    p.sel_prefix[c] = 0ull;
-    p.sel_krem[c] = static_cast<uint32_t>(p.k_m[c]);
-    p.sel_done[c] = 0u;
     p.cand_count[c] = 0u;
   }
 }

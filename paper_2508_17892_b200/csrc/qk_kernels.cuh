@@ -54,12 +54,8 @@ struct PrepParams {
   uint32_t* enc;
   uint32_t* bitmap;
   uint32_t* hist;
-  int hist_bins;
+  long long hist_words;     // words of the radix histograms to clear
   int n_comb;
-  int k_m[64];
-  unsigned long long* sel_prefix;
-  uint32_t* sel_krem;
-  uint32_t* sel_done;
   uint32_t* cand_count;
   uint32_t* grid_barrier;   // arrival counter of the selection kernel's grid barrier
 };

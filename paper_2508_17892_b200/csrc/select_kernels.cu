@@ -4,10 +4,13 @@
 //   A  A^C[t] = exp2(max_r log2 p_rt) from the scores pass' encoded maxima (Eq. 5);
 //   B  MaxPooling(size = stride = m), once per distinct m, then the stride-1 window pooling
 //      (average or max) of every (m, n) combination, and the first radix histogram;
-//   C  radix select of the K_m largest 64-bit keys (pooled value, then lower cell index
-//      first), 11/11/10 bits per pass, all combinations at once; passes stop as soon as every
-//      combination's threshold is settled;
-//   D  gather of the selected keys;
+//   C  radix select of the K_m-th largest pooled value, 11/11/10 bits per pass, all
+//      combinations at once: the histograms are global, but every CTA works out the bin of
+//      the combinations it scans by itself, so a pass costs one grid barrier;
+//   D  where that value has more holders than are still wanted, the ones with the lowest cell
+//      index win (Algorithm 1's order: value descending, cell ascending): the tiles are in
+//      cell order, so a count of the holders per tile plus an ordered rank inside the tile
+//      settle it; then the gather of the selected keys;
 //   E  ranking (value descending, cell ascending) by counting, spread over the grid;
 //   F  one CTA walks the combinations in loop order: maps cells back to tokens, skips tokens
 //      already allocated, stops each combination at its quota B_c, then writes the allocated
@@ -39,8 +42,8 @@ __device__ __forceinline__ unsigned long long make_key(float w, uint32_t cell) {
 }
 
 __device__ __forceinline__ void pass_bits(int pass, int& shift, int& bits) {
-  const int sh[kSelectPasses] = {53, 42, 32, 21, 10, 0};
-  const int bt[kSelectPasses] = {11, 11, 10, 11, 11, 10};
+  const int sh[kSelectPasses] = {53, 42, 32};
+  const int bt[kSelectPasses] = {11, 11, 10};
   shift = sh[pass];
   bits = bt[pass];
 }
@@ -51,6 +54,8 @@ struct SelShared {
   int flag;
   unsigned long long prefix[kMaxCombos];   // per combination: radix prefix found so far
   uint32_t state[kMaxCombos];              // per combination: threshold settled / candidate count
+  uint32_t krem[kMaxCombos];               // per combination: keys still wanted inside the prefix
+  uint32_t tot[2][32];                     // warp totals of the one-barrier block scan
 };
 
 // Grid-wide barrier (all CTAs are co-resident: cooperative launch).  The arrival counter is
@@ -248,15 +253,18 @@ __device__ __forceinline__ void pool_tile(const ComboTable& tbl, const SelectPar
   __syncthreads();
 }
 
-// The CTA that owns `combo` in this pass locates the bin holding the k-th largest key among
-// those that match the prefix so far, extends the prefix, and clears the histogram.
-__device__ __forceinline__ void bin_search(const SelectParams& p, int combo, int pass,
+// Locates the bin of pass `pass` that holds the k-th largest key of `combo` among those that
+// match the prefix so far and extends the prefix.  Every CTA does this for the combinations
+// whose tiles it scans, from the same global histogram, so all of them reach the same answer.
+// The state lives in shared memory.  A combination is settled (state = 1) when every key of
+// the chosen bin is wanted: then "key >= prefix" selects exactly K_m keys.
+__device__ __forceinline__ void bin_search(const SelectParams& p, int n_comb, int combo, int pass,
                                            SelShared* sh) {
   int shift, bits;
   pass_bits(pass, shift, bits);
-  uint32_t* gh = p.hist + static_cast<long long>(combo) * kHistBins;
-  const unsigned long long prefix = __ldcg(&p.sel_prefix[combo]);
-  const uint32_t k_rem = __ldcg(&p.sel_krem[combo]);
+  const uint32_t* gh = p.hist + (static_cast<long long>(pass) * n_comb + combo) * kHistBins;
+  const unsigned long long prefix = sh->prefix[combo];
+  const uint32_t k_rem = sh->krem[combo];
   constexpr int kPer = kHistBins / kSelThreads;
   uint32_t h[kPer];
   uint32_t total = 0;
@@ -266,7 +274,7 @@ __device__ __forceinline__ void bin_search(const SelectParams& p, int combo, int
     total += h[j];
   }
   uint32_t grand;
-  const uint32_t excl = block_exclusive_scan(total, sh->scan, &grand);
+  const uint32_t excl = block_exclusive_scan(total, sh->scan, &grand);   // ends with a barrier
   if (excl < k_rem && k_rem <= excl + total) {
     uint32_t cum = excl;
 #pragma unroll
@@ -274,16 +282,15 @@ __device__ __forceinline__ void bin_search(const SelectParams& p, int combo, int
       if (k_rem > cum && k_rem <= cum + h[j]) {
         const uint32_t bin = kHistBins - 1 - (kPer * threadIdx.x + j);
         const uint32_t new_k = k_rem - cum;
-        p.sel_prefix[combo] = prefix | (static_cast<unsigned long long>(bin) << shift);
-        p.sel_krem[combo] = new_k;
-        p.sel_done[combo] = (h[j] == new_k || pass == kSelectPasses - 1) ? 1u : 0u;
+        sh->prefix[combo] = prefix | (static_cast<unsigned long long>(bin) << shift);
+        sh->krem[combo] = new_k;
+        sh->state[combo] = (h[j] == new_k) ? 1u : 0u;
       }
       cum += h[j];
     }
   }
   if (threadIdx.x == 0 && (k_rem > grand || k_rem == 0))
-    p.sel_done[combo] = 1u;                                // fewer keys than asked: take all
-  for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) gh[b] = 0u;
+    sh->state[combo] = 1u;                                 // fewer keys than asked: take all
   __syncthreads();
 }
 
@@ -575,67 +582,98 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
   if (!grid_sync(p, &sh, epoch)) return;
   SEL_TRACE("pool+hist0");
 
-  // ---- C: radix select ----
-  for (int pass = 0; pass < kSelectPasses; ++pass) {
-    if (pass > 0) {
-      int shift, bits;
-      pass_bits(pass, shift, bits);
-      const uint32_t mask = (1u << bits) - 1u;
-      for (int combo = threadIdx.x; combo < tbl.n_comb; combo += kSelThreads) {
-        sh.state[combo] = __ldcg(&p.sel_done[combo]);
-        sh.prefix[combo] = __ldcg(&p.sel_prefix[combo]);
-      }
-      __syncthreads();
-      int cur = -1, load_cursor = 0, cursor = 0;
-      for (int t0 = t_begin; t0 < t_end; t0 += kScanGroup) {
-        float wv[kScanGroup][kTilePer];
+  // ---- C: radix select of the K_m-th largest value ----
+  // combinations whose tiles this CTA scans
+  int c_lo = 0, c_hi = -1;
+  if (t_begin < t_end) {
+    int cursor = 0;
+    c_lo = combo_of_tile(tbl, t_begin, cursor);
+    c_hi = combo_of_tile(tbl, t_end - 1, cursor);
+  }
+  for (int combo = c_lo + threadIdx.x; combo <= c_hi; combo += kSelThreads) {
+    sh.prefix[combo] = 0ull;
+    sh.krem[combo] = static_cast<uint32_t>(tbl.k_m[combo]);
+    sh.state[combo] = 0u;
+  }
+  __syncthreads();
+  for (int combo = c_lo; combo <= c_hi; ++combo) bin_search(p, tbl.n_comb, combo, 0, &sh);
+  for (int pass = 1; pass < kSelectPasses; ++pass) {
+    int shift, bits;
+    pass_bits(pass, shift, bits);
+    const uint32_t mask = (1u << bits) - 1u;
+    uint32_t* hist_pass = p.hist + static_cast<long long>(pass) * tbl.n_comb * kHistBins;
+    int cur = -1, load_cursor = 0, cursor = 0;
+    for (int t0 = t_begin; t0 < t_end; t0 += kScanGroup) {
+      float wv[kScanGroup][kTilePer];
 #pragma unroll
-        for (int g = 0; g < kScanGroup; ++g)
-          if (t0 + g < t_end) fetch_tile(tbl, p, t0 + g, load_cursor, sh.state, wv[g]);
+      for (int g = 0; g < kScanGroup; ++g)
+        if (t0 + g < t_end) fetch_tile(tbl, p, t0 + g, load_cursor, sh.state, wv[g]);
 #pragma unroll
-        for (int g = 0; g < kScanGroup; ++g) {
-          const int tile = t0 + g;
-          if (tile >= t_end) break;
-          const int combo = combo_of_tile(tbl, tile, cursor);
-          if (sh.state[combo]) continue;
-          if (combo != cur && cur >= 0)
-            hist_flush(sh.hist, p.hist + static_cast<long long>(cur) * kHistBins);
-          cur = combo;
-          const unsigned long long prefix = sh.prefix[combo];
-          const int c0 = (tile - tbl.tile_begin[combo]) * kSelTile;
-          const int c1 = min(tbl.len[combo], c0 + kSelTile);
+      for (int g = 0; g < kScanGroup; ++g) {
+        const int tile = t0 + g;
+        if (tile >= t_end) break;
+        const int combo = combo_of_tile(tbl, tile, cursor);
+        if (sh.state[combo]) continue;
+        if (combo != cur && cur >= 0)
+          hist_flush(sh.hist, hist_pass + static_cast<long long>(cur) * kHistBins);
+        cur = combo;
+        const unsigned long long prefix = sh.prefix[combo];
+        const int c0 = (tile - tbl.tile_begin[combo]) * kSelTile;
+        const int c1 = min(tbl.len[combo], c0 + kSelTile);
 #pragma unroll
-          for (int k = 0; k < kTilePer; ++k) {
-            const int c = c0 + k * kSelThreads + threadIdx.x;
-            uint32_t digit = 0xFFFFFFFFu;                    // sentinel: does not take part
-            if (c < c1) {
-              const unsigned long long key = make_key(wv[g][k], static_cast<uint32_t>(c));
-              if (((key ^ prefix) >> (shift + bits)) == 0ull)
-                digit = static_cast<uint32_t>(key >> shift) & mask;
-            }
-            hist_add(sh.hist, digit);
+        for (int k = 0; k < kTilePer; ++k) {
+          const int c = c0 + k * kSelThreads + threadIdx.x;
+          uint32_t digit = 0xFFFFFFFFu;                    // sentinel: does not take part
+          if (c < c1) {
+            const unsigned long long key = make_key(wv[g][k], static_cast<uint32_t>(c));
+            if (((key ^ prefix) >> (shift + bits)) == 0ull)
+              digit = static_cast<uint32_t>(key >> shift) & mask;
           }
+          hist_add(sh.hist, digit);
         }
       }
-      if (cur >= 0) hist_flush(sh.hist, p.hist + static_cast<long long>(cur) * kHistBins);
-      if (!grid_sync(p, &sh, epoch)) return;
-      SEL_TRACE("histogram");
     }
-    for (int combo = blockIdx.x; combo < tbl.n_comb; combo += gridDim.x)
-      if (__ldcg(&p.sel_done[combo]) == 0u) bin_search(p, combo, pass, &sh);
+    if (cur >= 0) hist_flush(sh.hist, hist_pass + static_cast<long long>(cur) * kHistBins);
     if (!grid_sync(p, &sh, epoch)) return;
-    SEL_TRACE("bin search");
-    int pending = 0;
-    for (int combo = threadIdx.x; combo < tbl.n_comb; combo += kSelThreads)
-      pending |= (__ldcg(&p.sel_done[combo]) == 0u);
-    if (!__syncthreads_or(pending)) break;                   // same data in every CTA
+    SEL_TRACE("histogram");
+    for (int combo = c_lo; combo <= c_hi; ++combo)
+      if (sh.state[combo] == 0u) bin_search(p, tbl.n_comb, combo, pass, &sh);
   }
 
-  // ---- D: gather the keys at or above each combination's threshold ----
+  // ---- D: ties at the K_m-th value, then the gather ----
+  // A combination that is not settled by now has its K_m-th value v (upper half of the
+  // prefix) and wants krem of the cells that hold exactly v: the ones with the lowest index.
   {
-    for (int combo = threadIdx.x; combo < tbl.n_comb; combo += kSelThreads)
-      sh.prefix[combo] = __ldcg(&p.sel_prefix[combo]);
-    __syncthreads();
+    int load_cursor = 0, cursor = 0;
+    for (int t0 = t_begin; t0 < t_end; t0 += kScanGroup) {
+      float wv[kScanGroup][kTilePer];
+#pragma unroll
+      for (int g = 0; g < kScanGroup; ++g)
+        if (t0 + g < t_end) fetch_tile(tbl, p, t0 + g, load_cursor, sh.state, wv[g]);
+#pragma unroll
+      for (int g = 0; g < kScanGroup; ++g) {
+        const int tile = t0 + g;
+        if (tile >= t_end) break;
+        const int combo = combo_of_tile(tbl, tile, cursor);
+        if (sh.state[combo]) continue;
+        const uint32_t v_star = static_cast<uint32_t>(sh.prefix[combo] >> 32);
+        const int c0 = (tile - tbl.tile_begin[combo]) * kSelTile;
+        const int c1 = min(tbl.len[combo], c0 + kSelTile);
+        int mine = 0;
+#pragma unroll
+        for (int k = 0; k < kTilePer; ++k) {
+          const int c = c0 + k * kSelThreads + threadIdx.x;
+          mine += (c < c1 && float_to_ordered(wv[g][k]) == v_star) ? 1 : 0;
+        }
+        const int holders = __syncthreads_count(mine & 1) + 2 * __syncthreads_count(mine & 2) +
+                            4 * __syncthreads_count(mine & 4);
+        if (threadIdx.x == 0) p.tile_ties[tile] = holders;
+      }
+    }
+  }
+  if (!grid_sync(p, &sh, epoch)) return;
+  SEL_TRACE("tie count");
+  {
     const int lane = threadIdx.x & 31;
     int load_cursor = 0, cursor = 0;
     for (int t0 = t_begin; t0 < t_end; t0 += kScanGroup) {
@@ -648,18 +686,43 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
         const int tile = t0 + g;
         if (tile >= t_end) break;
         const int combo = combo_of_tile(tbl, tile, cursor);
+        const bool settled = sh.state[combo] != 0u;
         const unsigned long long threshold = sh.prefix[combo];
+        const uint32_t v_star = static_cast<uint32_t>(threshold >> 32);
+        const uint32_t wanted = sh.krem[combo];
         unsigned long long* cand = p.cand + static_cast<long long>(combo) * p.cand_stride;
         const int c0 = (tile - tbl.tile_begin[combo]) * kSelTile;
         const int c1 = min(tbl.len[combo], c0 + kSelTile);
+        // holders of v in the earlier tiles of this combination (tiles are in cell order)
+        uint32_t before = 0;
+        bool ties_here = false;
+        if (!settled) {
+          ties_here = __ldcg(&p.tile_ties[tile]) > 0;      // uniform
+          if (ties_here) {
+            uint32_t part = 0;
+            for (int t = tbl.tile_begin[combo] + threadIdx.x; t < tile; t += kSelThreads)
+              part += static_cast<uint32_t>(__ldcg(&p.tile_ties[t]));
+            block_exclusive_scan_1(part, sh.tot, 0, &before);
+            __syncthreads();
+          }
+        }
 #pragma unroll
         for (int k = 0; k < kTilePer; ++k) {
           const int c = c0 + k * kSelThreads + threadIdx.x;
           unsigned long long key = 0ull;
-          bool take = false;
+          bool take = false, holder = false;
           if (c < c1) {
             key = make_key(wv[g][k], static_cast<uint32_t>(c));
-            take = key >= threshold;
+            const uint32_t v = static_cast<uint32_t>(key >> 32);
+            if (settled) take = key >= threshold;
+            else { take = v > v_star; holder = v == v_star; }
+          }
+          if (ties_here) {                                 // uniform
+            uint32_t in_row;
+            const uint32_t rank = before + block_exclusive_scan_1(holder ? 1u : 0u, sh.tot, 1, &in_row);
+            __syncthreads();
+            if (holder && rank < wanted) take = true;
+            before += in_row;
           }
           const uint32_t votes = __ballot_sync(0xFFFFFFFFu, take);
           if (votes) {

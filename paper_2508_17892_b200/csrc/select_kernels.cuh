@@ -11,7 +11,7 @@ static constexpr int kHistBins = 2048;
 static constexpr int kMaxWin = 1024;        // largest stride-1 window size
 static constexpr int kMaxMaxSize = 64;      // largest strided max-pool size
 static constexpr int kMaxKm = 16384;        // largest K_m (bounds the candidate lists)
-static constexpr int kSelectPasses = 6;     // 64-bit (value, index) key, 11/11/10 bits twice
+static constexpr int kSelectPasses = 3;     // 32 value bits of the key in 11/11/10-bit digits
 static constexpr int kSelThreads = 1024;    // threads per CTA of the selection kernel
 static constexpr int kSelTile = 4096;       // cells of one combination per work tile
 static constexpr int kSrcTileTokens = 8192; // tokens per work tile of the strided max-pool
@@ -48,10 +48,8 @@ struct SelectParams {
   long long maxpooled_stride;
   float* pooled;           // [n_comb][pooled_stride]
   long long pooled_stride;
-  uint32_t* hist;          // [n_comb][kHistBins], zero on entry and on exit
-  unsigned long long* sel_prefix;
-  uint32_t* sel_krem;
-  uint32_t* sel_done;
+  uint32_t* hist;          // [kSelectPasses][n_comb][kHistBins], zero on entry
+  int* tile_ties;          // [work tiles]: cells of a tile that hold the K_m-th value
   unsigned long long* cand;   // [n_comb][cand_stride] selected 64-bit keys
   int cand_stride;
   uint32_t* cand_count;
