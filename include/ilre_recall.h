@@ -198,8 +198,8 @@ int ilre_recall_status(ilre_recall_t* h);
  * resets the history.  ilre_recall_stage_times synchronises on those events and writes up to
  * n entries, each the mean over the recorded runs (milliseconds), in this order:
  *   0 prepare (query packing, clears)   1 row statistics (QK^T + online softmax)
- *   2 statistics merge                  3 scores (QK^T + max over rows)
- *   4 Algorithm 1 (A^C from the maxima, pooling, top-K_m selection and ranking, allocation,
+ *   2 scores (statistics merge, QK^T + max over rows)
+ *   3 Algorithm 1 (A^C from the maxima, pooling, top-K_m selection and ranking, allocation,
  *     ascending output; one kernel)
  * Returns the number of entries written, or a negative status.
  */

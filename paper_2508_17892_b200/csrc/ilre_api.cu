@@ -25,7 +25,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-constexpr int kNumStages = 5;            // timed stages (see ilre_recall_stage_times)
+constexpr int kNumStages = 4;            // timed stages (see ilre_recall_stage_times)
 constexpr int kProfRing = 32;            // runs whose stage events are kept for averaging
 constexpr int kMaxSinkStaging = 65536;
 
@@ -42,7 +42,6 @@ struct ilre_recall {
   // workspace (device)
   void* qp;
   float* partial;
-  float* nlse2;
   float* row_lse;
   uint32_t* enc;
   float* scores;
@@ -122,7 +121,7 @@ bool dev_alloc(T** p, size_t count) {
 }
 
 void free_all(ilre_recall* h) {
-  cudaFree(h->qp); cudaFree(h->partial); cudaFree(h->nlse2); cudaFree(h->row_lse);
+  cudaFree(h->qp); cudaFree(h->partial); cudaFree(h->row_lse);
   cudaFree(h->enc); cudaFree(h->scores); cudaFree(h->pooled); cudaFree(h->maxpooled); cudaFree(h->hist);
   cudaFree(h->tile_ties); cudaFree(h->grid_barrier); cudaFree(h->rope_table); cudaFree(h->pos_lo); cudaFree(h->pos_hi);
   cudaFree(h->cand); cudaFree(h->cand_count); cudaFree(h->ranked); cudaFree(h->bitmap);
@@ -226,7 +225,6 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out) {
   bool ok = true;
   ok = ok && dev_alloc(reinterpret_cast<uint8_t**>(&h->qp), cfg->n_kv_heads * rows_pad * 256);
   ok = ok && dev_alloc(&h->partial, max_items * kMaxRbRows * 2);
-  ok = ok && dev_alloc(&h->nlse2, cfg->n_kv_heads * rows_pad);
   ok = ok && dev_alloc(&h->row_lse, static_cast<size_t>(cfg->max_q_len) * cfg->n_q_heads);
   ok = ok && dev_alloc(&h->enc, maxL);
   ok = ok && dev_alloc(&h->scores, maxL);
@@ -333,7 +331,7 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
   qk.L = L; qk.n_tiles = g.n_tiles; qk.n_groups = g.n_groups; qk.n_rb = g.n_rb;
   qk.rb_rows = g.rb_rows; qk.cpg = g.cpg; qk.stages = g.stages;
   qk.c2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(kHeadDim)));
-  qk.partial = h->partial; qk.nlse2 = h->nlse2; qk.enc = h->enc; qk.status = h->status;
+  qk.partial = h->partial; qk.enc = h->enc; qk.status = h->status;
 
   PrepParams pp;
   std::memset(&pp, 0, sizeof(pp));
@@ -347,7 +345,7 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
   MergeParams mp;
   mp.n_groups = g.n_groups; mp.n_rb = g.n_rb; mp.rb_rows = g.rb_rows; mp.cpg = g.cpg;
   mp.group_size = g.group_size; mp.q_len = q_len; mp.n_q = h->cfg.n_q_heads;
-  mp.partial = h->partial; mp.nlse2 = h->nlse2; mp.row_lse = h->row_lse;
+  mp.partial = h->partial; mp.row_lse = h->row_lse;
 
   SelectParams sp;
   std::memset(&sp, 0, sizeof(sp));
@@ -386,12 +384,10 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
   ILRE_MARK(1);
   ILRE_CUDA(launch_row_stats(map_k, map_q, qk, st)); ++launches;
   ILRE_MARK(2);
-  ILRE_CUDA(launch_merge_stats(mp, st)); ++launches;
+  ILRE_CUDA(launch_scores(map_k, map_q, qk, mp, st)); ++launches;
   ILRE_MARK(3);
-  ILRE_CUDA(launch_scores(map_k, map_q, qk, st)); ++launches;
-  ILRE_MARK(4);
   ILRE_CUDA(launch_select(tbl, sp, select_grid, select_smem, st)); ++launches;
-  ILRE_MARK(5);
+  ILRE_MARK(4);
 #undef ILRE_MARK
   h->last_launches = launches;
   if (prof) ++h->prof_runs;

@@ -293,12 +293,36 @@ row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
   cta_teardown(tmem_base);
 }
 
+// Combines the per-key-chunk partial statistics of one row into -lse (log2 units; -inf marks
+// a padding row); `publish` also stores the user-visible natural-log lse.
+__device__ __forceinline__ float merged_neg_lse2(const MergeParams& p, int group, int within,
+                                                 bool publish) {
+  const int g = group / p.n_rb, rb = group % p.n_rb;
+  const int rg = rb * p.rb_rows + within;
+  if (rg >= p.group_size * p.q_len) return -INFINITY;
+  const float2* part = reinterpret_cast<const float2*>(p.partial) +
+                       static_cast<size_t>(group) * p.cpg * p.rb_rows + within;
+  float mm = -INFINITY;
+  for (int c = 0; c < p.cpg; ++c) mm = fmaxf(mm, __ldcg(&part[static_cast<size_t>(c) * p.rb_rows]).x);
+  float zz = 0.f;
+  for (int c = 0; c < p.cpg; ++c) {
+    const float2 v = __ldcg(&part[static_cast<size_t>(c) * p.rb_rows]);
+    zz += v.y * exp2f(v.x - mm);
+  }
+  const float lse2 = mm + log2f(zz);
+  if (publish) {
+    const int i = rg / p.group_size, j = rg % p.group_size;
+    p.row_lse[i * p.n_q + g * p.group_size + j] = lse2 * 0.69314718055994530942f;
+  }
+  return -lse2;
+}
+
 // ---------------------------------------------------------------------------------------
 // Pass B: scores.  D[key, row]; per context position max over rows of log2-probability.
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kQkThreads, 1)
 scores_kernel(const __grid_constant__ CUtensorMap tmapK,
-              const __grid_constant__ CUtensorMap tmapQ, const QkParams p) {
+              const __grid_constant__ CUtensorMap tmapQ, const QkParams p, const MergeParams mp) {
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t smem_base = smem_u32(smem);
   const uint32_t q_s = smem_base;
@@ -310,8 +334,10 @@ scores_kernel(const __grid_constant__ CUtensorMap tmapK,
   const CtaItem it = decode_item(p);
   const int n_nh = (p.rb_rows + 255) / 256;
 
+  // Every CTA merges the per-key-chunk statistics of its own rows (a few KB from L2); the
+  // CTAs of the first key chunk also publish the natural-log lse.
   for (int i = threadIdx.x; i < p.rb_rows; i += blockDim.x)
-    nl[i] = p.nlse2[static_cast<size_t>(it.group) * p.rb_rows + i];
+    nl[i] = merged_neg_lse2(mp, it.group, i, it.chunk == 0);
   const uint32_t tmem_base = cta_setup(tail, smem_base, p.stages, 2, kConsumerWarps, p.status);
   const bool run = (it.n_tiles > 0) && (*abort_flag == 0);
 
@@ -438,30 +464,6 @@ __global__ void prepare_kernel(const uint4* __restrict__ q, uint4* __restrict__ 
   }
 }
 
-// Combines the per-key-chunk partial statistics of every row into lse (log2 units, negated
-// for the scores pass; -inf marks padding rows) and the user-visible natural-log lse.
-__global__ void merge_stats_kernel(MergeParams p) {
-  const int prow = blockIdx.x * blockDim.x + threadIdx.x;
-  if (prow >= p.n_groups * p.rb_rows) return;
-  const int within = prow % p.rb_rows, group = prow / p.rb_rows;
-  const int g = group / p.n_rb, rb = group % p.n_rb;
-  const int rg = rb * p.rb_rows + within;
-  if (rg >= p.group_size * p.q_len) { p.nlse2[prow] = -INFINITY; return; }
-  const float2* part = reinterpret_cast<const float2*>(p.partial) +
-                       static_cast<size_t>(group) * p.cpg * p.rb_rows + within;
-  float mm = -INFINITY;
-  for (int c = 0; c < p.cpg; ++c) mm = fmaxf(mm, part[static_cast<size_t>(c) * p.rb_rows].x);
-  float zz = 0.f;
-  for (int c = 0; c < p.cpg; ++c) {
-    const float2 v = part[static_cast<size_t>(c) * p.rb_rows];
-    zz += v.y * exp2f(v.x - mm);
-  }
-  const float lse2 = mm + log2f(zz);
-  p.nlse2[prow] = -lse2;
-  const int i = rg / p.group_size, j = rg % p.group_size;
-  p.row_lse[i * p.n_q + g * p.group_size + j] = lse2 * 0.69314718055994530942f;
-}
-
 // ---------------------------------------------------------------------------------------
 // host-side launchers
 // ---------------------------------------------------------------------------------------
@@ -496,24 +498,18 @@ cudaError_t launch_row_stats(const CUtensorMap& tk, const CUtensorMap& tq, const
 }
 
 cudaError_t launch_scores(const CUtensorMap& tk, const CUtensorMap& tq, const QkParams& p,
-                          cudaStream_t st) {
+                          const MergeParams& mp, cudaStream_t st) {
   const size_t smem = scores_smem_bytes(p.rb_rows, p.stages);
   cudaError_t e = cudaFuncSetAttribute(scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
-  scores_kernel<<<p.n_groups * p.cpg, kQkThreads, smem, st>>>(tk, tq, p);
+  scores_kernel<<<p.n_groups * p.cpg, kQkThreads, smem, st>>>(tk, tq, p, mp);
   return cudaGetLastError();
 }
 
 cudaError_t launch_prepare(const void* q, void* qp, const PrepParams& p, int n_sm,
                            cudaStream_t st) {
   prepare_kernel<<<n_sm * 4, 256, 0, st>>>(static_cast<const uint4*>(q), static_cast<uint4*>(qp), p);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_merge_stats(const MergeParams& p, cudaStream_t st) {
-  const int n = p.n_groups * p.rb_rows;
-  merge_stats_kernel<<<(n + 127) / 128, 128, 0, st>>>(p);
   return cudaGetLastError();
 }
 

@@ -42,7 +42,6 @@ struct QkParams {
   int stages;
   float c2;          // log2(e) / sqrt(d)
   float* partial;    // [n_groups][cpg][rb_rows][2]: (max * c2, sum-exp) per key chunk
-  const float* nlse2;  // [n_groups][rb_rows]: -lse in log2 units, -inf for padding rows
   uint32_t* enc;     // [L]: order-preserving uint of max_r log2 p_rt
   int* status;
 };
@@ -63,7 +62,6 @@ struct PrepParams {
 struct MergeParams {
   int n_groups, n_rb, rb_rows, cpg, group_size, q_len, n_q;
   const float* partial;
-  float* nlse2;
   float* row_lse;    // [q_len][n_q] natural-log lse
 };
 
@@ -73,8 +71,7 @@ size_t scores_smem_bytes(int rb_rows, int stages);
 cudaError_t launch_prepare(const void* q, void* qp, const PrepParams& p, int n_sm, cudaStream_t st);
 cudaError_t launch_row_stats(const CUtensorMap& tk, const CUtensorMap& tq, const QkParams& p,
                              cudaStream_t st);
-cudaError_t launch_merge_stats(const MergeParams& p, cudaStream_t st);
 cudaError_t launch_scores(const CUtensorMap& tk, const CUtensorMap& tq, const QkParams& p,
-                          cudaStream_t st);
+                          const MergeParams& mp, cudaStream_t st);
 
 }  // namespace ilre

@@ -15,7 +15,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libilre_recall.so")
 
-STAGE_NAMES = ("prepare", "row_stats", "merge_stats", "scores", "select")
+STAGE_NAMES = ("prepare", "row_stats", "scores", "select")
 
 EXPORTED_SYMBOLS = (
     "ilre_recall_create", "ilre_recall_run", "ilre_recall_run_host", "ilre_recall_fill_keys",
