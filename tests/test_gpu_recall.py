@@ -134,6 +134,38 @@ def test_selection_kernel_edge_paths(case):
     eng.close()
 
 
+@pytest.mark.parametrize("pattern", ["all_equal", "two_levels", "blocks_of_equal"])
+@pytest.mark.parametrize("win_op", [0, 1])
+def test_massive_ties_follow_the_cell_order(pattern, win_op):
+    """Keys that repeat make whole stretches of the scores bit-identical, so the K_m-th value
+    is held by thousands of cells and the lower cell index has to decide (reading 11)."""
+    import dataclasses
+    L, q_len = 9000, 3
+    w = small_workload(L, q_len, seed=3, n_spans=0, budget=700, max_sizes=(1, 2), win_sizes=(1, 3),
+                       win_op=win_op, n_sink=2)
+    x = make_inputs(w)
+    g = torch.Generator().manual_seed(17)
+    K = x.K.clone()
+    if pattern == "all_equal":
+        K[:] = K[0]
+    elif pattern == "two_levels":
+        K[: L // 2] = K[0]
+        K[L // 2:] = K[1]
+    else:
+        protos = torch.randn(9, 8, 128, generator=g).to(torch.bfloat16)
+        for b in range(9):
+            K[b * 1000:(b + 1) * 1000] = protos[b]
+    x = dataclasses.replace(x, K=K.contiguous())
+    eng = _engine(w)
+    idx, sc = _run(eng, x)
+    rep = parity.check_recall(x.K, x.Q, w, idx, sc)
+    # the device scores really are bit-identical inside a stretch
+    if pattern == "all_equal":
+        assert np.unique(sc).size == 1
+    print(pattern, win_op, rep)
+    eng.close()
+
+
 def test_handle_reuse_and_determinism(cases):
     # one handle, different shapes back to back, and bit-identical repeats
     big = make_inputs(CONFIGS["cfg2_L32k"])
