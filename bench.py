@@ -363,6 +363,44 @@ def run_ours(args, world, rank, local):
                     bound="tensor", peak=pk, frac=fl / (ms * 1e-3) / 1e12 / pk)
         del Qa, Ka, Va
 
+    # Key-range sharded recall: the three per-rank steps of a P-way split, timed on one
+    # GPU for the first shard (the exchanges between them, 2 floats per query row and one
+    # float per position, are not timed here)
+    shard = None
+    if args.shards > 1 and rank == 0:
+        from paper_2508_17892_b200.sharded import shard_bounds
+        lo, hi = shard_bounds(w.L, args.shards, 0)
+        Ks = K[lo:hi]
+        n_rows = w.q_len * w.n_q_heads
+        st_one = torch.empty(n_rows, 2, dtype=torch.float32, device=dev)
+        sc_one = torch.empty(hi - lo, dtype=torch.float32, device=dev)
+        sc_all = torch.empty(w.L, dtype=torch.float32, device=dev)
+        eng.run(K, Q, *spec, out_idx=out_idx, out_scores=sc_all)
+        eng.shard_stats(Ks, Q, out=st_one)
+        st_all = st_one.unsqueeze(0).repeat(args.shards, 1, 1).contiguous()
+
+        def timed_ms(fn, reps=50):
+            for _ in range(3):
+                fn()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record()
+            for _ in range(reps):
+                fn()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / reps
+
+        ms_stats = timed_ms(lambda: eng.shard_stats(Ks, Q, out=st_one))
+        ms_scores = timed_ms(lambda: eng.shard_scores(Ks, Q, st_all, out=sc_one))
+        ms_alloc = timed_ms(lambda: eng.allocate(sc_all, *spec, out_idx=out_idx))
+        shard = dict(shards=args.shards, keys_per_shard=hi - lo, shard_stats_ms=ms_stats,
+                     shard_scores_ms=ms_scores, allocate_ms=ms_alloc,
+                     per_rank_ms=ms_stats + ms_scores + ms_alloc,
+                     exchange_bytes_per_rank=dict(statistics=n_rows * 8, scores=(hi - lo) * 4),
+                     note="one GPU, first shard; all-gathers not included")
+        eng.check_status()
+
     elapsed_max, units = aggregate(elapsed_ms, float(k_bytes) * args.steps, dev)
     if rank != 0:
         return
@@ -414,6 +452,7 @@ def run_ours(args, world, rank, local):
                 clocks=clocks, e2e=e2e, gpu_launches=launches, roofline=roofline,
                 cpu_baseline=cpu_baseline,
                 stages_ms=stages, dca_rerope=dca, key_fill=fill, chunk_attention=attn,
+                sharded_steps=shard,
                 whole_step=dict(hbm_frac_one_read_of_K=step_hbm_frac,
                                 tensor_frac_one_qk=step_tensor_frac,
                                 hbm_frac_of_8TBps=(k_bytes / (ms_per_step * 1e-3) / 1e9) / 8000.0))
@@ -438,6 +477,8 @@ def main():
                     help="also time the chunked prefill attention of one chunk (0 = skip)")
     ap.add_argument("--fill-tokens", type=int, default=1048576,
                     help="also time the key-cache fill over this many tokens (0 = skip)")
+    ap.add_argument("--shards", type=int, default=8,
+                    help="also time the per-rank steps of a key-range split this many ways (0 = skip)")
     ap.add_argument("--cpu-sample-keys", type=int, default=131072)
     ap.add_argument("--ref-sample-keys", type=int, default=4096)
     args = ap.parse_args()

@@ -107,6 +107,40 @@ int ilre_recall_run_host(ilre_recall_t* h,
                          void* cuda_stream);
 
 /*
+ * Key-range sharded recall (the context's keys split by position over several GPUs, as the
+ * key cache of a long context is when it does not fit, or is not produced on, one device).
+ * Eq. 4's softmax runs over ALL keys, so a shard needs every shard's row statistics before it
+ * can score its own positions; Eq. 5 and Algorithm 1 then need every position's score.  The
+ * three calls below are the per-rank steps, with one all-gather between each pair (the caller
+ * owns the exchange; the library never talks to a peer):
+ *
+ *   1. ilre_recall_shard_stats: for this shard's keys, per query row r = i * n_q_heads + h,
+ *      stats_out_dev[r] = (max_t x_rt, sum_t 2^(x_rt - max)) with x = log2(e) q.k / sqrt(128),
+ *      fp32 pairs [q_len * n_q_heads][2].
+ *      -> all-gather into stats_all_dev [n_shards][q_len * n_q_heads][2] (any shard order).
+ *   2. ilre_recall_shard_scores: A^C (Eq. 5) of this shard's positions under the softmax over
+ *      all shards' keys: scores_out_dev fp32 [L_shard].  Also publishes the global per-row lse
+ *      (ilre_recall_copy_row_lse).
+ *      -> all-gather into scores [L] in position order.
+ *   3. ilre_recall_allocate: Algorithm 1 on given scores (fp32 [L], finite and >= 0; read
+ *      only): out_idx_dev int32 [n_sink + budget] ascending.  Every rank may run it (the result
+ *      is the same everywhere) or one rank may and broadcast the indices.
+ *
+ * With one shard the three calls give exactly what ilre_recall_run gives.  With several, the
+ * scores differ from the unsharded run only in the rounding order of the softmax denominator
+ * (a few fp32 ulps).  L_shard, q_len, budget, spec: as for ilre_recall_run, against the
+ * handle's capacities.  Asynchronous on cuda_stream; workspace rule as for ilre_recall_run.
+ */
+int ilre_recall_shard_stats(ilre_recall_t* h, const void* k_shard_dev, int64_t L_shard,
+                            const void* query_dev, int32_t q_len, float* stats_out_dev,
+                            void* cuda_stream);
+int ilre_recall_shard_scores(ilre_recall_t* h, const void* k_shard_dev, int64_t L_shard,
+                             const void* query_dev, int32_t q_len, const float* stats_all_dev,
+                             int32_t n_shards, float* scores_out_dev, void* cuda_stream);
+int ilre_recall_allocate(ilre_recall_t* h, const float* scores_dev, int64_t L, int32_t budget,
+                         const ilre_pool_spec_t* spec, int32_t* out_idx_dev, void* cuda_stream);
+
+/*
  * Streaming chunked prefill attention of one chunk in a layer before the retrieval layer
  * (Section 3.1, Eq. 2 with the Lambda-shaped mask; Section 3.3: "only cache the sink and sliding
  * part of the key states and value states"):

@@ -142,9 +142,13 @@ bool encode_2d(EncodeTiledFn fn, CUtensorMap* map, const void* base, uint64_t in
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// with_qk: the call reads a key cache and a query; with_select: it runs Algorithm 1.
 int validate_run(const ilre_recall* h, const void* k, long long L, const void* q, int q_len,
-                 int budget, const ilre_pool_spec_t* spec, const void* out_idx) {
-  if (!h || !k || !q || !spec || !out_idx) return ILRE_ERR_INVALID_ARG;
+                 int budget, const ilre_pool_spec_t* spec, const void* out_idx, bool with_qk,
+                 bool with_select) {
+  if (!h || !spec) return ILRE_ERR_INVALID_ARG;
+  if (with_qk && (!k || !q)) return ILRE_ERR_INVALID_ARG;
+  if (with_select && !out_idx) return ILRE_ERR_INVALID_ARG;
   if (L < 1 || q_len < 1 || budget < 0) return ILRE_ERR_INVALID_ARG;
   if (spec->n_max < 1 || spec->n_win < 1 || !spec->max_sizes || !spec->win_sizes)
     return ILRE_ERR_INVALID_ARG;
@@ -163,7 +167,7 @@ int validate_run(const ilre_recall* h, const void* k, long long L, const void* q
       n_comb > h->cfg.max_combinations)
     return ILRE_ERR_CAPACITY;
   if (spec->n_sink > L || budget > L - spec->n_sink) return ILRE_ERR_BUDGET;
-  if ((reinterpret_cast<uintptr_t>(k) & 15u) || (reinterpret_cast<uintptr_t>(q) & 15u))
+  if (with_qk && ((reinterpret_cast<uintptr_t>(k) & 15u) || (reinterpret_cast<uintptr_t>(q) & 15u)))
     return ILRE_ERR_ALIGNMENT;
   return ILRE_OK;
 }
@@ -265,10 +269,35 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out) {
   return ILRE_OK;
 }
 
-int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const void* query_dev,
-                    int32_t q_len, int32_t budget, const ilre_pool_spec_t* spec,
-                    int32_t* out_idx_dev, float* out_scores_dev, void* cuda_stream) {
-  const int v = validate_run(h, k_cache_dev, L, query_dev, q_len, budget, spec, out_idx_dev);
+}  // extern "C"
+
+namespace {
+
+enum : int { kStageStats = 1, kStageScores = 2, kStageSelect = 4 };
+
+// What one call computes: any of the three stages of the recall, with the hand-over points of
+// a key-range sharded run (statistics out / in, scores out / in).
+struct RunIo {
+  int stages;
+  float2* stats_out;            // kStageStats alone: per-row (max in log2 units, sum) of this shard
+  const float2* ext_stats;      // kStageScores alone: the shards' statistics [n_ext][q_len * n_q]
+  int n_ext;
+  float* shard_scores_out;      // kStageScores alone: A^C of this shard's positions
+  const float* scores_in;       // kStageSelect alone: A^C of the whole context
+};
+
+int recall_impl(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const void* query_dev,
+                int32_t q_len, int32_t budget, const ilre_pool_spec_t* spec,
+                int32_t* out_idx_dev, float* out_scores_dev, void* cuda_stream, const RunIo& io) {
+  static const int32_t kOne = 1;
+  static const ilre_pool_spec_t kNoPooling = {1, &kOne, 1, &kOne, 0, 0, 0};
+  const bool with_qk = (io.stages & (kStageStats | kStageScores)) != 0;
+  const bool with_select = (io.stages & kStageSelect) != 0;
+  if (!h) return ILRE_ERR_INVALID_ARG;
+  if (!with_select) { spec = &kNoPooling; budget = 0; }
+  if (!with_qk) q_len = 1;
+  const int v = validate_run(h, k_cache_dev, L, query_dev, q_len, budget, spec, out_idx_dev,
+                             with_qk, with_select);
   if (v != ILRE_OK) return v;
   DeviceGuard guard(h->cfg.device);
   if (!guard.ok) return ILRE_ERR_CUDA;
@@ -321,10 +350,12 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
     }
 
   CUtensorMap map_k, map_q;
-  if (!encode_2d(h->encode, &map_k, k_cache_dev, static_cast<uint64_t>(h->cfg.n_kv_heads) * 128,
-                 static_cast<uint64_t>(L), static_cast<uint64_t>(h->cfg.n_kv_heads) * 256))
-    return ILRE_ERR_CUDA;
-  if (!encode_2d(h->encode, &map_q, h->qp, 128, static_cast<uint64_t>(g.n_groups) * g.rb_rows, 256))
+  std::memset(&map_k, 0, sizeof(map_k));
+  std::memset(&map_q, 0, sizeof(map_q));
+  if (with_qk &&
+      (!encode_2d(h->encode, &map_k, k_cache_dev, static_cast<uint64_t>(h->cfg.n_kv_heads) * 128,
+                  static_cast<uint64_t>(L), static_cast<uint64_t>(h->cfg.n_kv_heads) * 256) ||
+       !encode_2d(h->encode, &map_q, h->qp, 128, static_cast<uint64_t>(g.n_groups) * g.rb_rows, 256)))
     return ILRE_ERR_CUDA;
 
   QkParams qk;
@@ -379,14 +410,25 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
   cudaEvent_t* ev = h->ev[h->prof_runs % kProfRing];
 #define ILRE_MARK(i) do { if (prof) ILRE_CUDA(cudaEventRecord(ev[i], st)); } while (0)
 
+  if (!with_qk) pp.n_rb = 0;                             // no query to pack
+  mp.ext_stats = io.ext_stats; mp.n_ext = io.n_ext;
+  if (io.scores_in) { sp.scores = const_cast<float*>(io.scores_in); sp.scores_given = 1; }
   ILRE_MARK(0);
   ILRE_CUDA(launch_prepare(query_dev, h->qp, pp, h->n_sm, st)); ++launches;
   ILRE_MARK(1);
-  ILRE_CUDA(launch_row_stats(map_k, map_q, qk, st)); ++launches;
+  if (io.stages & kStageStats) {
+    ILRE_CUDA(launch_row_stats(map_k, map_q, qk, st)); ++launches;
+    if (io.stats_out) { ILRE_CUDA(launch_export_stats(mp, io.stats_out, st)); ++launches; }
+  }
   ILRE_MARK(2);
-  ILRE_CUDA(launch_scores(map_k, map_q, qk, mp, st)); ++launches;
+  if (io.stages & kStageScores) {
+    ILRE_CUDA(launch_scores(map_k, map_q, qk, mp, st)); ++launches;
+    if (io.shard_scores_out) {
+      ILRE_CUDA(launch_decode_scores(h->enc, io.shard_scores_out, L, st)); ++launches;
+    }
+  }
   ILRE_MARK(3);
-  ILRE_CUDA(launch_select(tbl, sp, select_grid, select_smem, st)); ++launches;
+  if (with_select) { ILRE_CUDA(launch_select(tbl, sp, select_grid, select_smem, st)); ++launches; }
   ILRE_MARK(4);
 #undef ILRE_MARK
   h->last_launches = launches;
@@ -394,12 +436,51 @@ int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const 
   return ILRE_OK;
 }
 
+}  // namespace
+
+extern "C" {
+
+int ilre_recall_run(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const void* query_dev,
+                    int32_t q_len, int32_t budget, const ilre_pool_spec_t* spec,
+                    int32_t* out_idx_dev, float* out_scores_dev, void* cuda_stream) {
+  const RunIo io = {kStageStats | kStageScores | kStageSelect, nullptr, nullptr, 0, nullptr, nullptr};
+  return recall_impl(h, k_cache_dev, L, query_dev, q_len, budget, spec, out_idx_dev, out_scores_dev,
+                     cuda_stream, io);
+}
+
+int ilre_recall_shard_stats(ilre_recall_t* h, const void* k_shard_dev, int64_t L_shard,
+                            const void* query_dev, int32_t q_len, float* stats_out_dev,
+                            void* cuda_stream) {
+  if (!stats_out_dev) return ILRE_ERR_INVALID_ARG;
+  const RunIo io = {kStageStats, reinterpret_cast<float2*>(stats_out_dev), nullptr, 0, nullptr, nullptr};
+  return recall_impl(h, k_shard_dev, L_shard, query_dev, q_len, 0, nullptr, nullptr, nullptr,
+                     cuda_stream, io);
+}
+
+int ilre_recall_shard_scores(ilre_recall_t* h, const void* k_shard_dev, int64_t L_shard,
+                             const void* query_dev, int32_t q_len, const float* stats_all_dev,
+                             int32_t n_shards, float* scores_out_dev, void* cuda_stream) {
+  if (!stats_all_dev || n_shards < 1 || !scores_out_dev) return ILRE_ERR_INVALID_ARG;
+  const RunIo io = {kStageScores, nullptr, reinterpret_cast<const float2*>(stats_all_dev), n_shards,
+                    scores_out_dev, nullptr};
+  return recall_impl(h, k_shard_dev, L_shard, query_dev, q_len, 0, nullptr, nullptr, nullptr,
+                     cuda_stream, io);
+}
+
+int ilre_recall_allocate(ilre_recall_t* h, const float* scores_dev, int64_t L, int32_t budget,
+                         const ilre_pool_spec_t* spec, int32_t* out_idx_dev, void* cuda_stream) {
+  if (!scores_dev) return ILRE_ERR_INVALID_ARG;
+  const RunIo io = {kStageSelect, nullptr, nullptr, 0, nullptr, scores_dev};
+  return recall_impl(h, nullptr, L, nullptr, 1, budget, spec, out_idx_dev, nullptr, cuda_stream, io);
+}
+
 int ilre_recall_run_host(ilre_recall_t* h, const void* k_cache_host, int64_t L,
                          const void* query_host, int32_t q_len, int32_t budget,
                          const ilre_pool_spec_t* spec, int32_t* out_idx_host,
                          float* out_scores_host, void* cuda_stream) {
   if (!h || !h->stage_k) return ILRE_ERR_INVALID_ARG;
-  const int v = validate_run(h, k_cache_host, L, query_host, q_len, budget, spec, out_idx_host);
+  const int v = validate_run(h, k_cache_host, L, query_host, q_len, budget, spec, out_idx_host,
+                             true, true);
   if (v != ILRE_OK && v != ILRE_ERR_ALIGNMENT) return v;
   if (spec->n_sink > kMaxSinkStaging) return ILRE_ERR_CAPACITY;
   DeviceGuard guard(h->cfg.device);

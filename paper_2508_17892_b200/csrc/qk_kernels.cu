@@ -293,28 +293,62 @@ row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
   cta_teardown(tmem_base);
 }
 
-// Combines the per-key-chunk partial statistics of one row into -lse (log2 units; -inf marks
-// a padding row); `publish` also stores the user-visible natural-log lse.
-__device__ __forceinline__ float merged_neg_lse2(const MergeParams& p, int group, int within,
-                                                 bool publish) {
+// Combines the partial statistics of one row (per key chunk of this launch, or per key shard)
+// into (max in log2 units, sum); -lse in log2 units for the scores pass (-inf marks a padding
+// row); `publish` also stores the user-visible natural-log lse.
+__device__ __forceinline__ float2 merged_stats(const MergeParams& p, int group, int within,
+                                               int* user_row) {
   const int g = group / p.n_rb, rb = group % p.n_rb;
   const int rg = rb * p.rb_rows + within;
-  if (rg >= p.group_size * p.q_len) return -INFINITY;
-  const float2* part = reinterpret_cast<const float2*>(p.partial) +
-                       static_cast<size_t>(group) * p.cpg * p.rb_rows + within;
+  *user_row = -1;
+  if (rg >= p.group_size * p.q_len) return make_float2(-INFINITY, 0.f);
+  const int i = rg / p.group_size, j = rg % p.group_size;
+  *user_row = i * p.n_q + g * p.group_size + j;
+  const float2* part;
+  size_t stride;
+  int n;
+  if (p.n_ext > 0) {                     // one entry per key shard
+    part = p.ext_stats + *user_row;
+    stride = static_cast<size_t>(p.q_len) * p.n_q;
+    n = p.n_ext;
+  } else {                               // one entry per key chunk of this launch
+    part = reinterpret_cast<const float2*>(p.partial) +
+           static_cast<size_t>(group) * p.cpg * p.rb_rows + within;
+    stride = p.rb_rows;
+    n = p.cpg;
+  }
   float mm = -INFINITY;
-  for (int c = 0; c < p.cpg; ++c) mm = fmaxf(mm, __ldcg(&part[static_cast<size_t>(c) * p.rb_rows]).x);
+  for (int c = 0; c < n; ++c) mm = fmaxf(mm, __ldcg(&part[c * stride]).x);
   float zz = 0.f;
-  for (int c = 0; c < p.cpg; ++c) {
-    const float2 v = __ldcg(&part[static_cast<size_t>(c) * p.rb_rows]);
+  for (int c = 0; c < n; ++c) {
+    const float2 v = __ldcg(&part[c * stride]);
     zz += v.y * exp2f(v.x - mm);
   }
-  const float lse2 = mm + log2f(zz);
-  if (publish) {
-    const int i = rg / p.group_size, j = rg % p.group_size;
-    p.row_lse[i * p.n_q + g * p.group_size + j] = lse2 * 0.69314718055994530942f;
-  }
+  return make_float2(mm, zz);
+}
+
+__device__ __forceinline__ float merged_neg_lse2(const MergeParams& p, int group, int within,
+                                                 bool publish) {
+  int user_row;
+  const float2 st = merged_stats(p, group, within, &user_row);
+  if (user_row < 0) return -INFINITY;
+  const float lse2 = st.x + log2f(st.y);
+  if (publish) p.row_lse[user_row] = lse2 * 0.69314718055994530942f;
   return -lse2;
+}
+
+__global__ void export_stats_kernel(MergeParams p, float2* __restrict__ out) {
+  const int prow = blockIdx.x * blockDim.x + threadIdx.x;
+  if (prow >= p.n_groups * p.rb_rows) return;
+  int user_row;
+  const float2 st = merged_stats(p, prow / p.rb_rows, prow % p.rb_rows, &user_row);
+  if (user_row >= 0) out[user_row] = st;
+}
+
+__global__ void decode_scores_kernel(const uint32_t* __restrict__ enc, float* __restrict__ out,
+                                     long long L) {
+  const long long t = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (t < L) out[t] = exp2f(ordered_to_float(enc[t]));
 }
 
 // ---------------------------------------------------------------------------------------
@@ -495,6 +529,17 @@ cudaError_t launch_row_stats(const CUtensorMap& tk, const CUtensorMap& tq, const
     case 4: return launch_row_stats_mt<4>(tk, tq, p, st);
     default: return cudaErrorInvalidValue;
   }
+}
+
+cudaError_t launch_export_stats(const MergeParams& p, float2* out, cudaStream_t st) {
+  const int n = p.n_groups * p.rb_rows;
+  export_stats_kernel<<<(n + 127) / 128, 128, 0, st>>>(p, out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_decode_scores(const uint32_t* enc, float* out, long long L, cudaStream_t st) {
+  decode_scores_kernel<<<static_cast<unsigned>((L + 255) / 256), 256, 0, st>>>(enc, out, L);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_scores(const CUtensorMap& tk, const CUtensorMap& tq, const QkParams& p,

@@ -63,6 +63,11 @@ struct MergeParams {
   int n_groups, n_rb, rb_rows, cpg, group_size, q_len, n_q;
   const float* partial;
   float* row_lse;    // [q_len][n_q] natural-log lse
+  // Key-range sharding: when n_ext > 0 the statistics come from ext_stats
+  // [n_ext][q_len * n_q] (max in log2 units, sum) -- one entry per shard, rows in the
+  // caller's order i * n_q + h -- instead of this launch's own partials.
+  const float2* ext_stats;
+  int n_ext;
 };
 
 size_t row_stats_smem_bytes(int rb_rows, int stages);
@@ -71,6 +76,11 @@ size_t scores_smem_bytes(int rb_rows, int stages);
 cudaError_t launch_prepare(const void* q, void* qp, const PrepParams& p, int n_sm, cudaStream_t st);
 cudaError_t launch_row_stats(const CUtensorMap& tk, const CUtensorMap& tq, const QkParams& p,
                              cudaStream_t st);
+// (max in log2 units, sum of exponentials) of every query row over the keys of this launch,
+// rows in the caller's order i * n_q + h.
+cudaError_t launch_export_stats(const MergeParams& p, float2* out, cudaStream_t st);
+// out[t] = exp2 of the encoded maxima (the scores of Eq. 5 for a key shard)
+cudaError_t launch_decode_scores(const uint32_t* enc, float* out, long long L, cudaStream_t st);
 cudaError_t launch_scores(const CUtensorMap& tk, const CUtensorMap& tq, const QkParams& p,
                           const MergeParams& mp, cudaStream_t st);
 

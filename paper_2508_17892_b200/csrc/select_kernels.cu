@@ -538,7 +538,7 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
 #endif
 
   // ---- A: scores from the encoded maxima, one exp per position ----
-  {
+  if (!p.scores_given) {
     const long long stride = static_cast<long long>(gridDim.x) * kSelThreads;
     for (long long t = static_cast<long long>(blockIdx.x) * kSelThreads + threadIdx.x; t < p.L;
          t += stride) {

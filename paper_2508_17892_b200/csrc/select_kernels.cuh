@@ -41,6 +41,7 @@ struct SelectParams {
   const uint32_t* enc;     // [L] order-preserving uint of max_r log2 p_rt (scores pass output)
   float* scores;           // A^C [L]
   float* user_scores;      // optional copy of A^C for the caller, or null
+  int scores_given;        // 1: `scores` already holds A^C (phase A is skipped)
   long long L;
   int n_sink;
   int win_op;              // 0 average, 1 max

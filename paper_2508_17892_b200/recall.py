@@ -19,6 +19,7 @@ STAGE_NAMES = ("prepare", "row_stats", "scores", "select")
 
 EXPORTED_SYMBOLS = (
     "ilre_recall_create", "ilre_recall_run", "ilre_recall_run_host", "ilre_recall_fill_keys",
+    "ilre_recall_shard_stats", "ilre_recall_shard_scores", "ilre_recall_allocate",
     "ilre_recall_chunk_attention", "ilre_recall_rerope_keys", "ilre_gather_input_ids",
     "ilre_recall_copy_row_lse",
     "ilre_recall_status", "ilre_recall_set_profiling", "ilre_recall_stage_times",
@@ -66,6 +67,9 @@ def load_library() -> ctypes.CDLL:
     lib.ilre_recall_create.argtypes = [ctypes.POINTER(IlreConfig), ctypes.POINTER(vp)]
     lib.ilre_recall_run.argtypes = [vp, vp, i64, vp, i32, i32, ctypes.POINTER(IlrePoolSpec), vp, vp, vp]
     lib.ilre_recall_run_host.argtypes = lib.ilre_recall_run.argtypes
+    lib.ilre_recall_shard_stats.argtypes = [vp, vp, i64, vp, i32, vp, vp]
+    lib.ilre_recall_shard_scores.argtypes = [vp, vp, i64, vp, i32, vp, i32, vp, vp]
+    lib.ilre_recall_allocate.argtypes = [vp, vp, i64, i32, ctypes.POINTER(IlrePoolSpec), vp, vp]
     lib.ilre_recall_chunk_attention.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp]
     lib.ilre_recall_fill_keys.argtypes = [vp, vp, i64, i32, vp, vp, i64, ctypes.c_double, vp, i64, vp]
     lib.ilre_recall_rerope_keys.argtypes = [vp, vp, vp, i64, i32, i32, ctypes.c_double, vp]
@@ -180,6 +184,76 @@ class IlreRecall:
         if rc != 0:
             raise IlreError(rc, "ilre_recall_run")
         return out_idx, out_scores
+
+    # -- key-range sharded recall: the per-rank steps -----------------------------------
+    def _check_kq(self, K: torch.Tensor, Q: torch.Tensor):
+        assert K.is_cuda and Q.is_cuda and K.dtype == torch.bfloat16 and Q.dtype == torch.bfloat16
+        assert K.is_contiguous() and Q.is_contiguous()
+        assert K.shape[1:] == (self.cfg.n_kv_heads, self.cfg.head_dim)
+        assert Q.shape[1:] == (self.cfg.n_q_heads, self.cfg.head_dim)
+
+    def shard_stats(self, K_shard: torch.Tensor, Q: torch.Tensor,
+                    out: Optional[torch.Tensor] = None,
+                    stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        """(max in log2 units, sum of exponentials) of every query row over this shard's keys:
+        fp32 [q_len * n_q_heads, 2], to be all-gathered over the shards."""
+        self._check_kq(K_shard, Q)
+        n_rows = Q.shape[0] * self.cfg.n_q_heads
+        if out is None:
+            out = torch.empty(n_rows, 2, dtype=torch.float32, device=K_shard.device)
+        assert out.is_cuda and out.dtype == torch.float32 and out.is_contiguous()
+        assert out.numel() == 2 * n_rows
+        st = stream if stream is not None else torch.cuda.current_stream(K_shard.device)
+        with torch.cuda.device(K_shard.device):
+            rc = self._lib.ilre_recall_shard_stats(self._h, K_shard.data_ptr(), K_shard.shape[0],
+                                                   Q.data_ptr(), Q.shape[0], out.data_ptr(),
+                                                   st.cuda_stream)
+        if rc != 0:
+            raise IlreError(rc, "ilre_recall_shard_stats")
+        return out
+
+    def shard_scores(self, K_shard: torch.Tensor, Q: torch.Tensor, stats_all: torch.Tensor,
+                     out: Optional[torch.Tensor] = None,
+                     stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        """A^C of this shard's positions given every shard's statistics
+        (fp32 [n_shards, q_len * n_q_heads, 2]); fp32 [L_shard], to be all-gathered in
+        position order."""
+        self._check_kq(K_shard, Q)
+        n_rows = Q.shape[0] * self.cfg.n_q_heads
+        assert stats_all.is_cuda and stats_all.dtype == torch.float32 and stats_all.is_contiguous()
+        assert stats_all.dim() == 3 and stats_all.shape[1:] == (n_rows, 2)
+        if out is None:
+            out = torch.empty(K_shard.shape[0], dtype=torch.float32, device=K_shard.device)
+        assert out.is_cuda and out.dtype == torch.float32 and out.is_contiguous()
+        assert out.numel() == K_shard.shape[0]
+        st = stream if stream is not None else torch.cuda.current_stream(K_shard.device)
+        with torch.cuda.device(K_shard.device):
+            rc = self._lib.ilre_recall_shard_scores(self._h, K_shard.data_ptr(), K_shard.shape[0],
+                                                    Q.data_ptr(), Q.shape[0], stats_all.data_ptr(),
+                                                    stats_all.shape[0], out.data_ptr(),
+                                                    st.cuda_stream)
+        if rc != 0:
+            raise IlreError(rc, "ilre_recall_shard_scores")
+        return out
+
+    def allocate(self, scores: torch.Tensor, budget: int, max_sizes: Sequence[int],
+                 win_sizes: Sequence[int], win_op: int = 0, n_sink: int = 0,
+                 out_idx: Optional[torch.Tensor] = None,
+                 stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        """Algorithm 1 on given scores (fp32 [L], finite, >= 0): ascending int32 indices."""
+        assert scores.is_cuda and scores.dtype == torch.float32 and scores.is_contiguous()
+        assert scores.dim() == 1
+        if out_idx is None:
+            out_idx = torch.empty(n_sink + budget, dtype=torch.int32, device=scores.device)
+        spec, _keep = _spec(max_sizes, win_sizes, win_op, n_sink)
+        st = stream if stream is not None else torch.cuda.current_stream(scores.device)
+        with torch.cuda.device(scores.device):
+            rc = self._lib.ilre_recall_allocate(self._h, scores.data_ptr(), scores.numel(), budget,
+                                                ctypes.byref(spec), out_idx.data_ptr(),
+                                                st.cuda_stream)
+        if rc != 0:
+            raise IlreError(rc, "ilre_recall_allocate")
+        return out_idx
 
     def run_host(self, K: torch.Tensor, Q: torch.Tensor, budget: int, max_sizes: Sequence[int],
                  win_sizes: Sequence[int], win_op: int = 0, n_sink: int = 0,
