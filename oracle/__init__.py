@@ -247,3 +247,28 @@ def chunk_attention(Q, K, V, n_prefix: int) -> np.ndarray:
             p /= p.sum()
             out[j, h, :] = p @ v[: n_prefix + j + 1, g, :]
     return out
+
+
+def span_hits(idx: Sequence[int], spans: Sequence[Sequence[int]]) -> np.ndarray:
+    """How many positions of every planted key phrase (begin, length) the recalled index list
+    contains (retrieval task of Appendix A.1).  Plain set membership, position by position."""
+    have = set(int(i) for i in idx)
+    return np.array([sum(1 for p in range(int(b), int(b) + int(n)) if p in have)
+                     for b, n in spans], dtype=np.int64)
+
+
+def layer_choice(idx_per_layer: Sequence[Sequence[int]], spans: Sequence[Sequence[int]]):
+    """Offline choice of the retrieval layer (Section 3.3, first paragraph; Appendix A.1).
+
+    A phrase counts as retrieved only if every one of its positions was recalled (exact match);
+    a layer's recall rate is the fraction of phrases retrieved; l_R is the layer with the
+    smallest index among those with the highest recall rate.  Returns
+    (hits [n_layers, n_spans], retrieved phrases per layer [n_layers], l_R)."""
+    lens = np.array([int(n) for _, n in spans], dtype=np.int64)
+    hits = np.stack([span_hits(idx, spans) for idx in idx_per_layer]) if len(spans) else \
+        np.zeros((len(idx_per_layer), 0), dtype=np.int64)
+    full = (hits == lens[None, :]).sum(axis=1)
+    rates = [f / max(len(spans), 1) for f in full]
+    best = max(rates)
+    l_r = next(l for l, r in enumerate(rates) if r == best)
+    return hits, full, l_r
