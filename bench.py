@@ -17,6 +17,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import subprocess
 import sys
@@ -401,6 +402,55 @@ def run_ours(args, world, rank, local):
                      note="one GPU, first shard; all-gathers not included")
         eng.check_status()
 
+    # Offline retrieval-layer sweep: the same recall against the caches of several candidate
+    # layers of one context, then the exact-match layer choice.  Keys and queries drawn on
+    # the device, phrases planted along each layer's mean query direction.
+    sweep = None
+    if args.sweep_layers > 0 and rank == 0:
+        from paper_2508_17892_b200 import layer_recall
+        gen = torch.Generator(device=dev).manual_seed(777)
+        Ls, qs, n_lay, n_ph, ph_len = min(w.L, 131072), min(w.q_len, 64), args.sweep_layers, 20, 32
+        seg = Ls // n_ph
+        sb = torch.arange(n_ph, dtype=torch.int32, device=dev) * seg + seg // 3
+        sl = torch.full((n_ph,), ph_len, dtype=torch.int32, device=dev)
+        Kl, Ql = [], []
+        for l in range(n_lay):
+            q = torch.randn(qs, w.n_q_heads, w.d, generator=gen, device=dev).to(torch.bfloat16)
+            k = torch.randn(Ls, w.n_kv_heads, w.d, generator=gen, device=dev)
+            u = q.float().view(qs, w.n_kv_heads, -1, w.d).mean(dim=(0, 2))
+            u = u / u.norm(dim=-1, keepdim=True)
+            gain = 0.4 + 2.6 * l / max(n_lay - 1, 1)
+            for b in sb.tolist():
+                k[b:b + ph_len] = gain * math.sqrt(w.d) * u[None] + 0.5 * k[b:b + ph_len]
+            Kl.append(k.to(torch.bfloat16))
+            Ql.append(q)
+            del k
+        idx_all = torch.empty(n_lay, w.n_sink + 1024, dtype=torch.int32, device=dev)
+        sspec = (1024, w.max_sizes, w.win_sizes, w.win_op, w.n_sink)
+
+        def one_sweep():
+            for l in range(n_lay):
+                eng.run(Kl[l], Ql[l], *sspec, out_idx=idx_all[l])
+            return layer_recall(idx_all, sb, sl)
+
+        for _ in range(3):
+            one_sweep()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 20
+        torch.cuda.synchronize()
+        s0.record()
+        for _ in range(reps):
+            _, full, layer = one_sweep()
+        s1.record()
+        torch.cuda.synchronize()
+        ms = s0.elapsed_time(s1) / reps
+        swept = float(n_lay) * Ls * w.n_kv_heads * w.d * 2
+        sweep = dict(layers=n_lay, L=Ls, q_len=qs, budget=1024, phrases=n_ph, ms=ms,
+                     ms_per_layer=ms / n_lay, key_cache_gbs=swept / (ms * 1e-3) / 1e9,
+                     retrieved_per_layer=full.tolist(), chosen_layer=int(layer.item()))
+        eng.check_status()
+        del Kl, Ql
+
     elapsed_max, units = aggregate(elapsed_ms, float(k_bytes) * args.steps, dev)
     if rank != 0:
         return
@@ -452,7 +502,7 @@ def run_ours(args, world, rank, local):
                 clocks=clocks, e2e=e2e, gpu_launches=launches, roofline=roofline,
                 cpu_baseline=cpu_baseline,
                 stages_ms=stages, dca_rerope=dca, key_fill=fill, chunk_attention=attn,
-                sharded_steps=shard,
+                sharded_steps=shard, layer_sweep=sweep,
                 whole_step=dict(hbm_frac_one_read_of_K=step_hbm_frac,
                                 tensor_frac_one_qk=step_tensor_frac,
                                 hbm_frac_of_8TBps=(k_bytes / (ms_per_step * 1e-3) / 1e9) / 8000.0))
@@ -479,6 +529,9 @@ def main():
                     help="also time the key-cache fill over this many tokens (0 = skip)")
     ap.add_argument("--shards", type=int, default=8,
                     help="also time the per-rank steps of a key-range split this many ways (0 = skip)")
+    ap.add_argument("--sweep-layers", type=int, default=8,
+                    help="also time the offline retrieval-layer sweep over this many candidate "
+                         "layers at L = 128K (0 = skip)")
     ap.add_argument("--cpu-sample-keys", type=int, default=131072)
     ap.add_argument("--ref-sample-keys", type=int, default=4096)
     args = ap.parse_args()

@@ -213,6 +213,27 @@ int ilre_gather_input_ids(const int32_t* input_ids_dev, int64_t L, const int32_t
                           int32_t* out_ids_dev, void* cuda_stream);
 
 /*
+ * Offline choice of the retrieval layer l_R (Section 3.3, first paragraph, with the retrieval
+ * task of Appendix A.1): the recall is run once per candidate layer on a context with planted
+ * key phrases; a phrase counts as retrieved only if every one of its positions was recalled
+ * (exact match); a layer's recall rate is its share of retrieved phrases; l_R is the layer
+ * with the smallest index among those with the highest rate.
+ *   idx_dev         int32 [n_layers][n_idx]: each layer's recalled positions, ascending,
+ *                   without repeats (ilre_recall_run's output, one row per layer)
+ *   span_begin_dev  int32 [n_spans]: first position of each phrase
+ *   span_len_dev    int32 [n_spans]: its length, >= 1
+ *   hits_out_dev    int32 [n_layers][n_spans]: recalled positions inside each phrase (NULL to skip)
+ *   full_out_dev    int32 [n_layers]: phrases retrieved completely (rate = this / n_spans)
+ *   layer_out_dev   int32 [1]: the chosen layer's row index
+ * All pointers on the current device.  n_layers <= 1024 (ILRE_ERR_CAPACITY beyond).  No handle;
+ * asynchronous on cuda_stream.
+ */
+int ilre_layer_recall(const int32_t* idx_dev, int32_t n_layers, int32_t n_idx,
+                      const int32_t* span_begin_dev, const int32_t* span_len_dev, int32_t n_spans,
+                      int32_t* hits_out_dev, int32_t* full_out_dev, int32_t* layer_out_dev,
+                      void* cuda_stream);
+
+/*
  * Row statistics of the last run (Eq. 4's softmax denominator): copies
  * lse[i * n_q_heads + h] = log(sum_t exp(s[h,i,t])) (natural log, fp32) for the q_len rows
  * of that run into out_lse_dev, asynchronously on cuda_stream.

@@ -11,7 +11,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ_DIR = os.path.join(HERE, "_build")
 LIB_PATH = os.path.join(HERE, "libilre_recall.so")
 SOURCES = ["ilre_api.cu", "qk_kernels.cu", "select_kernels.cu", "rerope_kernels.cu", "fill_kernels.cu",
-           "attn_kernels.cu",
+           "attn_kernels.cu", "sweep_kernels.cu",
            "topk_noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]

@@ -13,6 +13,7 @@
 #include "fill_kernels.cuh"
 #include "qk_kernels.cuh"
 #include "rerope_kernels.cuh"
+#include "sweep_kernels.cuh"
 #include "select_kernels.cuh"
 #include "sm100_ptx.cuh"
 
@@ -624,6 +625,20 @@ int ilre_gather_input_ids(const int32_t* input_ids_dev, int64_t L, const int32_t
     return ILRE_ERR_INVALID_ARG;
   ILRE_CUDA(launch_gather_ids(input_ids_dev, L, idx_dev, n_idx, query_ids_dev, n_query, out_ids_dev,
                               static_cast<cudaStream_t>(cuda_stream)));
+  return ILRE_OK;
+}
+
+int ilre_layer_recall(const int32_t* idx_dev, int32_t n_layers, int32_t n_idx,
+                      const int32_t* span_begin_dev, const int32_t* span_len_dev, int32_t n_spans,
+                      int32_t* hits_out_dev, int32_t* full_out_dev, int32_t* layer_out_dev,
+                      void* cuda_stream) {
+  if (n_layers < 1 || n_idx < 0 || n_spans < 0 || !full_out_dev || !layer_out_dev ||
+      (n_idx > 0 && !idx_dev) || (n_spans > 0 && (!span_begin_dev || !span_len_dev)))
+    return ILRE_ERR_INVALID_ARG;
+  if (n_layers > kMaxSweepLayers) return ILRE_ERR_CAPACITY;
+  ILRE_CUDA(launch_layer_recall(idx_dev, n_layers, n_idx, span_begin_dev, span_len_dev, n_spans,
+                                hits_out_dev, full_out_dev, layer_out_dev,
+                                static_cast<cudaStream_t>(cuda_stream)));
   return ILRE_OK;
 }
 

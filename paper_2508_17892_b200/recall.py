@@ -21,6 +21,7 @@ EXPORTED_SYMBOLS = (
     "ilre_recall_create", "ilre_recall_run", "ilre_recall_run_host", "ilre_recall_fill_keys",
     "ilre_recall_shard_stats", "ilre_recall_shard_scores", "ilre_recall_allocate",
     "ilre_recall_chunk_attention", "ilre_recall_rerope_keys", "ilre_gather_input_ids",
+    "ilre_layer_recall",
     "ilre_recall_copy_row_lse",
     "ilre_recall_status", "ilre_recall_set_profiling", "ilre_recall_stage_times",
     "ilre_recall_last_launch_count", "ilre_recall_destroy", "ilre_strerror",
@@ -74,6 +75,7 @@ def load_library() -> ctypes.CDLL:
     lib.ilre_recall_fill_keys.argtypes = [vp, vp, i64, i32, vp, vp, i64, ctypes.c_double, vp, i64, vp]
     lib.ilre_recall_rerope_keys.argtypes = [vp, vp, vp, i64, i32, i32, ctypes.c_double, vp]
     lib.ilre_gather_input_ids.argtypes = [vp, i64, vp, i32, vp, i32, vp, vp]
+    lib.ilre_layer_recall.argtypes = [vp, i32, i32, vp, vp, i32, vp, vp, vp, vp]
     lib.ilre_recall_copy_row_lse.argtypes = [vp, vp, i32, vp]
     lib.ilre_recall_status.argtypes = [vp]
     lib.ilre_recall_set_profiling.argtypes = [vp, i32]
@@ -115,6 +117,31 @@ def gather_input_ids(input_ids: torch.Tensor, idx: torch.Tensor, query_ids: torc
     if rc != 0:
         raise IlreError(rc, "ilre_gather_input_ids")
     return out
+
+
+def layer_recall(idx: torch.Tensor, span_begin: torch.Tensor, span_len: torch.Tensor,
+                 stream: Optional[torch.cuda.Stream] = None):
+    """Offline retrieval-layer choice from the recalled lists of the candidate layers.
+
+    idx: int32 [n_layers, n_idx] (ascending rows); span_begin / span_len: int32 [n_spans], the
+    planted key phrases.  Returns (hits int32 [n_layers, n_spans], phrases retrieved completely
+    int32 [n_layers], chosen layer int32 [1]) on the device."""
+    for t in (idx, span_begin, span_len):
+        assert t.is_cuda and t.dtype == torch.int32 and t.is_contiguous()
+    assert idx.dim() == 2 and span_begin.dim() == 1 and span_begin.shape == span_len.shape
+    n_layers, n_idx = idx.shape
+    n_spans = span_begin.numel()
+    hits = torch.empty(n_layers, n_spans, dtype=torch.int32, device=idx.device)
+    full = torch.empty(n_layers, dtype=torch.int32, device=idx.device)
+    layer = torch.empty(1, dtype=torch.int32, device=idx.device)
+    st = stream if stream is not None else torch.cuda.current_stream(idx.device)
+    with torch.cuda.device(idx.device):
+        rc = load_library().ilre_layer_recall(idx.data_ptr(), n_layers, n_idx, span_begin.data_ptr(),
+                                              span_len.data_ptr(), n_spans, hits.data_ptr(),
+                                              full.data_ptr(), layer.data_ptr(), st.cuda_stream)
+    if rc != 0:
+        raise IlreError(rc, "ilre_layer_recall")
+    return hits, full, layer
 
 
 def topk_positions_noalloc(scores: torch.Tensor, k: int,

@@ -3,7 +3,8 @@
 Holds no part of the recall method's arithmetic.
 """
 from .recall_inputs import (CONFIGS, PAPER_DEFAULT_MAX_SIZES, PAPER_DEFAULT_WIN_SIZES,
-                            RecallInputs, RecallWorkload, make_inputs, small_workload)
+                            RecallInputs, RecallWorkload, layer_sweep_workloads, make_inputs,
+                            small_workload)
 
 __all__ = ["CONFIGS", "PAPER_DEFAULT_MAX_SIZES", "PAPER_DEFAULT_WIN_SIZES", "RecallInputs",
-           "RecallWorkload", "make_inputs", "small_workload"]
+           "RecallWorkload", "layer_sweep_workloads", "make_inputs", "small_workload"]

@@ -16,7 +16,8 @@ fixed order; all math in fp32 with one final round-to-nearest-even to bf16):
    recipe: the stream of normal variates depends on it), each block rotated by RoPE
    (rotate-half pairing i <-> i + d/2, inv_freq_i = theta^(-2i/d), theta = 500000, position =
    index in the cache; Eq. 3 of the paper) and rounded to bf16;
-5. needle noise: for every span, every kv head g: key = 3*sqrt(d)*u_g + 0.5*N(0,I), where
+5. needle noise: for every span, every kv head g: key = gain*sqrt(d)*u_g + 0.5*N(0,I)
+   (gain 3 unless the workload says otherwise), where
    u_g is the unit vector along the mean of the 4*q_len bf16 query vectors of group g.  The
    needles overwrite the cache after RoPE (they live in cache space).
 
@@ -52,6 +53,10 @@ class RecallWorkload:
     win_sizes: Tuple[int, ...] = (1,)        # stride-1 window sizes n_j (Algorithm 1)
     win_op: int = 1                          # 0 = average (Algorithm 1), 1 = max
     n_sink: int = 0
+    needle_gain: float = 3.0                 # needle key = gain * sqrt(d) * u_g + noise
+    span_seed: int = -1                      # >= 0: span offsets/lengths from a generator of
+                                             # their own (same spans for workloads that differ
+                                             # in seed, e.g. the layers of one context)
 
 
 @dataclass
@@ -142,8 +147,9 @@ def make_inputs(w: RecallWorkload) -> RecallInputs:
     if w.n_spans > 0:
         seg = L // w.n_spans
         lo, hi = w.span_len
-        u_off = torch.rand(w.n_spans, generator=g, dtype=torch.float64)
-        lens = torch.randint(lo, hi + 1, (w.n_spans,), generator=g)
+        gs = g if w.span_seed < 0 else torch.Generator().manual_seed(w.span_seed)
+        u_off = torch.rand(w.n_spans, generator=gs, dtype=torch.float64)
+        lens = torch.randint(lo, hi + 1, (w.n_spans,), generator=gs)
         for s in range(w.n_spans):
             n = int(lens[s])
             if n > seg:
@@ -176,7 +182,7 @@ def make_inputs(w: RecallWorkload) -> RecallInputs:
         u = mean_dir / mean_dir.norm(dim=-1, keepdim=True)
         for off, n in spans:
             noise = torch.randn(n, H, d, generator=g)
-            K[off:off + n] = (3.0 * math.sqrt(d) * u[None] + 0.5 * noise).to(torch.bfloat16)
+            K[off:off + n] = (w.needle_gain * math.sqrt(d) * u[None] + 0.5 * noise).to(torch.bfloat16)
 
     return RecallInputs(w, K.contiguous(), Q.contiguous(), spans)
 
@@ -191,3 +197,14 @@ def small_workload(L: int, q_len: int, seed: int = 7, n_kv_heads: int = 8, n_q_h
                           n_spans=n_spans, span_len=span_len, budget=budget,
                           max_sizes=tuple(max_sizes), win_sizes=tuple(win_sizes), win_op=win_op,
                           n_sink=n_sink)
+
+
+def layer_sweep_workloads(base: RecallWorkload, gains) -> List[RecallWorkload]:
+    """One workload per candidate layer of the same context: the same planted spans
+    (span_seed), a different query and key cache per layer (seed), and a per-layer needle
+    gain that makes the phrases easier or harder to recall, as layers differ in the paper's
+    retrieval task."""
+    import dataclasses
+    return [dataclasses.replace(base, name=f"{base.name}_layer{l}", seed=base.seed + 1000 * (l + 1),
+                                span_seed=base.seed, needle_gain=float(gain))
+            for l, gain in enumerate(gains)]
