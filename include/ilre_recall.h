@@ -142,8 +142,8 @@ int ilre_recall_allocate(ilre_recall_t* h, const float* scores_dev, int64_t L, i
 
 /*
  * Streaming chunked prefill attention of one chunk in a layer before the retrieval layer
- * (Section 3.1, Eq. 2 with the Lambda-shaped mask; Section 3.3: "only cache the sink and sliding
- * part of the key states and value states"):
+ * (Section 3.1, Eq. 2 with the Lambda-shaped mask; Section 3.3, the step for layers 1..l_R-1,
+ * where only S sink and W sliding-window rows of K and V are kept between chunks):
  *   out[j, h, :] = sum_k softmax_k(q[j, h, :] . k[k, kv(h), :] / sqrt(128)) v[k, kv(h), :],
  *   k = 0 .. n_prefix + j,
  * where the first n_prefix rows of k/v are the cached sink and sliding-window tokens, visible to
@@ -162,8 +162,9 @@ int ilre_recall_chunk_attention(ilre_recall_t* h, const void* q_dev, const void*
                                 void* out_dev, void* cuda_stream);
 
 /*
- * Key-cache fill of the retrieval layer (Section 3.3: "calculate the key states for the context
- * ... fill the cache with chunked key states"; Eq. 1 with the positional encoding of Eq. 3):
+ * Key-cache fill of the retrieval layer (Section 3.3, the step at layer l_R: the context's key
+ * states are computed chunk by chunk into a cache pre-allocated for all L positions; Eq. 1 with
+ * the positional encoding of Eq. 3):
  *   K[pos0 + t, g, :] = R(pos0 + t) (x[t, :] . W_K[g*128 : (g+1)*128, :]^T + b[g*128 : (g+1)*128])
  * for t = 0 .. n_tok-1 and every kv head g, where R(p) is RoPE at position p in the
  * rotate-half layout (pair (c, c + 64) turns by p * rope_theta^(-2c/128)).  One call fills the

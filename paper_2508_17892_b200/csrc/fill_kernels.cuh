@@ -1,5 +1,5 @@
 // Key-cache fill of the retrieval layer: K = PE(X W_K^T + b) written into the cache (Eq. 1 with
-// the RoPE of Eq. 3; Section 3.3, "calculate the key states for the context ... fill the cache").
+// the RoPE of Eq. 3; Section 3.3, the step at the retrieval layer).
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
