@@ -97,7 +97,11 @@ int ilre_recall_run(ilre_recall_t* h,
  * Same computation from HOST buffers (handle created with host_staging != 0): copies the
  * key cache and query to device staging, runs, copies the indices (and scores if asked)
  * back, and synchronises the stream before returning.  For throughput the host buffers
- * should be page-locked.
+ * should be page-locked.  Contexts of 131072 positions or more are uploaded in up to 16 pieces
+ * on an internal stream while the row statistics of the pieces already on the device are
+ * computed; the pieces' statistics are merged as those of key shards are, so the scores may
+ * differ from ilre_recall_run's in the rounding order of the softmax denominator (a few fp32
+ * ulps).
  */
 int ilre_recall_run_host(ilre_recall_t* h,
                          const void* k_cache_host, int64_t L,

@@ -29,6 +29,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 constexpr int kNumStages = 4;            // timed stages (see ilre_recall_stage_times)
 constexpr int kProfRing = 32;            // runs whose stage events are kept for averaging
 constexpr int kMaxSinkStaging = 65536;
+static constexpr int kHostPieces = 16;              // most pieces of a pipelined host upload
+static constexpr long long kHostPieceMinKeys = 65536;   // no piece shorter than this (128-key multiple)
 
 struct Geometry {
   int group_size, n_rb, rb_rows, n_groups, cpg, n_tiles, stages;
@@ -67,6 +69,12 @@ struct ilre_recall {
   void* stage_k;
   void* stage_q;
   int* stage_idx;
+  // pipelined upload of the host entry point: the key cache is copied in pieces on a stream
+  // of its own while the row statistics of the pieces already on the device are computed
+  cudaStream_t copy_stream;
+  cudaEvent_t copy_begin;
+  cudaEvent_t piece_done[kHostPieces];
+  float2* piece_stats;                  // [kHostPieces][max_q_len * n_q_heads]
   // bookkeeping
   cudaEvent_t ev[kProfRing][kNumStages + 1];
   int profiling;
@@ -127,6 +135,11 @@ void free_all(ilre_recall* h) {
   cudaFree(h->tile_ties); cudaFree(h->grid_barrier); cudaFree(h->rope_table); cudaFree(h->pos_lo); cudaFree(h->pos_hi);
   cudaFree(h->cand); cudaFree(h->cand_count); cudaFree(h->ranked); cudaFree(h->bitmap);
   cudaFree(h->status); cudaFree(h->stage_k); cudaFree(h->stage_q); cudaFree(h->stage_idx);
+  cudaFree(h->piece_stats);
+  if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
+  if (h->copy_begin) cudaEventDestroy(h->copy_begin);
+  for (int i = 0; i < kHostPieces; ++i)
+    if (h->piece_done[i]) cudaEventDestroy(h->piece_done[i]);
   for (int r = 0; r < kProfRing; ++r)
     for (int i = 0; i <= kNumStages; ++i)
       if (h->ev[r][i]) cudaEventDestroy(h->ev[r][i]);
@@ -252,6 +265,11 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out) {
     ok = ok && dev_alloc(reinterpret_cast<uint8_t**>(&h->stage_q),
                          static_cast<size_t>(cfg->max_q_len) * cfg->n_q_heads * 256);
     ok = ok && dev_alloc(&h->stage_idx, static_cast<size_t>(cfg->max_budget) + kMaxSinkStaging);
+    ok = ok && dev_alloc(&h->piece_stats, static_cast<size_t>(kHostPieces) * cfg->max_q_len * cfg->n_q_heads);
+    ok = ok && (cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking) == cudaSuccess);
+    ok = ok && (cudaEventCreateWithFlags(&h->copy_begin, cudaEventDisableTiming) == cudaSuccess);
+    for (int i = 0; ok && i < kHostPieces; ++i)
+      ok = (cudaEventCreateWithFlags(&h->piece_done[i], cudaEventDisableTiming) == cudaSuccess);
   }
   for (int r = 0; ok && r < kProfRing; ++r)
     for (int i = 0; ok && i <= kNumStages; ++i)
@@ -489,10 +507,45 @@ int ilre_recall_run_host(ilre_recall_t* h, const void* k_cache_host, int64_t L,
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const size_t k_bytes = static_cast<size_t>(L) * h->cfg.n_kv_heads * 256;
   const size_t q_bytes = static_cast<size_t>(q_len) * h->cfg.n_q_heads * 256;
-  ILRE_CUDA(cudaMemcpyAsync(h->stage_k, k_cache_host, k_bytes, cudaMemcpyHostToDevice, st));
   ILRE_CUDA(cudaMemcpyAsync(h->stage_q, query_host, q_bytes, cudaMemcpyHostToDevice, st));
-  const int rc = ilre_recall_run(h, h->stage_k, L, h->stage_q, q_len, budget, spec, h->stage_idx,
-                                 nullptr, st);
+  // Long contexts: the upload takes ten times longer than the kernels, so the cache goes up in
+  // pieces on the copy stream and the row statistics of every piece (Eq. 4's max and sum over
+  // its keys) are computed as soon as it has landed; what is left after the last piece is its
+  // statistics, the scores pass (which merges the pieces' statistics like those of key
+  // shards) and Algorithm 1.
+  long long piece_keys = ((L + kHostPieces - 1) / kHostPieces + 127) / 128 * 128;
+  if (piece_keys < kHostPieceMinKeys) piece_keys = kHostPieceMinKeys;
+  const int n_pieces = static_cast<int>((L + piece_keys - 1) / piece_keys);
+  int rc;
+  if (n_pieces < 2) {
+    ILRE_CUDA(cudaMemcpyAsync(h->stage_k, k_cache_host, k_bytes, cudaMemcpyHostToDevice, st));
+    rc = ilre_recall_run(h, h->stage_k, L, h->stage_q, q_len, budget, spec, h->stage_idx, nullptr,
+                         st);
+  } else {
+    const size_t row_bytes = static_cast<size_t>(h->cfg.n_kv_heads) * 256;
+    const size_t n_rows = static_cast<size_t>(q_len) * h->cfg.n_q_heads;
+    ILRE_CUDA(cudaEventRecord(h->copy_begin, st));            // the staging buffer is free again
+    ILRE_CUDA(cudaStreamWaitEvent(h->copy_stream, h->copy_begin, 0));
+    rc = ILRE_OK;
+    for (int i = 0; i < n_pieces && rc == ILRE_OK; ++i) {
+      const long long lo = i * piece_keys;
+      const long long hi = (lo + piece_keys < L) ? lo + piece_keys : static_cast<long long>(L);
+      uint8_t* dst = static_cast<uint8_t*>(h->stage_k) + lo * row_bytes;
+      ILRE_CUDA(cudaMemcpyAsync(dst, static_cast<const uint8_t*>(k_cache_host) + lo * row_bytes,
+                                (hi - lo) * row_bytes, cudaMemcpyHostToDevice, h->copy_stream));
+      ILRE_CUDA(cudaEventRecord(h->piece_done[i], h->copy_stream));
+      ILRE_CUDA(cudaStreamWaitEvent(st, h->piece_done[i], 0));
+      const RunIo io = {kStageStats, h->piece_stats + i * n_rows, nullptr, 0, nullptr, nullptr};
+      rc = recall_impl(h, dst, hi - lo, h->stage_q, q_len, 0, nullptr, nullptr, nullptr, st, io);
+    }
+    if (rc == ILRE_OK) {
+      const RunIo io = {kStageScores | kStageSelect, nullptr, h->piece_stats, n_pieces, nullptr,
+                        nullptr};
+      rc = recall_impl(h, h->stage_k, L, h->stage_q, q_len, budget, spec, h->stage_idx, nullptr, st,
+                       io);
+    }
+    if (rc != ILRE_OK) cudaStreamSynchronize(h->copy_stream);   // nothing in flight on return
+  }
   if (rc != ILRE_OK) return rc;
   ILRE_CUDA(cudaMemcpyAsync(out_idx_host, h->stage_idx,
                             static_cast<size_t>(spec->n_sink + budget) * sizeof(int32_t),
