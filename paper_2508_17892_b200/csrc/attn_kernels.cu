@@ -5,7 +5,7 @@
 //
 // One CTA per (128 query tokens, pair of query heads that share a kv head).  Both contractions
 // run on the tensor cores: S = Q K^T into tensor memory, and O += P V with P written to shared
-// memory as bf16 by the softmax warps (eight per head).  The two heads are two independent streams over the
+// memory as bf16 by the softmax warps (four per head, one thread per query row).  The two heads are two independent streams over the
 // same key/value tiles (one TMA ring feeds both): while the softmax warpgroup of one stream
 // works on its S tile, the tensor cores serve the other stream.  One sweep over the key tiles
 // with an online softmax: probabilities are taken against a per-row reference maximum, O
@@ -22,8 +22,7 @@ namespace ilre {
 static constexpr int kAttnStages = 3;
 static constexpr int kAttnTileBytes = 128 * 128 * 2;       // one 128 x 128 bf16 tile
 static constexpr int kAttnTailBytes = 256;
-static constexpr int kAttnSoftmaxWarps = 8;                // per stream: two per TMEM lane quadrant
-static constexpr int kAttnXchgBytes = 2 * 1024;            // per stream: [2 halves][128 rows] floats
+static constexpr int kAttnSoftmaxWarps = 4;                // per stream: one per TMEM lane quadrant
 
 struct AttnTail {
   uint64_t q_full;
@@ -59,7 +58,6 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
   const uint32_t p_s = ring_s + kAttnStages * kAttnTileBytes;           // 2 tiles
   uint8_t* p_ptr = smem + (2 + kAttnStages) * kAttnTileBytes;
   AttnTail* tail = reinterpret_cast<AttnTail*>(smem + (4 + kAttnStages) * kAttnTileBytes);
-  float* xchg_all = reinterpret_cast<float*>(smem + (4 + kAttnStages) * kAttnTileBytes + kAttnTailBytes);
   volatile int* abort_flag = &tail->abort_flag;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -157,6 +155,18 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
         const int v_item = 2 * t + 1, k_item = 2 * t + 2;
         const uint32_t v_s = ring_s + (v_item % kAttnStages) * kAttnTileBytes;
         for (int x = 0; x < n_streams && ok; ++x) {
+          // S_x of the next tile first: it needs only that the softmax warps have taken S_x(t)
+          // out of tensor memory, which they do before they finish P_x(t); the next softmax
+          // can then start while O_x += P_x V_t is still running
+          if (t + 1 < n_tiles) {
+            ok = mbar_wait(smem_u32(&tail->s_empty[x]), static_cast<uint32_t>(t) & 1u, abort_flag,
+                           p.status, kDevWaitAccEmpty);
+            if (ok && x == 0) ok = ring_wait(k_item);
+            if (!ok) break;
+            tc_fence_after();
+            issue_s(x, t + 1);
+            if (x == n_streams - 1) umma_commit(smem_u32(&tail->kv_empty[k_item % kAttnStages]));
+          }
           // O_x += P_x V_t
           ok = mbar_wait(smem_u32(&tail->p_full[x]), static_cast<uint32_t>(t) & 1u, abort_flag,
                          p.status, kDevWaitAccFull);
@@ -173,67 +183,60 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
                         (t | kb | ks) != 0);
           umma_commit(smem_u32(&tail->p_empty[x]));
           if (x == n_streams - 1) umma_commit(smem_u32(&tail->kv_empty[v_item % kAttnStages]));
-          // S_x of the next tile: its softmax warps have read S_x(t) before they wrote P_x(t)
-          if (t + 1 < n_tiles) {
-            ok = mbar_wait(smem_u32(&tail->s_empty[x]), static_cast<uint32_t>(t) & 1u, abort_flag,
-                           p.status, kDevWaitAccEmpty);
-            if (ok && x == 0) ok = ring_wait(k_item);
-            if (!ok) break;
-            tc_fence_after();
-            issue_s(x, t + 1);
-            if (x == n_streams - 1) umma_commit(smem_u32(&tail->kv_empty[k_item % kAttnStages]));
-          }
         }
       }
       if (ok) umma_commit(smem_u32(&tail->o_full));
     }
   } else if ((warp - 2) / kAttnSoftmaxWarps < n_streams) {
-    // Softmax warps of stream x: warp w reads TMEM lane quadrant w % 4; the two warps of a
-    // quadrant split the 128 columns (keys of S, channels of O) in halves, so a thread owns
-    // half a query row; the halves meet through shared memory once per tile (the maximum).
-    // Every warp runs all iterations, also after a wait was abandoned, so that the stream's
-    // named barrier always gets its 256 threads.
+    // Softmax warps of stream x: warp w reads TMEM lane quadrant w % 4, so a thread owns one
+    // query row: its 128 logits of the tile, its running reference and sum, its row of P and
+    // of O.  No thread ever needs another's values.
     const int x = (warp - 2) / kAttnSoftmaxWarps;
-    const int quad = warp & 3, half = ((warp - 2) % kAttnSoftmaxWarps) >> 2;
+    const int quad = warp & 3;
     const int row = quad * 32 + lane;
     const int qj = j0 + row;
     const int h = h0 + x;
     const int limit = p.n_prefix + qj;                   // last visible key row of this query
-    const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + half * 64;
+    const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
     const uint32_t s_tm = lane_base + x * 128, o_tm = lane_base + 256 + x * 128;
-    uint8_t* p_mine = p_ptr + x * kAttnTileBytes + half * 16384;
-    float* xchg = xchg_all + x * 256;                    // [2][128]
-    const int bar_id = 1 + x;
+    uint8_t* p_mine = p_ptr + x * kAttnTileBytes;
     const float c2 = p.c2;
     bool ok = run;
-    // Online softmax: `ref` is the row's reference maximum (raw logits), `l` this thread's
-    // share of the sum of 2^((s - ref) c2) over the keys seen so far.
+    // Online softmax: `ref` is the row's reference maximum (raw logits), `l` the sum of
+    // 2^((s - ref) c2) over the keys seen so far.
     constexpr float kRefSlack = 8.f;                     // log2 units
     float ref = -INFINITY, l = 0.f;
-    for (int t = 0; t < n_tiles; ++t) {
-      if (ok)
-        ok = mbar_wait(smem_u32(&tail->s_full[x]), static_cast<uint32_t>(t) & 1u, abort_flag,
-                       p.status, kDevWaitAccFull);
-      // tile maximum of the visible logits
-      float cm = -INFINITY;
-      if (ok) {
-        tc_fence_after();
-#pragma unroll 1
-        for (int q2 = 0; q2 < 2; ++q2) {
-          float v[32];
-          tmem_ld32(s_tm + q2 * 32, v);
-          tmem_ld_wait();
-          const int k0 = t * 128 + half * 64 + q2 * 32;
+    for (int t = 0; t < n_tiles && ok; ++t) {
+      ok = mbar_wait(smem_u32(&tail->s_full[x]), static_cast<uint32_t>(t) & 1u, abort_flag,
+                     p.status, kDevWaitAccFull);
+      if (!ok) break;
+      // The row's 128 logits stay in registers for both the maximum and the exponentials, so
+      // S leaves tensor memory once and the tensor cores get it back for the next tile right
+      // away.  Only the tiles on the causal diagonal need the mask; there the hidden logits
+      // become -inf, which the code below turns into probability 0.
+      float vv[4][32];
+#define V(i) vv[(i) >> 5][(i) & 31]
+      tc_fence_after();
+      tmem_ld32(s_tm, vv[0]);
+      tmem_ld32(s_tm + 32, vv[1]);
+      tmem_ld32(s_tm + 64, vv[2]);
+      tmem_ld32(s_tm + 96, vv[3]);
+      tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&tail->s_empty[x]));
+      const int k0 = t * 128;
+      if (k0 + 127 > p.n_prefix + j0) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (k0 + i <= limit) cm = fmaxf(cm, v[i]);
-        }
+        for (int i = 0; i < 128; ++i) V(i) = (k0 + i <= limit) ? V(i) : -INFINITY;
       }
-      xchg[half * 128 + row] = cm;
-      asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(kAttnSoftmaxWarps * 32) : "memory");
-      cm = fmaxf(cm, xchg[(half ^ 1) * 128 + row]);
-      asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(kAttnSoftmaxWarps * 32) : "memory");
-      if (!ok) continue;
+      float m0 = fmax3(V(0), V(1), V(2)), m1 = fmax3(V(3), V(4), V(5));
+#pragma unroll
+      for (int i = 6; i < 126; i += 4) {
+        m0 = fmax3(m0, V(i), V(i + 1));
+        m1 = fmax3(m1, V(i + 2), V(i + 3));
+      }
+      const float cm = fmax3(m0, m1, fmaxf(V(126), V(127)));
       // move the reference only when the maximum has run ahead of it
       float scale = 1.f;
       if ((cm - ref) * c2 > kRefSlack || ref == -INFINITY) {
@@ -241,71 +244,60 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
         ref = (cm == -INFINITY) ? ref : cm;
       }
       const float nr = (ref == -INFINITY) ? 0.f : -ref * c2;
-      uint32_t packed[32];
-      float sum = 0.f;
+      // the bf16 pairs go back into the registers of the logits they replace
+      float2 sum2 = make_float2(0.f, 0.f);
 #pragma unroll
-      for (int q2 = 0; q2 < 2; ++q2) {
-        float v[32];
-        tmem_ld32(s_tm + q2 * 32, v);
-        tmem_ld_wait();
-        const int k0 = t * 128 + half * 64 + q2 * 32;
-#pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          const float p0 = (k0 + i <= limit) ? ex2_approx(fmaf(v[i], c2, nr)) : 0.f;
-          const float p1 = (k0 + i + 1 <= limit) ? ex2_approx(fmaf(v[i + 1], c2, nr)) : 0.f;
-          sum += p0 + p1;
-          const __nv_bfloat162 pr = __floats2bfloat162_rn(p0, p1);
-          packed[q2 * 16 + (i >> 1)] = *reinterpret_cast<const uint32_t*>(&pr);
-        }
+      for (int i = 0; i < 128; i += 2) {
+        const float2 a = ffma2(make_float2(V(i), V(i + 1)), make_float2(c2, c2), make_float2(nr, nr));
+        const float2 pp = make_float2(ex2_approx(a.x), ex2_approx(a.y));
+        sum2 = fadd2(sum2, pp);
+        const __nv_bfloat162 pr = __floats2bfloat162_rn(pp.x, pp.y);
+        V(i >> 1) = __uint_as_float(*reinterpret_cast<const uint32_t*>(&pr));
       }
-      l = fmaf(l, scale, sum);
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&tail->s_empty[x]));
+      l = fmaf(l, scale, sum2.x + sum2.y);
       // the previous tile's P must have been consumed (and O updated) by its MMAs
       ok = mbar_wait(smem_u32(&tail->p_empty[x]), (static_cast<uint32_t>(t) & 1u) ^ 1u, abort_flag,
                      p.status, kDevWaitAccEmpty);
-      if (!ok) continue;
+      if (!ok) break;
       if (t > 0 && __any_sync(0xFFFFFFFFu, scale != 1.f)) {
-        // rescale this warp's share of O (32 rows x 64 channels) to the new references
+        // rescale this warp's 32 rows of O to the new references
         tc_fence_after();
 #pragma unroll 1
-        for (int q2 = 0; q2 < 2; ++q2) {
+        for (int q4 = 0; q4 < 4; ++q4) {
           float o[32];
-          tmem_ld32(o_tm + q2 * 32, o);
+          tmem_ld32(o_tm + q4 * 32, o);
           tmem_ld_wait();
 #pragma unroll
           for (int i = 0; i < 32; ++i) o[i] *= scale;
-          tmem_st32(o_tm + q2 * 32, o);
+          tmem_st32(o_tm + q4 * 32, o);
         }
         tmem_st_wait();
         tc_fence_before();
       }
-      // P[row][key]: one half of 64 keys per warp of the quadrant, rows of 128 bytes, 16-byte
-      // groups XOR-swizzled by the row index (the layout TMA's 128-byte swizzle produces for
-      // the other operands)
+      // P[row][key]: two halves of 64 keys, rows of 128 bytes, 16-byte groups XOR-swizzled by
+      // the row index (the layout TMA's 128-byte swizzle produces for the other operands)
 #pragma unroll
-      for (int c16 = 0; c16 < 8; ++c16) {
-        uint4* dst = reinterpret_cast<uint4*>(p_mine + row * 128 + ((c16 ^ (row & 7)) << 4));
-        *dst = make_uint4(packed[c16 * 4], packed[c16 * 4 + 1], packed[c16 * 4 + 2],
-                          packed[c16 * 4 + 3]);
+      for (int c16 = 0; c16 < 16; ++c16) {
+        uint4* dst = reinterpret_cast<uint4*>(p_mine + (c16 >> 3) * 16384 + row * 128 +
+                                              (((c16 & 7) ^ (row & 7)) << 4));
+        *dst = make_uint4(__float_as_uint(V(c16 * 4)), __float_as_uint(V(c16 * 4 + 1)),
+                          __float_as_uint(V(c16 * 4 + 2)), __float_as_uint(V(c16 * 4 + 3)));
       }
+#undef V
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&tail->p_full[x]));
     }
-    // ---- output: O / (sum of both halves), this thread's 64 channels ----
-    xchg[half * 128 + row] = l;
-    asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(kAttnSoftmaxWarps * 32) : "memory");
-    const float inv_l = 1.f / (l + xchg[(half ^ 1) * 128 + row]);
+    // ---- output: O / sum, this thread's row ----
+    const float inv_l = 1.f / l;
     if (ok) ok = mbar_wait(smem_u32(&tail->o_full), 0, abort_flag, p.status, kDevWaitAccFull);
     if (ok) {
       tc_fence_after();
-      uint16_t* dst = p.out + (static_cast<size_t>(qj) * p.n_q + h) * 128 + half * 64;
+      uint16_t* dst = p.out + (static_cast<size_t>(qj) * p.n_q + h) * 128;
 #pragma unroll 1
-      for (int q2 = 0; q2 < 2; ++q2) {
+      for (int q4 = 0; q4 < 4; ++q4) {
         float v[32];
-        tmem_ld32(o_tm + q2 * 32, v);
+        tmem_ld32(o_tm + q4 * 32, v);
         tmem_ld_wait();
         if (qj < p.c) {
           uint32_t w[16];
@@ -314,7 +306,7 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
             const __nv_bfloat162 pr = __floats2bfloat162_rn(v[i] * inv_l, v[i + 1] * inv_l);
             w[i >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
           }
-          uint4* d4 = reinterpret_cast<uint4*>(dst + q2 * 32);
+          uint4* d4 = reinterpret_cast<uint4*>(dst + q4 * 32);
 #pragma unroll
           for (int q = 0; q < 4; ++q) d4[q] = make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
         }
@@ -330,7 +322,7 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
 }
 
 size_t attn_smem_bytes() {
-  return static_cast<size_t>(4 + kAttnStages) * kAttnTileBytes + kAttnTailBytes + kAttnXchgBytes;
+  return static_cast<size_t>(4 + kAttnStages) * kAttnTileBytes + kAttnTailBytes;
 }
 
 cudaError_t launch_chunk_attention(const CUtensorMap& map_q, const CUtensorMap& map_k,

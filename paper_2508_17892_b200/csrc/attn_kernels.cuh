@@ -8,7 +8,7 @@
 
 namespace ilre {
 
-static constexpr int kAttnThreads = 576;     // warp 0 TMA, warp 1 MMA, warps 2..9 / 10..17 softmax
+static constexpr int kAttnThreads = 320;     // warp 0 TMA, warp 1 MMA, warps 2..5 / 6..9 softmax
 
 struct AttnParams {
   int c;             // query tokens of the chunk
