@@ -129,11 +129,6 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
       constexpr uint32_t idesc_o = umma_idesc_bf16(128, 128) | (1u << 16);   // B = V: channels contiguous
       bool ok = mbar_wait(smem_u32(&tail->q_full), 0, abort_flag, p.status, kDevWaitQFull);
       tc_fence_after();
-      auto ring_wait = [&](int item) -> bool {
-        return mbar_wait(smem_u32(&tail->kv_full[item % kAttnStages]),
-                         static_cast<uint32_t>(item / kAttnStages) & 1u, abort_flag, p.status,
-                         kDevWaitKFull);
-      };
       auto issue_s = [&](int x, int t) {                  // S_x = Q_x K_t^T
         const uint32_t k_s = ring_s + ((2 * t) % kAttnStages) * kAttnTileBytes;
         const uint32_t qx = q_s + x * kAttnTileBytes;
@@ -145,44 +140,72 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
                       umma_desc_sw128(k_s + kb * 16384 + ks * 32), idesc_s, (kb | ks) != 0);
         umma_commit(smem_u32(&tail->s_full[x]));
       };
-      if (ok) ok = ring_wait(0);
-      if (ok) {
-        tc_fence_after();
-        for (int x = 0; x < n_streams; ++x) issue_s(x, 0);
-        umma_commit(smem_u32(&tail->kv_empty[0]));
-      }
-      for (int t = 0; t < n_tiles && ok; ++t) {
-        const int v_item = 2 * t + 1, k_item = 2 * t + 2;
-        const uint32_t v_s = ring_s + (v_item % kAttnStages) * kAttnTileBytes;
-        for (int x = 0; x < n_streams && ok; ++x) {
-          // S_x of the next tile first: it needs only that the softmax warps have taken S_x(t)
-          // out of tensor memory, which they do before they finish P_x(t); the next softmax
-          // can then start while O_x += P_x V_t is still running
-          if (t + 1 < n_tiles) {
-            ok = mbar_wait(smem_u32(&tail->s_empty[x]), static_cast<uint32_t>(t) & 1u, abort_flag,
-                           p.status, kDevWaitAccEmpty);
-            if (ok && x == 0) ok = ring_wait(k_item);
-            if (!ok) break;
+      // Event-driven issue: per stream the next S = Q K^T (needs the softmax warps to have
+      // taken the previous S out of tensor memory, and the key tile) and the next
+      // O += P V (needs P and the value tile); whichever is ready goes first, so neither
+      // stream ever waits for the other's softmax.  A ring slot is released once both
+      // streams have issued the MMAs that read it.
+      auto ring_ready = [&](int item) -> bool {
+        return mbar_test_wait(smem_u32(&tail->kv_full[item % kAttnStages]),
+                              static_cast<uint32_t>(item / kAttnStages) & 1u);
+      };
+      int next_s[2] = {0, 0}, next_pv[2] = {0, 0};
+      if (n_streams == 1) next_s[1] = next_pv[1] = n_tiles;
+      int k_released = 0, v_released = 0;
+      long long t_idle = 0;
+      uint32_t spins = 0;
+      while (ok && (next_pv[0] < n_tiles || next_pv[1] < n_tiles)) {
+        bool progress = false;
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+          int t = next_s[x];
+          if (t < n_tiles && ring_ready(2 * t) &&
+              (t == 0 || mbar_test_wait(smem_u32(&tail->s_empty[x]), static_cast<uint32_t>(t - 1) & 1u))) {
             tc_fence_after();
-            issue_s(x, t + 1);
-            if (x == n_streams - 1) umma_commit(smem_u32(&tail->kv_empty[k_item % kAttnStages]));
+            issue_s(x, t);
+            next_s[x] = t + 1;
+            progress = true;
+            while (k_released < min(next_s[0], next_s[1])) {
+              umma_commit(smem_u32(&tail->kv_empty[(2 * k_released) % kAttnStages]));
+              ++k_released;
+            }
           }
-          // O_x += P_x V_t
-          ok = mbar_wait(smem_u32(&tail->p_full[x]), static_cast<uint32_t>(t) & 1u, abort_flag,
-                         p.status, kDevWaitAccFull);
-          if (ok && x == 0) ok = ring_wait(v_item);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t px = p_s + x * kAttnTileBytes;
+          t = next_pv[x];
+          if (t < n_tiles && t < next_s[x] && ring_ready(2 * t + 1) &&
+              mbar_test_wait(smem_u32(&tail->p_full[x]), static_cast<uint32_t>(t) & 1u)) {
+            tc_fence_after();
+            const uint32_t v_s = ring_s + ((2 * t + 1) % kAttnStages) * kAttnTileBytes;
+            const uint32_t px = p_s + x * kAttnTileBytes;
 #pragma unroll
-          for (int kb = 0; kb < 2; ++kb)
+            for (int kb = 0; kb < 2; ++kb)
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-              umma_bf16(tmem_base + 256 + x * 128, umma_desc_sw128(px + kb * 16384 + ks * 32),
-                        umma_desc_sw128_mn(v_s + (kb * 64 + ks * 16) * 128, 16384, 1024), idesc_o,
-                        (t | kb | ks) != 0);
-          umma_commit(smem_u32(&tail->p_empty[x]));
-          if (x == n_streams - 1) umma_commit(smem_u32(&tail->kv_empty[v_item % kAttnStages]));
+              for (int ks = 0; ks < 4; ++ks)
+                umma_bf16(tmem_base + 256 + x * 128, umma_desc_sw128(px + kb * 16384 + ks * 32),
+                          umma_desc_sw128_mn(v_s + (kb * 64 + ks * 16) * 128, 16384, 1024), idesc_o,
+                          (t | kb | ks) != 0);
+            umma_commit(smem_u32(&tail->p_empty[x]));
+            next_pv[x] = t + 1;
+            progress = true;
+            while (v_released < min(next_pv[0], next_pv[1])) {
+              umma_commit(smem_u32(&tail->kv_empty[(2 * v_released + 1) % kAttnStages]));
+              ++v_released;
+            }
+          }
+        }
+        // bounded: give up when nothing became ready for kWaitCycleLimit cycles
+        if (progress) {
+          spins = 0;
+        } else {
+          if (spins == 0) t_idle = clock64();
+          if ((++spins & 0x3FF) == 0) {
+            if (*abort_flag) {
+              ok = false;
+            } else if (clock64() - t_idle > kWaitCycleLimit) {
+              *abort_flag = 1;
+              atomicCAS(p.status, 0, kDevWaitAccFull);
+              ok = false;
+            }
+          }
         }
       }
       if (ok) umma_commit(smem_u32(&tail->o_full));
