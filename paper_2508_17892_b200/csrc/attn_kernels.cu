@@ -267,21 +267,36 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
         ref = (cm == -INFINITY) ? ref : cm;
       }
       const float nr = (ref == -INFINITY) ? 0.f : -ref * c2;
-      // the bf16 pairs go back into the registers of the logits they replace
-      float2 sum2 = make_float2(0.f, 0.f);
-#pragma unroll
-      for (int i = 0; i < 128; i += 2) {
-        const float2 a = ffma2(make_float2(V(i), V(i + 1)), make_float2(c2, c2), make_float2(nr, nr));
-        const float2 pp = make_float2(ex2_approx(a.x), ex2_approx(a.y));
-        sum2 = fadd2(sum2, pp);
-        const __nv_bfloat162 pr = __floats2bfloat162_rn(pp.x, pp.y);
-        V(i >> 1) = __uint_as_float(*reinterpret_cast<const uint32_t*>(&pr));
-      }
-      l = fmaf(l, scale, sum2.x + sum2.y);
       // the previous tile's P must have been consumed (and O updated) by its MMAs
       ok = mbar_wait(smem_u32(&tail->p_empty[x]), (static_cast<uint32_t>(t) & 1u) ^ 1u, abort_flag,
                      p.status, kDevWaitAccEmpty);
       if (!ok) break;
+      // Exponentials in groups of 32 keys; each group's bf16 pairs go straight to P[row][key]
+      // (two halves of 64 keys, rows of 128 bytes, 16-byte groups XOR-swizzled by the row index:
+      // the layout TMA's 128-byte swizzle produces for the other operands), so the stores
+      // drain while the next group is computed.
+      float2 sum2 = make_float2(0.f, 0.f);
+#pragma unroll
+      for (int g32 = 0; g32 < 4; ++g32) {
+        uint32_t w[16];
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+          const float2 a = ffma2(make_float2(V(g32 * 32 + i), V(g32 * 32 + i + 1)), make_float2(c2, c2),
+                                 make_float2(nr, nr));
+          const float2 pp = make_float2(ex2_approx(a.x), ex2_approx(a.y));
+          sum2 = fadd2(sum2, pp);
+          const __nv_bfloat162 pr = __floats2bfloat162_rn(pp.x, pp.y);
+          w[i >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
+        }
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int c16 = g32 * 4 + c;
+          uint4* dst = reinterpret_cast<uint4*>(p_mine + (c16 >> 3) * 16384 + row * 128 +
+                                                (((c16 & 7) ^ (row & 7)) << 4));
+          *dst = make_uint4(w[c * 4], w[c * 4 + 1], w[c * 4 + 2], w[c * 4 + 3]);
+        }
+      }
+      l = fmaf(l, scale, sum2.x + sum2.y);
       if (t > 0 && __any_sync(0xFFFFFFFFu, scale != 1.f)) {
         // rescale this warp's 32 rows of O to the new references
         tc_fence_after();
@@ -296,15 +311,6 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
         }
         tmem_st_wait();
         tc_fence_before();
-      }
-      // P[row][key]: two halves of 64 keys, rows of 128 bytes, 16-byte groups XOR-swizzled by
-      // the row index (the layout TMA's 128-byte swizzle produces for the other operands)
-#pragma unroll
-      for (int c16 = 0; c16 < 16; ++c16) {
-        uint4* dst = reinterpret_cast<uint4*>(p_mine + (c16 >> 3) * 16384 + row * 128 +
-                                              (((c16 & 7) ^ (row & 7)) << 4));
-        *dst = make_uint4(__float_as_uint(V(c16 * 4)), __float_as_uint(V(c16 * 4 + 1)),
-                          __float_as_uint(V(c16 * 4 + 2)), __float_as_uint(V(c16 * 4 + 3)));
       }
 #undef V
       fence_proxy_async_smem();
