@@ -99,7 +99,7 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
   const bool run = (*abort_flag == 0);
 
   // TMEM columns: S of stream x at 128 x, O of stream x at 256 + 128 x.
-  // Ring items: K_0, V_0, K_1, V_1, ... each used by both streams.
+  // Ring items (key and value tiles) are each used by both streams.
   if (warp == 0) {
     if (lane == 0 && run) {
       const uint32_t qf = smem_u32(&tail->q_full);
@@ -108,6 +108,9 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
         tma_load_2d(q_s + x * kAttnTileBytes, &map_q, (h0 + x) * 128, j0, qf);
         tma_load_2d(q_s + x * kAttnTileBytes + 16384, &map_q, (h0 + x) * 128 + 64, j0, qf);
       }
+      // Ring order K_0, K_1, V_0, K_2, V_1, ..., K_{n-1}, V_{n-2}, V_{n-1}: the key tile runs
+      // one tile ahead of the value tile, because S of the next tile is issued while the
+      // softmax of the current one is still running (see the MMA warp).
       const int n_items = 2 * n_tiles;
       for (int it = 0; it < n_items; ++it) {
         const int s = it % kAttnStages;
@@ -115,8 +118,9 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
         if (!mbar_wait(smem_u32(&tail->kv_empty[s]), (use & 1u) ^ 1u, abort_flag, p.status,
                        kDevWaitKEmpty))
           break;
-        const CUtensorMap* map = (it & 1) ? &map_v : &map_k;
-        const int t = it >> 1;
+        const bool is_k = (it == 0) || ((it & 1) && it != n_items - 1);
+        const int t = (it == 0) ? 0 : (it == n_items - 1) ? n_tiles - 1 : is_k ? (it + 1) / 2 : it / 2 - 1;
+        const CUtensorMap* map = is_k ? &map_k : &map_v;
         const uint32_t bar = smem_u32(&tail->kv_full[s]);
         mbar_arrive_expect_tx(bar, kAttnTileBytes);
         tma_load_2d(ring_s + s * kAttnTileBytes, map, g * 128, t * 128, bar);
@@ -129,8 +133,10 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
       constexpr uint32_t idesc_o = umma_idesc_bf16(128, 128) | (1u << 16);   // B = V: channels contiguous
       bool ok = mbar_wait(smem_u32(&tail->q_full), 0, abort_flag, p.status, kDevWaitQFull);
       tc_fence_after();
+      auto k_item = [&](int t) -> int { return t == 0 ? 0 : 2 * t - 1; };
+      auto v_item = [&](int t) -> int { return t < n_tiles - 1 ? 2 * t + 2 : 2 * n_tiles - 1; };
       auto issue_s = [&](int x, int t) {                  // S_x = Q_x K_t^T
-        const uint32_t k_s = ring_s + ((2 * t) % kAttnStages) * kAttnTileBytes;
+        const uint32_t k_s = ring_s + (k_item(t) % kAttnStages) * kAttnTileBytes;
         const uint32_t qx = q_s + x * kAttnTileBytes;
 #pragma unroll
         for (int kb = 0; kb < 2; ++kb)
@@ -159,22 +165,22 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
           int t = next_s[x];
-          if (t < n_tiles && ring_ready(2 * t) &&
+          if (t < n_tiles && ring_ready(k_item(t)) &&
               (t == 0 || mbar_test_wait(smem_u32(&tail->s_empty[x]), static_cast<uint32_t>(t - 1) & 1u))) {
             tc_fence_after();
             issue_s(x, t);
             next_s[x] = t + 1;
             progress = true;
             while (k_released < min(next_s[0], next_s[1])) {
-              umma_commit(smem_u32(&tail->kv_empty[(2 * k_released) % kAttnStages]));
+              umma_commit(smem_u32(&tail->kv_empty[k_item(k_released) % kAttnStages]));
               ++k_released;
             }
           }
           t = next_pv[x];
-          if (t < n_tiles && t < next_s[x] && ring_ready(2 * t + 1) &&
+          if (t < n_tiles && t < next_s[x] && ring_ready(v_item(t)) &&
               mbar_test_wait(smem_u32(&tail->p_full[x]), static_cast<uint32_t>(t) & 1u)) {
             tc_fence_after();
-            const uint32_t v_s = ring_s + ((2 * t + 1) % kAttnStages) * kAttnTileBytes;
+            const uint32_t v_s = ring_s + (v_item(t) % kAttnStages) * kAttnTileBytes;
             const uint32_t px = p_s + x * kAttnTileBytes;
 #pragma unroll
             for (int kb = 0; kb < 2; ++kb)
@@ -187,7 +193,7 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
             next_pv[x] = t + 1;
             progress = true;
             while (v_released < min(next_pv[0], next_pv[1])) {
-              umma_commit(smem_u32(&tail->kv_empty[(2 * v_released + 1) % kAttnStages]));
+              umma_commit(smem_u32(&tail->kv_empty[v_item(v_released) % kAttnStages]));
               ++v_released;
             }
           }
