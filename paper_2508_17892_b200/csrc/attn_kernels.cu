@@ -162,21 +162,10 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
       uint32_t spins = 0;
       while (ok && (next_pv[0] < n_tiles || next_pv[1] < n_tiles)) {
         bool progress = false;
+        // O += P V first: it frees the stream's P buffer, which its softmax warps need soonest
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
-          int t = next_s[x];
-          if (t < n_tiles && ring_ready(k_item(t)) &&
-              (t == 0 || mbar_test_wait(smem_u32(&tail->s_empty[x]), static_cast<uint32_t>(t - 1) & 1u))) {
-            tc_fence_after();
-            issue_s(x, t);
-            next_s[x] = t + 1;
-            progress = true;
-            while (k_released < min(next_s[0], next_s[1])) {
-              umma_commit(smem_u32(&tail->kv_empty[k_item(k_released) % kAttnStages]));
-              ++k_released;
-            }
-          }
-          t = next_pv[x];
+          const int t = next_pv[x];
           if (t < n_tiles && t < next_s[x] && ring_ready(v_item(t)) &&
               mbar_test_wait(smem_u32(&tail->p_full[x]), static_cast<uint32_t>(t) & 1u)) {
             tc_fence_after();
@@ -195,6 +184,21 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
             while (v_released < min(next_pv[0], next_pv[1])) {
               umma_commit(smem_u32(&tail->kv_empty[v_item(v_released) % kAttnStages]));
               ++v_released;
+            }
+          }
+        }
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+          const int t = next_s[x];
+          if (t < n_tiles && ring_ready(k_item(t)) &&
+              (t == 0 || mbar_test_wait(smem_u32(&tail->s_empty[x]), static_cast<uint32_t>(t - 1) & 1u))) {
+            tc_fence_after();
+            issue_s(x, t);
+            next_s[x] = t + 1;
+            progress = true;
+            while (k_released < min(next_s[0], next_s[1])) {
+              umma_commit(smem_u32(&tail->kv_empty[k_item(k_released) % kAttnStages]));
+              ++k_released;
             }
           }
         }
