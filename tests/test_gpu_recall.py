@@ -269,4 +269,24 @@ def test_full_size_1m_config_sampled():
     assert np.all(np.isfinite(sc)) and sc.min() > 0 and sc.max() <= 1
     own = oracle.allocate(sc.astype(np.float64), w.budget, w.max_sizes, w.win_sizes, w.win_op, 0)
     np.testing.assert_array_equal(idx, own)
+    # The same context as eight key shards of 131072 positions (the per-rank steps bench.py
+    # times with --shards 8): merged statistics, sampled scores and the selection logic
+    # against the oracle, and the scores against the unsharded run's.
+    from paper_2508_17892_b200.sharded import shard_bounds
+    K, Q = x.K.cuda(), x.Q.cuda()
+    bounds = [shard_bounds(w.L, 8, r) for r in range(8)]
+    stats = torch.stack([eng.shard_stats(K[a:b], Q) for a, b in bounds])
+    sc8 = torch.cat([eng.shard_scores(K[a:b], Q, stats) for a, b in bounds])
+    idx8 = eng.allocate(sc8, w.budget, w.max_sizes, w.win_sizes, w.win_op, w.n_sink)
+    torch.cuda.synchronize()
+    eng.check_status()
+    sc8, idx8 = sc8.cpu().numpy(), idx8.cpu().numpy()
+    lse8 = eng.row_lse(w.q_len).cpu().numpy().reshape(-1).astype(np.float64)
+    assert np.abs(lse8[rows] - (m + np.log(z))).max() < 5e-4
+    assert np.abs(lse8 - gpu_lse).max() < 1e-5
+    rep8 = parity.score_errors(sc8[pos].astype(np.float64), ref)
+    assert rep8["n_bad"] == 0, rep8
+    assert np.abs(sc8 - sc).max() <= 2e-5 * sc.max() and np.all(np.abs(sc8 - sc) <= 1e-4 * sc)
+    own8 = oracle.allocate(sc8.astype(np.float64), w.budget, w.max_sizes, w.win_sizes, w.win_op, 0)
+    np.testing.assert_array_equal(idx8, own8)
     eng.close()
