@@ -303,10 +303,15 @@ def run_ours(args, world, rank, local):
     barrier()
     elapsed_ms = start.elapsed_time(stop)
     stages = eng.stage_times()
+    sm_mhz_in_kernel = eng.sm_clock_mhz()
     eng.set_profiling(False)
     launches = eng.last_launch_count() * args.steps
     eng.check_status()
     clocks = sampler.stop() if rank == 0 else None
+    if clocks is not None:
+        # what the driver reports is the clock it asks for; under the power cap the SMs run
+        # slower: cycles / global-timer nanoseconds of the last row-statistics launch
+        clocks["sm_mhz_in_kernel"] = sm_mhz_in_kernel
 
     # end to end through the host entry point: pinned host inputs, copies inside the timing
     e2e = None
@@ -541,7 +546,9 @@ def run_ours(args, world, rank, local):
     roofline["row_stats_exponentials"] = dict(
         bound="alu", achieved=exp_rate / 1e12, peak=exp_peak / 1e12, unit="Texp/s",
         frac=exp_rate / exp_peak,
-        peak_source=f"16 ex2 per clock per SM x {n_sm} SMs x {sm_max_ghz:.3f} GHz")
+        peak_source=f"16 ex2 per clock per SM x {n_sm} SMs x {sm_max_ghz:.3f} GHz",
+        frac_at_in_kernel_clock=(exp_rate / (16.0 * n_sm * sm_mhz_in_kernel * 1e6)
+                                 if sm_mhz_in_kernel > 0 else None))
     step_hbm_frac = (k_bytes / (ms_per_step * 1e-3) / 1e9) / peaks["hbm_gbs"]
     step_tensor_frac = (flops / (ms_per_step * 1e-3) / 1e12) / peaks["bf16_tflops_sustained"]
 

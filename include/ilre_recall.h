@@ -253,6 +253,14 @@ int ilre_recall_copy_row_lse(ilre_recall_t* h, float* out_lse_dev, int32_t q_len
 int ilre_recall_status(ilre_recall_t* h);
 
 /*
+ * SM clock, in MHz, that the row-statistics kernel of the last run with profiling on really ran
+ * at: SM cycles of its first CTA over the global timer's nanoseconds (0 if no such run yet).
+ * Under the board's power cap this is well below the clock the driver reports.  Measurement
+ * aid; the paper has no counterpart.  Synchronises the last run's stream.
+ */
+int ilre_recall_sm_clock(ilre_recall_t* h, float* mhz_out_host);
+
+/*
  * Stage timing.  With profiling on, run() records CUDA events between its stages on the
  * caller's stream (the events of the 32 most recent runs are kept).  Switching profiling on
  * resets the history.  ilre_recall_stage_times synchronises on those events and writes up to

@@ -65,6 +65,7 @@ struct ilre_recall {
   int* ranked;
   uint32_t* bitmap;
   int* status;
+  unsigned long long* clk;              // (cycles, ns) of the last profiled row-statistics launch
   // optional staging for the host entry point
   void* stage_k;
   void* stage_q;
@@ -134,7 +135,7 @@ void free_all(ilre_recall* h) {
   cudaFree(h->enc); cudaFree(h->scores); cudaFree(h->pooled); cudaFree(h->maxpooled); cudaFree(h->hist);
   cudaFree(h->tile_ties); cudaFree(h->grid_barrier); cudaFree(h->rope_table); cudaFree(h->pos_lo); cudaFree(h->pos_hi);
   cudaFree(h->cand); cudaFree(h->cand_count); cudaFree(h->ranked); cudaFree(h->bitmap);
-  cudaFree(h->status); cudaFree(h->stage_k); cudaFree(h->stage_q); cudaFree(h->stage_idx);
+  cudaFree(h->status); cudaFree(h->clk); cudaFree(h->stage_k); cudaFree(h->stage_q); cudaFree(h->stage_idx);
   cudaFree(h->piece_stats);
   if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
   if (h->copy_begin) cudaEventDestroy(h->copy_begin);
@@ -260,6 +261,7 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out) {
   ok = ok && dev_alloc(&h->ranked, ncomb * h->cand_stride);
   ok = ok && dev_alloc(&h->bitmap, (maxL + 31) / 32);
   ok = ok && dev_alloc(&h->status, 1);
+  ok = ok && dev_alloc(&h->clk, 2);
   if (ok && cfg->host_staging) {
     ok = ok && dev_alloc(reinterpret_cast<uint8_t**>(&h->stage_k), maxL * cfg->n_kv_heads * 256);
     ok = ok && dev_alloc(reinterpret_cast<uint8_t**>(&h->stage_q),
@@ -275,6 +277,7 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out) {
     for (int i = 0; ok && i <= kNumStages; ++i)
       ok = (cudaEventCreate(&h->ev[r][i]) == cudaSuccess);
   if (ok) ok = (cudaMemset(h->status, 0, sizeof(int)) == cudaSuccess);
+  if (ok) ok = (cudaMemset(h->clk, 0, 2 * sizeof(unsigned long long)) == cudaSuccess);
   if (ok) ok = (cudaMemset(h->grid_barrier, 0, sizeof(uint32_t)) == cudaSuccess);
   if (ok) ok = (select_max_grid(h->n_sm, &h->select_max_grid) == cudaSuccess);
   if (ok) ok = (cudaDeviceSynchronize() == cudaSuccess);
@@ -382,6 +385,7 @@ int recall_impl(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const void
   qk.rb_rows = g.rb_rows; qk.cpg = g.cpg; qk.stages = g.stages;
   qk.c2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(kHeadDim)));
   qk.partial = h->partial; qk.enc = h->enc; qk.status = h->status;
+  qk.clk = h->profiling ? h->clk : nullptr;
 
   PrepParams pp;
   std::memset(&pp, 0, sizeof(pp));
@@ -716,6 +720,17 @@ int ilre_recall_status(ilre_recall_t* h) {
   if (word != 0) ILRE_CUDA(cudaMemset(h->status, 0, sizeof(int)));
   if (word == 0) return ILRE_OK;
   return (word == kDevQuota) ? ILRE_ERR_QUOTA : ILRE_ERR_DEVICE_WAIT;
+}
+
+int ilre_recall_sm_clock(ilre_recall_t* h, float* mhz_out_host) {
+  if (!h || !mhz_out_host) return ILRE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return ILRE_ERR_CUDA;
+  ILRE_CUDA(cudaStreamSynchronize(h->last_stream));
+  unsigned long long w[2] = {0, 0};
+  ILRE_CUDA(cudaMemcpy(w, h->clk, sizeof(w), cudaMemcpyDeviceToHost));
+  *mhz_out_host = (w[1] > 0) ? static_cast<float>(1e3 * static_cast<double>(w[0]) / static_cast<double>(w[1])) : 0.f;
+  return ILRE_OK;
 }
 
 int ilre_recall_set_profiling(ilre_recall_t* h, int32_t on) {

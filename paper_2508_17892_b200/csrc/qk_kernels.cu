@@ -170,6 +170,13 @@ row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
 
   const uint32_t tmem_base = cta_setup(tail, smem_base, p.stages, 4, 4, p.status);
   const bool run = (it.n_tiles > 0) && (*abort_flag == 0);
+  const bool stamp = (p.clk != nullptr) && blockIdx.x == 0 && threadIdx.x == 0;
+  long long cyc0 = 0;
+  unsigned long long ns0 = 0;
+  if (stamp) {
+    cyc0 = clock64();
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns0));
+  }
 
   if (warp == 0) {
     if (lane == 0 && run) producer_loop(&tmapK, &tmapQ, p, it, tail, q_s, k_s);
@@ -289,6 +296,12 @@ row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
         out[mt * 128 + row_in_tile] = make_float2(mm * c2, zz);
       }
     }
+  }
+  if (stamp) {
+    unsigned long long ns1;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns1));
+    p.clk[0] = static_cast<unsigned long long>(clock64() - cyc0);
+    p.clk[1] = ns1 - ns0;
   }
   cta_teardown(tmem_base);
 }

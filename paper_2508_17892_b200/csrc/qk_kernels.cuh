@@ -44,6 +44,10 @@ struct QkParams {
   float* partial;    // [n_groups][cpg][rb_rows][2]: (max * c2, sum-exp) per key chunk
   uint32_t* enc;     // [L]: order-preserving uint of max_r log2 p_rt
   int* status;
+  // When non-null, CTA 0 of the row-statistics kernel stores how long it ran in SM cycles and
+  // in nanoseconds of the global timer: their ratio is the SM clock the kernel really ran at
+  // (under the power cap it is well below what the driver reports).
+  unsigned long long* clk;
 };
 
 struct PrepParams {

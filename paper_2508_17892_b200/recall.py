@@ -24,6 +24,7 @@ EXPORTED_SYMBOLS = (
     "ilre_layer_recall",
     "ilre_recall_copy_row_lse",
     "ilre_recall_status", "ilre_recall_set_profiling", "ilre_recall_stage_times",
+    "ilre_recall_sm_clock",
     "ilre_recall_last_launch_count", "ilre_recall_destroy", "ilre_strerror",
     "ilre_topk_positions_noalloc",
 )
@@ -78,6 +79,7 @@ def load_library() -> ctypes.CDLL:
     lib.ilre_layer_recall.argtypes = [vp, i32, i32, vp, vp, i32, vp, vp, vp, vp]
     lib.ilre_recall_copy_row_lse.argtypes = [vp, vp, i32, vp]
     lib.ilre_recall_status.argtypes = [vp]
+    lib.ilre_recall_sm_clock.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     lib.ilre_recall_set_profiling.argtypes = [vp, i32]
     lib.ilre_recall_stage_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float), i32]
     lib.ilre_recall_last_launch_count.argtypes = [vp]
@@ -380,6 +382,14 @@ class IlreRecall:
         if n < 0:
             raise IlreError(n, "ilre_recall_stage_times")
         return {STAGE_NAMES[i]: float(buf[i]) for i in range(n)}
+
+    def sm_clock_mhz(self) -> float:
+        """SM clock the row-statistics kernel of the last profiled run really ran at (0 = none)."""
+        mhz = ctypes.c_float(0.0)
+        rc = self._lib.ilre_recall_sm_clock(self._h, ctypes.byref(mhz))
+        if rc != 0:
+            raise IlreError(rc, "ilre_recall_sm_clock")
+        return float(mhz.value)
 
     def last_launch_count(self) -> int:
         return self._lib.ilre_recall_last_launch_count(self._h)

@@ -215,6 +215,18 @@ def test_run_host_pipelined_upload_matches_oracle(cases, name):
     eng.close()
 
 
+def test_in_kernel_sm_clock_is_plausible(cases):
+    x, _, _ = cases("cfg2_L32k")
+    eng = _engine(x.workload)
+    assert eng.sm_clock_mhz() == 0.0                      # nothing profiled yet
+    eng.set_profiling(True)
+    _run(eng, x)
+    mhz = eng.sm_clock_mhz()
+    eng.set_profiling(False)
+    assert 300.0 < mhz < 2500.0, mhz
+    eng.close()
+
+
 def test_error_codes_on_device(cases):
     from paper_2508_17892_b200 import IlreError
     x, _, _ = cases("cfg1_L4k")
