@@ -184,6 +184,28 @@ def dca_rerope(K, chunk: int, n_sink: int = 0, theta: float = 500000.0) -> np.nd
     return out
 
 
+def dca_rerope_sinks(K_sink, chunk_index: int, chunk: int, theta: float = 500000.0) -> np.ndarray:
+    """Eq. 6: the sink keys of a layer before the retrieval layer as the i-th chunk sees them,
+    K^{S,i} = R^{i-2}(D_C) K^S for i > 2 (1-based chunk index; the first two chunks see the
+    sinks as cached).  Written as the equation states it: the rotation by the chunk size D_C
+    applied i - 2 times to the cached sink keys, fp64, not rounded.  R(D) turns the channel
+    pair (c, c + d/2) by the angle D * theta^(-2c/d) (rotate-half layout, as in Eq. 7).
+
+    K_sink: bf16 [n_sink, n_kv, d].  Returns fp64 [n_sink, n_kv, d]."""
+    import torch
+    k = K_sink.to(torch.float64).numpy().copy()
+    d = k.shape[-1]
+    half = d // 2
+    c = np.arange(half, dtype=np.float64)
+    ang = float(chunk) * theta ** (-2.0 * c / d)
+    cs, sn = np.cos(ang), np.sin(ang)
+    for _ in range(max(0, int(chunk_index) - 2)):
+        lo, hi = k[..., :half].copy(), k[..., half:].copy()
+        k[..., :half] = lo * cs - hi * sn
+        k[..., half:] = lo * sn + hi * cs
+    return k
+
+
 def round_to_bf16(x: np.ndarray) -> np.ndarray:
     """Round fp64 values to the nearest bf16 (ties to even); returns the uint16 patterns."""
     import torch

@@ -105,3 +105,62 @@ def test_short_contexts_are_left_alone():
     for chunk in (50, 64, 100, 1000):              # N_C <= 2
         out = oracle.dca_rerope(K, chunk=chunk, n_sink=0, theta=ROPE_THETA)
         np.testing.assert_array_equal(out, K.to(torch.float64).numpy())
+
+
+# ---- Eq. 6: the sink keys of the layers before the retrieval layer ----
+
+def _complex_rotation(x, dist, theta=500000.0):
+    """Independent route: the pair (c, c + d/2) as a complex number times e^{i dist w_c}."""
+    d = x.shape[-1]
+    half = d // 2
+    w = theta ** (-2.0 * np.arange(half) / d)
+    z = (x[..., :half] + 1j * x[..., half:]) * np.exp(1j * dist * w)
+    return np.concatenate([z.real, z.imag], axis=-1)
+
+
+def test_sinks_first_two_chunks_see_the_cached_keys():
+    g = torch.Generator().manual_seed(3)
+    ks = torch.randn(4, 2, 128, generator=g).to(torch.bfloat16)
+    for i in (1, 2):
+        assert np.array_equal(oracle.dca_rerope_sinks(ks, i, 1024), ks.to(torch.float64).numpy())
+
+
+def test_sinks_power_of_the_rotation_is_one_rotation_by_the_summed_distance():
+    g = torch.Generator().manual_seed(4)
+    ks = torch.randn(4, 8, 128, generator=g).to(torch.bfloat16)
+    x = ks.to(torch.float64).numpy()
+    for i, chunk in ((3, 1024), (4, 1024), (7, 512), (40, 100)):
+        got = oracle.dca_rerope_sinks(ks, i, chunk)
+        ref = _complex_rotation(x, (i - 2) * chunk)
+        assert np.abs(got - ref).max() < 1e-9
+        # pair norms are kept
+        n0 = x[..., :64] ** 2 + x[..., 64:] ** 2
+        n1 = got[..., :64] ** 2 + got[..., 64:] ** 2
+        assert np.abs(n0 - n1).max() < 1e-9
+
+
+def test_sinks_hand_computed_quarter_turn():
+    # theta = 1 makes every pair turn by the distance itself; a chunk of pi/2 "positions"
+    # cannot be given (integer), so use d = 2, theta = 1, chunk = 1 and check against
+    # cos(1), sin(1) applied twice: (1, 0) -> (cos 2, sin 2)
+    ks = torch.tensor([[[1.0, 0.0]]]).to(torch.bfloat16)
+    got = oracle.dca_rerope_sinks(ks, 4, 1, theta=1.0)
+    assert np.allclose(got[0, 0], [np.cos(2.0), np.sin(2.0)], atol=1e-12)
+
+
+def test_sinks_keep_their_distance_to_the_chunk():
+    """What Eq. 6 is for: a sink key cached with RoPE at position s, seen from chunk i, sits
+    (i - 2) chunks further along, so its logit against a query at position p of chunk i equals
+    the logit of the un-rotated key against a query (i - 2) chunks earlier."""
+    g = torch.Generator().manual_seed(5)
+    raw_k = torch.randn(1, 1, 128, generator=g, dtype=torch.float64).numpy()
+    raw_q = torch.randn(128, generator=g, dtype=torch.float64).numpy()
+    s, chunk, i = 2, 256, 6
+    k_cached = _complex_rotation(raw_k, s)                       # RoPE at its own position
+    kb = torch.from_numpy(k_cached).to(torch.bfloat16)
+    k_i = oracle.dca_rerope_sinks(kb, i, chunk)[0, 0]
+    p = 4 + (i - 1) * chunk + 17                                  # some position in chunk i
+    q_p = _complex_rotation(raw_q[None], p)[0]
+    q_back = _complex_rotation(raw_q[None], p - (i - 2) * chunk)[0]
+    kb64 = kb.to(torch.float64).numpy()[0, 0]
+    assert abs(np.dot(q_p, k_i) - np.dot(q_back, kb64)) < 1e-9
