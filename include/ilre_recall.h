@@ -208,6 +208,23 @@ int ilre_recall_rerope_keys(ilre_recall_t* h, const void* k_cache_dev, void* k_o
                             void* cuda_stream);
 
 /*
+ * Dual Chunk Attention in the layers before the retrieval layer (Eq. 6): the sink keys as the
+ * prefill of chunk i sees them, K^{S,i} = R^{i-2}(D_C) K^S for i > 2 (chunk_index is 1-based;
+ * the first two chunks see the cached keys, which are then only copied).  The power of the
+ * rotation is applied as one rotation by (chunk_index - 2) * chunk_size positions to the
+ * CACHED sink keys (keep them; do not feed a rotated copy back in), so the result is rounded
+ * to bf16 once.  R(D) as in ilre_recall_rerope_keys.
+ *   k_sink_dev  bf16 [n_sink][n_kv_heads][128], 16-byte aligned; read only
+ *   k_out_dev   bf16 [n_sink][n_kv_heads][128]; may be k_sink_dev (in place)
+ * chunk_index <= 8194 (ILRE_ERR_CAPACITY beyond).  Shares the handle's angle table with
+ * ilre_recall_rerope_keys: calls on one handle must not overlap, and alternating between
+ * different chunk sizes rebuilds the table.  Asynchronous on cuda_stream.
+ */
+int ilre_recall_rerope_sinks(ilre_recall_t* h, const void* k_sink_dev, void* k_out_dev,
+                             int32_t n_sink, int32_t chunk_size, int32_t chunk_index,
+                             double rope_theta, void* cuda_stream);
+
+/*
  * The compressed prompt (Algorithm 1's last line, C~ = C[I], and Section 3.3's last step):
  *   out[i] = input_ids[idx[i]] for i < n_idx, then the n_query ids of the query part.
  * All pointers are int32 arrays on the current device; idx is what ilre_recall_run returned.

@@ -674,6 +674,42 @@ int ilre_recall_rerope_keys(ilre_recall_t* h, const void* k_cache_dev, void* k_o
   return ILRE_OK;
 }
 
+int ilre_recall_rerope_sinks(ilre_recall_t* h, const void* k_sink_dev, void* k_out_dev,
+                             int32_t n_sink, int32_t chunk_size, int32_t chunk_index,
+                             double rope_theta, void* cuda_stream) {
+  if (!h || !k_sink_dev || !k_out_dev || n_sink < 0 || chunk_size < 1 || chunk_index < 1 ||
+      !(rope_theta > 1.0))
+    return ILRE_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(k_sink_dev) & 15u) || (reinterpret_cast<uintptr_t>(k_out_dev) & 15u))
+    return ILRE_ERR_ALIGNMENT;
+  const long long turns = static_cast<long long>(chunk_index) - 2;     // power of R(D_C)
+  if (turns > kRopeTableRows) return ILRE_ERR_CAPACITY;
+  if (n_sink == 0 || (turns < 1 && k_out_dev == k_sink_dev)) return ILRE_OK;
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return ILRE_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  h->last_stream = st;
+  int launches = 0;
+  const float2* row = nullptr;
+  if (turns >= 1) {
+    // Table row r holds the distance (r + 1) * chunk.  Chunks arrive one after another, so
+    // the table is built ahead in powers of two rather than one row per call.
+    if (h->rope_chunk != chunk_size || h->rope_theta != rope_theta || h->rope_rows < turns) {
+      long long want = 64;
+      while (want < turns) want *= 2;
+      if (want > kRopeTableRows) want = kRopeTableRows;
+      ILRE_CUDA(launch_rope_table(h->rope_table, static_cast<int>(want), chunk_size, rope_theta, st));
+      h->rope_chunk = chunk_size; h->rope_theta = rope_theta; h->rope_rows = static_cast<int>(want);
+      ++launches;
+    }
+    row = h->rope_table + (turns - 1) * kRopeHalfDim;
+  }
+  ILRE_CUDA(launch_rotate_rows(static_cast<const uint4*>(k_sink_dev), static_cast<uint4*>(k_out_dev),
+                               static_cast<long long>(n_sink) * h->cfg.n_kv_heads, row, st));
+  h->last_launches = launches + 1;
+  return ILRE_OK;
+}
+
 int ilre_gather_input_ids(const int32_t* input_ids_dev, int64_t L, const int32_t* idx_dev,
                           int32_t n_idx, const int32_t* query_ids_dev, int32_t n_query,
                           int32_t* out_ids_dev, void* cuda_stream) {

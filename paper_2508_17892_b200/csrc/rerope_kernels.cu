@@ -87,6 +87,31 @@ rerope_kernel(const ReropeParams p) {
   }
 }
 
+// Eq. 6: K^{S,i} = R^{i-2}(D_C) K^S, the sink keys of a layer before the retrieval layer as
+// chunk i > 2 sees them.  The power of the rotation is one rotation by (i - 2) * D_C, taken
+// from the cached (never re-rotated) sink keys, so the keys are rounded once however large i is.
+// `cs` is the table row of that distance.  A few KB: one item per thread.
+__global__ void rotate_rows_kernel(const uint4* __restrict__ k_in, uint4* __restrict__ k_out,
+                                   long long n_items, const float2* __restrict__ cs) {
+  const long long item = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (item >= n_items) return;
+  const long long row = item >> 3;
+  const int seg = static_cast<int>(item & 7);
+  uint4 lo = k_in[row * 16 + seg], hi = k_in[row * 16 + 8 + seg];
+  if (cs) rotate8(lo, hi, cs + seg * 8);
+  k_out[row * 16 + seg] = lo;
+  k_out[row * 16 + 8 + seg] = hi;
+}
+
+cudaError_t launch_rotate_rows(const uint4* k_in, uint4* k_out, long long n_rows,
+                               const float2* table_row, cudaStream_t st) {
+  const long long n_items = n_rows * 8;
+  if (n_items < 1) return cudaSuccess;
+  rotate_rows_kernel<<<static_cast<unsigned>((n_items + 255) / 256), 256, 0, st>>>(k_in, k_out, n_items,
+                                                                                  table_row);
+  return cudaGetLastError();
+}
+
 // Algorithm 1's last step and the hand-over to the inference engine: the compressed prompt is
 // the input ids at the chosen positions followed by the ids of the query part.
 __global__ void gather_ids_kernel(const int32_t* __restrict__ ids, long long L,

@@ -25,6 +25,11 @@ cudaError_t launch_rope_table(float2* table, int n_rows, int chunk, double theta
 // K~ = R(D_i) K for the chunks before the last two; the last two are copied when out != in.
 cudaError_t launch_rerope(const ReropeParams& p, int n_sm, cudaStream_t st);
 
+// Every (row, kv head) vector of k_in [n_rows][128] turned by the distance of `table_row`
+// ([64] (cos, sin)); a null row copies.  k_out may alias k_in.
+cudaError_t launch_rotate_rows(const uint4* k_in, uint4* k_out, long long n_rows,
+                               const float2* table_row, cudaStream_t st);
+
 // out = ids[idx[0..n_idx)] followed by query_ids[0..n_query)
 cudaError_t launch_gather_ids(const int32_t* ids, long long L, const int32_t* idx, int n_idx,
                               const int32_t* query_ids, int n_query, int32_t* out,

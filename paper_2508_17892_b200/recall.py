@@ -20,7 +20,8 @@ STAGE_NAMES = ("prepare", "row_stats", "scores", "select")
 EXPORTED_SYMBOLS = (
     "ilre_recall_create", "ilre_recall_run", "ilre_recall_run_host", "ilre_recall_fill_keys",
     "ilre_recall_shard_stats", "ilre_recall_shard_scores", "ilre_recall_allocate",
-    "ilre_recall_chunk_attention", "ilre_recall_rerope_keys", "ilre_gather_input_ids",
+    "ilre_recall_chunk_attention", "ilre_recall_rerope_keys", "ilre_recall_rerope_sinks",
+    "ilre_gather_input_ids",
     "ilre_layer_recall",
     "ilre_recall_copy_row_lse",
     "ilre_recall_status", "ilre_recall_set_profiling", "ilre_recall_stage_times",
@@ -75,6 +76,7 @@ def load_library() -> ctypes.CDLL:
     lib.ilre_recall_chunk_attention.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp]
     lib.ilre_recall_fill_keys.argtypes = [vp, vp, i64, i32, vp, vp, i64, ctypes.c_double, vp, i64, vp]
     lib.ilre_recall_rerope_keys.argtypes = [vp, vp, vp, i64, i32, i32, ctypes.c_double, vp]
+    lib.ilre_recall_rerope_sinks.argtypes = [vp, vp, vp, i32, i32, i32, ctypes.c_double, vp]
     lib.ilre_gather_input_ids.argtypes = [vp, i64, vp, i32, vp, i32, vp, vp]
     lib.ilre_layer_recall.argtypes = [vp, i32, i32, vp, vp, i32, vp, vp, vp, vp]
     lib.ilre_recall_copy_row_lse.argtypes = [vp, vp, i32, vp]
@@ -354,6 +356,25 @@ class IlreRecall:
                                                st.cuda_stream)
         if rc != 0:
             raise IlreError(rc, "ilre_recall_rerope_keys")
+        return dst
+
+    def rerope_sinks(self, K_sink: torch.Tensor, chunk_size: int, chunk_index: int,
+                     rope_theta: float = 500000.0, out: Optional[torch.Tensor] = None,
+                     stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        """Eq. 6: the cached sink keys [n_sink, n_kv_heads, 128] as the prefill of chunk
+        ``chunk_index`` (1-based) sees them.  Pass the cached keys every time, not an earlier
+        result.  Returns a new tensor unless ``out`` is given (``out`` may be ``K_sink``)."""
+        dst = torch.empty_like(K_sink) if out is None else out
+        for t in (K_sink, dst):
+            assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+            assert t.shape[1:] == (self.cfg.n_kv_heads, self.cfg.head_dim)
+        assert dst.shape == K_sink.shape
+        st = stream if stream is not None else torch.cuda.current_stream(self.device)
+        rc = self._lib.ilre_recall_rerope_sinks(self._h, K_sink.data_ptr(), dst.data_ptr(),
+                                                K_sink.shape[0], chunk_size, chunk_index,
+                                                float(rope_theta), st.cuda_stream)
+        if rc != 0:
+            raise IlreError(rc, "ilre_recall_rerope_sinks")
         return dst
 
     # -- diagnostics -------------------------------------------------------------------

@@ -110,3 +110,62 @@ def test_recall_on_rerotated_keys_matches_oracle():
     planted = set(x.planted_positions().tolist())
     assert len(planted & set(idx.cpu().tolist())) == len(planted & set(ref_idx.tolist()))
     eng.close()
+
+
+# ---- Eq. 6: sink keys of the layers before the retrieval layer ----
+
+SINK_CASES = [
+    # n_sink, n_kv, chunk, chunk_index
+    (4, 8, 1024, 1), (4, 8, 1024, 2), (4, 8, 1024, 3), (4, 8, 1024, 4), (4, 8, 1024, 1024),
+    (1, 2, 64, 7), (64, 4, 512, 100), (4, 8, 8, 8194),
+]
+
+
+@pytest.mark.parametrize("case", SINK_CASES, ids=lambda c: f"S{c[0]}_kv{c[1]}_c{c[2]}_i{c[3]}")
+def test_sink_rerope_matches_oracle(case):
+    n_sink, n_kv, chunk, i = case
+    g = torch.Generator().manual_seed(100 + i)
+    ks = (4.0 * torch.randn(n_sink, n_kv, 128, generator=g)).to(torch.bfloat16)
+    eng = _engine(n_kv=n_kv, n_q=n_kv)
+    ref = oracle.dca_rerope_sinks(ks, i, chunk)
+    src = ks.cuda()
+    out = eng.rerope_sinks(src, chunk, i)
+    torch.cuda.synchronize()
+    eng.check_status()
+    assert torch.equal(src.cpu(), ks)                       # the cached keys are left alone
+    got = _as_f64(out)
+    if i <= 2:
+        assert np.array_equal(got, ref)
+    else:
+        assert np.all(np.abs(got - ref) <= REL_TOL * np.abs(ref) + ABS_TOL)
+        assert not np.array_equal(got, _as_f64(ks))
+    # in place gives the same bytes
+    inplace = ks.cuda()
+    eng.rerope_sinks(inplace, chunk, i, out=inplace)
+    torch.cuda.synchronize()
+    assert torch.equal(inplace, out)
+    eng.close()
+
+
+def test_sink_rerope_chunk_by_chunk_and_with_eq7_on_one_handle():
+    """Chunks arrive in order (the angle table grows ahead of them); Eq. 7 on the same handle
+    in between, with another chunk size, must not disturb later calls."""
+    from paper_2508_17892_b200 import IlreError
+    g = torch.Generator().manual_seed(9)
+    ks = torch.randn(4, 8, 128, generator=g).to(torch.bfloat16)
+    eng = _engine()
+    src = ks.cuda()
+    for i in list(range(1, 140)) + [70, 3]:
+        got = _as_f64(eng.rerope_sinks(src, 256, i))
+        ref = oracle.dca_rerope_sinks(ks, i, 256)
+        assert np.all(np.abs(got - ref) <= REL_TOL * np.abs(ref) + ABS_TOL), i
+        if i == 100:
+            x = make_inputs(small_workload(3000, 1, seed=5))
+            eng.rerope_keys(x.K.cuda(), 500, 0)
+    with pytest.raises(IlreError):
+        eng.rerope_sinks(src, 256, 8195)                     # beyond the angle table
+    with pytest.raises(IlreError):
+        eng.rerope_sinks(src, 256, 0)
+    torch.cuda.synchronize()
+    eng.check_status()
+    eng.close()
