@@ -82,6 +82,8 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out);
  *   budget        B, 0 <= B <= L - n_sink
  *   out_idx_dev   int32 [n_sink + budget]: chosen context positions, ascending
  *   out_scores_dev  optional fp32 [L]: A^C of Eq. 5 (NULL to skip)
+ * The call only encodes two tensor maps on the host and launches kernels on cuda_stream (no
+ * allocation, no synchronisation), so it may be captured into a CUDA graph and replayed.
  * Ranking inside a combination is (pooled value descending, cell index ascending); K_m =
  * B/m + 1 (+1 when L - n_sink is not a multiple of m), B_c = B/N_c with the remainder given
  * to the first combinations in loop order (max sizes outer, window sizes inner).

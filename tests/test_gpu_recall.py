@@ -215,6 +215,34 @@ def test_run_host_pipelined_upload_matches_oracle(cases, name):
     eng.close()
 
 
+def test_recall_can_be_captured_in_a_cuda_graph(cases):
+    """run() allocates nothing, never synchronises and only launches kernels (one of them
+    cooperative): it can be captured once and replayed, e.g. to shave launch overhead off short
+    contexts.  The replay must give what the direct call gives."""
+    x, _, _ = cases("cfg2_L32k")
+    w = x.workload
+    eng = _engine(w)
+    K, Q = x.K.cuda(), x.Q.cuda()
+    out = torch.empty(w.n_sink + w.budget, dtype=torch.int32, device="cuda")
+    spec = (w.budget, w.max_sizes, w.win_sizes, w.win_op, w.n_sink)
+    eng.run(K, Q, *spec, out_idx=out)
+    torch.cuda.synchronize()
+    direct = out.clone()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            eng.run(K, Q, *spec, out_idx=out, stream=side)
+    for _ in range(3):
+        out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, direct)
+    eng.check_status()
+    del graph
+    eng.close()
+
+
 def test_in_kernel_sm_clock_is_plausible(cases):
     x, _, _ = cases("cfg2_L32k")
     eng = _engine(x.workload)
