@@ -19,6 +19,9 @@ static constexpr int kConsumerWarps = 8;
 #define ILRE_STATS_WARPGROUPS 4
 #endif
 static constexpr int kStatsWarpgroups = ILRE_STATS_WARPGROUPS;
+// A warpgroup's first accumulator must be one of the first four (the number of TMEM buffers):
+// a parity wait on a buffer that has not completed its first phase yet would pass at once.
+static_assert(kStatsWarpgroups >= 1 && kStatsWarpgroups <= 4, "at most one warpgroup per TMEM buffer");
 static constexpr int kStatsConsumerWarps = 4 * kStatsWarpgroups;
 static constexpr int kStatsThreads = 64 + 32 * kStatsConsumerWarps;
 static constexpr int kSmemTailBytes = 256;
