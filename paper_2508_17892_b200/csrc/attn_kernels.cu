@@ -127,78 +127,82 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
         tma_load_2d(ring_s + s * kAttnTileBytes + 16384, map, g * 128 + 64, t * 128, bar);
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == 1 || warp == 2) {
+    // Two MMA-issuing threads.  tcgen05.mma holds its issuing thread until the tensor pipe
+    // takes the instruction, so one thread alone leaves the pipe idle whenever it tests
+    // barriers or commits.  Warp 1 issues every S = Q K^T (both streams), warp 2 every
+    // O += P V; each polls its two streams' barriers without blocking and issues whichever is
+    // ready, and the bookkeeping of one overlaps the MMAs of the other.  A key tile's ring
+    // slot is released by the S issuer, a value tile's by the PV issuer, once both streams
+    // have issued the MMAs that read it.
     if (lane == 0 && run) {
       constexpr uint32_t idesc_s = umma_idesc_bf16(128, 128);
       constexpr uint32_t idesc_o = umma_idesc_bf16(128, 128) | (1u << 16);   // B = V: channels contiguous
-      bool ok = mbar_wait(smem_u32(&tail->q_full), 0, abort_flag, p.status, kDevWaitQFull);
-      tc_fence_after();
+      const bool s_role = (warp == 1);
       auto k_item = [&](int t) -> int { return t == 0 ? 0 : 2 * t - 1; };
       auto v_item = [&](int t) -> int { return t < n_tiles - 1 ? 2 * t + 2 : 2 * n_tiles - 1; };
-      auto issue_s = [&](int x, int t) {                  // S_x = Q_x K_t^T
-        const uint32_t k_s = ring_s + (k_item(t) % kAttnStages) * kAttnTileBytes;
-        const uint32_t qx = q_s + x * kAttnTileBytes;
-#pragma unroll
-        for (int kb = 0; kb < 2; ++kb)
-#pragma unroll
-          for (int ks = 0; ks < 4; ++ks)
-            umma_bf16(tmem_base + x * 128, umma_desc_sw128(qx + kb * 16384 + ks * 32),
-                      umma_desc_sw128(k_s + kb * 16384 + ks * 32), idesc_s, (kb | ks) != 0);
-        umma_commit(smem_u32(&tail->s_full[x]));
-      };
-      // Event-driven issue: per stream the next S = Q K^T (needs the softmax warps to have
-      // taken the previous S out of tensor memory, and the key tile) and the next
-      // O += P V (needs P and the value tile); whichever is ready goes first, so neither
-      // stream ever waits for the other's softmax.  A ring slot is released once both
-      // streams have issued the MMAs that read it.
       auto ring_ready = [&](int item) -> bool {
         return mbar_test_wait(smem_u32(&tail->kv_full[item % kAttnStages]),
                               static_cast<uint32_t>(item / kAttnStages) & 1u);
       };
-      int next_s[2] = {0, 0}, next_pv[2] = {0, 0};
-      if (n_streams == 1) next_s[1] = next_pv[1] = n_tiles;
-      int k_released = 0, v_released = 0;
+      bool ok = true;
+      if (s_role) {
+        ok = mbar_wait(smem_u32(&tail->q_full), 0, abort_flag, p.status, kDevWaitQFull);
+        tc_fence_after();
+      }
+      int next[2] = {0, 0};                               // per stream: next tile to issue
+      if (n_streams == 1) next[1] = n_tiles;
+      int released = 0;
       long long t_idle = 0;
       uint32_t spins = 0;
-      while (ok && (next_pv[0] < n_tiles || next_pv[1] < n_tiles)) {
+      while (ok && (next[0] < n_tiles || next[1] < n_tiles)) {
         bool progress = false;
-        // O += P V first: it frees the stream's P buffer, which its softmax warps need soonest
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
-          const int t = next_pv[x];
-          if (t < n_tiles && t < next_s[x] && ring_ready(v_item(t)) &&
-              mbar_test_wait(smem_u32(&tail->p_full[x]), static_cast<uint32_t>(t) & 1u)) {
-            tc_fence_after();
-            const uint32_t v_s = ring_s + (v_item(t) % kAttnStages) * kAttnTileBytes;
-            const uint32_t px = p_s + x * kAttnTileBytes;
+          const int t = next[x];
+          if (t >= n_tiles) continue;
+          if (s_role) {
+            // S_x(t): needs the key tile and, after the first, S_x(t-1) read out of tensor memory
+            if (ring_ready(k_item(t)) &&
+                (t == 0 || mbar_test_wait(smem_u32(&tail->s_empty[x]), static_cast<uint32_t>(t - 1) & 1u))) {
+              tc_fence_after();
+              const uint32_t k_s = ring_s + (k_item(t) % kAttnStages) * kAttnTileBytes;
+              const uint32_t qx = q_s + x * kAttnTileBytes;
 #pragma unroll
-            for (int kb = 0; kb < 2; ++kb)
+              for (int kb = 0; kb < 2; ++kb)
 #pragma unroll
-              for (int ks = 0; ks < 4; ++ks)
-                umma_bf16(tmem_base + 256 + x * 128, umma_desc_sw128(px + kb * 16384 + ks * 32),
-                          umma_desc_sw128_mn(v_s + (kb * 64 + ks * 16) * 128, 16384, 1024), idesc_o,
-                          (t | kb | ks) != 0);
-            umma_commit(smem_u32(&tail->p_empty[x]));
-            next_pv[x] = t + 1;
-            progress = true;
-            while (v_released < min(next_pv[0], next_pv[1])) {
-              umma_commit(smem_u32(&tail->kv_empty[v_item(v_released) % kAttnStages]));
-              ++v_released;
+                for (int ks = 0; ks < 4; ++ks)
+                  umma_bf16(tmem_base + x * 128, umma_desc_sw128(qx + kb * 16384 + ks * 32),
+                            umma_desc_sw128(k_s + kb * 16384 + ks * 32), idesc_s, (kb | ks) != 0);
+              umma_commit(smem_u32(&tail->s_full[x]));
+              next[x] = t + 1;
+              progress = true;
+              while (released < min(next[0], next[1])) {
+                umma_commit(smem_u32(&tail->kv_empty[k_item(released) % kAttnStages]));
+                ++released;
+              }
             }
-          }
-        }
+          } else {
+            // O_x += P_x(t) V_t: needs P written and the value tile
+            if (mbar_test_wait(smem_u32(&tail->p_full[x]), static_cast<uint32_t>(t) & 1u) &&
+                ring_ready(v_item(t))) {
+              tc_fence_after();
+              const uint32_t v_s = ring_s + (v_item(t) % kAttnStages) * kAttnTileBytes;
+              const uint32_t px = p_s + x * kAttnTileBytes;
 #pragma unroll
-        for (int x = 0; x < 2; ++x) {
-          const int t = next_s[x];
-          if (t < n_tiles && ring_ready(k_item(t)) &&
-              (t == 0 || mbar_test_wait(smem_u32(&tail->s_empty[x]), static_cast<uint32_t>(t - 1) & 1u))) {
-            tc_fence_after();
-            issue_s(x, t);
-            next_s[x] = t + 1;
-            progress = true;
-            while (k_released < min(next_s[0], next_s[1])) {
-              umma_commit(smem_u32(&tail->kv_empty[k_item(k_released) % kAttnStages]));
-              ++k_released;
+              for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                  umma_bf16(tmem_base + 256 + x * 128, umma_desc_sw128(px + kb * 16384 + ks * 32),
+                            umma_desc_sw128_mn(v_s + (kb * 64 + ks * 16) * 128, 16384, 1024), idesc_o,
+                            (t | kb | ks) != 0);
+              umma_commit(smem_u32(&tail->p_empty[x]));
+              next[x] = t + 1;
+              progress = true;
+              while (released < min(next[0], next[1])) {
+                umma_commit(smem_u32(&tail->kv_empty[v_item(released) % kAttnStages]));
+                ++released;
+              }
             }
           }
         }
@@ -218,13 +222,13 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
           }
         }
       }
-      if (ok) umma_commit(smem_u32(&tail->o_full));
+      if (ok && !s_role) umma_commit(smem_u32(&tail->o_full));
     }
-  } else if ((warp - 2) / kAttnSoftmaxWarps < n_streams) {
+  } else if (warp >= 3 && (warp - 3) / kAttnSoftmaxWarps < n_streams) {
     // Softmax warps of stream x: warp w reads TMEM lane quadrant w % 4, so a thread owns one
     // query row: its 128 logits of the tile, its running reference and sum, its row of P and
     // of O.  No thread ever needs another's values.
-    const int x = (warp - 2) / kAttnSoftmaxWarps;
+    const int x = (warp - 3) / kAttnSoftmaxWarps;
     const int quad = warp & 3;
     const int row = quad * 32 + lane;
     const int qj = j0 + row;

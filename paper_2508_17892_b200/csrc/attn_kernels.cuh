@@ -8,7 +8,7 @@
 
 namespace ilre {
 
-static constexpr int kAttnThreads = 320;     // warp 0 TMA, warp 1 MMA, warps 2..5 / 6..9 softmax
+static constexpr int kAttnThreads = 352;     // warp 0 TMA, warp 1 S MMAs, warp 2 PV MMAs, warps 3..6 / 7..10 softmax
 
 struct AttnParams {
   int c;             // query tokens of the chunk
