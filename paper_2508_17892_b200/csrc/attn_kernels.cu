@@ -22,6 +22,10 @@ namespace ilre {
 static constexpr int kAttnStages = 3;
 static constexpr int kAttnTileBytes = 128 * 128 * 2;       // one 128 x 128 bf16 tile
 static constexpr int kAttnTailBytes = 256;
+#ifndef ILRE_ATTN_POLY_PAIRS
+#define ILRE_ATTN_POLY_PAIRS 2
+#endif
+static constexpr int kAttnPolyPairs = ILRE_ATTN_POLY_PAIRS;   // of every 16 pairs of exponentials
 static constexpr int kAttnSoftmaxWarps = 4;                // per stream: one per TMEM lane quadrant
 
 struct AttnTail {
@@ -297,7 +301,11 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
         for (int i = 0; i < 32; i += 2) {
           const float2 a = ffma2(make_float2(V(g32 * 32 + i), V(g32 * 32 + i + 1)), make_float2(c2, c2),
                                  make_float2(nr, nr));
-          const float2 pp = make_float2(ex2_approx(a.x), ex2_approx(a.y));
+          // kAttnPolyPairs of every 16 pairs take 2^x from the FMA-pipe polynomial: the two
+          // streams share each scheduler's special-function unit, which is the busiest pipe
+          const int pr16 = i >> 1;
+          const bool poly = ((pr16 + 1) * kAttnPolyPairs) / 16 > (pr16 * kAttnPolyPairs) / 16;
+          const float2 pp = poly ? exp2_poly2(a) : make_float2(ex2_approx(a.x), ex2_approx(a.y));
           sum2 = fadd2(sum2, pp);
           const __nv_bfloat162 pr = __floats2bfloat162_rn(pp.x, pp.y);
           w[i >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
