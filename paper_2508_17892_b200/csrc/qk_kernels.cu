@@ -44,7 +44,8 @@ __device__ __forceinline__ CtaItem decode_item(const QkParams& p) {
 
 // Common prologue: barrier init, TMEM allocation.  Returns the TMEM base address.
 __device__ __forceinline__ uint32_t cta_setup(SmemTail* tail, uint32_t smem_base, int stages,
-                                              int n_acc, int acc_readers, int* status) {
+                                              int n_acc, int acc_readers, int* status,
+                                              int k_releasers = 1) {
   const int warp = threadIdx.x >> 5;
   if (threadIdx.x == 0) {
     tail->abort_flag = 0;
@@ -55,7 +56,7 @@ __device__ __forceinline__ uint32_t cta_setup(SmemTail* tail, uint32_t smem_base
     mbar_init(smem_u32(&tail->q_full), 1);
     for (int s = 0; s < stages; ++s) {
       mbar_init(smem_u32(&tail->k_full[s]), 1);
-      mbar_init(smem_u32(&tail->k_empty[s]), 1);
+      mbar_init(smem_u32(&tail->k_empty[s]), k_releasers);
     }
     for (int b = 0; b < n_acc; ++b) {
       mbar_init(smem_u32(&tail->acc_full[b]), 1);
@@ -385,17 +386,26 @@ scores_kernel(const __grid_constant__ CUtensorMap tmapK,
   // CTAs of the first key chunk also publish the natural-log lse.
   for (int i = threadIdx.x; i < p.rb_rows; i += blockDim.x)
     nl[i] = merged_neg_lse2(mp, it.group, i, it.chunk == 0);
-  const uint32_t tmem_base = cta_setup(tail, smem_base, p.stages, 2, kConsumerWarps, p.status);
+  // Two MMA-issuing threads (warps 1 and 2), one per accumulator buffer: tcgen05.mma holds its
+  // issuing thread until the tensor pipe takes the instruction, so the waits and commits of
+  // one thread overlap the MMAs of the other.  With two row halves per key tile each thread
+  // issues one half of every tile and both release the tile's stage; with one, the threads
+  // take the tiles in turn.
+  const int k_releasers = (n_nh >= 2) ? 2 : 1;
+  const uint32_t tmem_base = cta_setup(tail, smem_base, p.stages, 2, kConsumerWarps, p.status,
+                                       k_releasers);
   const bool run = (it.n_tiles > 0) && (*abort_flag == 0);
 
   if (warp == 0) {
     if (lane == 0 && run) producer_loop(&tmapK, &tmapQ, p, it, tail, q_s, k_s);
-  } else if (warp == 1) {
+  } else if (warp == 1 || warp == 2) {
     if (lane == 0 && run) {
+      const uint32_t mine = static_cast<uint32_t>(warp - 1);          // accumulator buffer
       bool ok = mbar_wait(smem_u32(&tail->q_full), 0, abort_flag, p.status, kDevWaitQFull);
       tc_fence_after();
       uint32_t u = 0;
       for (int i = 0; i < it.n_tiles && ok; ++i) {
+        if (n_nh == 1 && ((static_cast<uint32_t>(i) & 1u) != mine)) { ++u; continue; }
         const int s = i % p.stages;
         const uint32_t kuse = static_cast<uint32_t>(i / p.stages);
         ok = mbar_wait(smem_u32(&tail->k_full[s]), kuse & 1u, abort_flag, p.status,
@@ -403,6 +413,7 @@ scores_kernel(const __grid_constant__ CUtensorMap tmapK,
         if (!ok) break;
         tc_fence_after();
         for (int nh = 0; nh < n_nh; ++nh, ++u) {
+          if ((u & 1u) != mine) continue;
           const int N = min(256, p.rb_rows - nh * 256);
           const uint32_t idesc = umma_idesc_bf16(128, N);
           const uint32_t b = u & 1u, use = u >> 1;

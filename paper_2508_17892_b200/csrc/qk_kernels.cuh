@@ -11,7 +11,7 @@ static constexpr int kTileKeys = 128;              // keys per K tile (one TMA s
 static constexpr int kStageBytes = kTileKeys * kHeadDim * 2;
 static constexpr int kMaxStages = 6;
 static constexpr int kMaxRbRows = 512;             // query rows resident in shared memory
-static constexpr int kQkThreads = 384;             // scores: warp 0 TMA, warp 1 MMA, warps 4..11 consumers
+static constexpr int kQkThreads = 384;             // scores: warp 0 TMA, warps 1-2 MMA, warps 4..11 consumers
 static constexpr int kConsumerWarps = 8;
 // Row statistics: warp 0 TMA, warp 1 MMA, then kStatsWarpgroups consumer warpgroups of four
 // warps (one per TMEM lane quadrant); accumulator buffer u belongs to warpgroup u % kStatsWarpgroups.
