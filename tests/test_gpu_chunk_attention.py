@@ -21,6 +21,8 @@ CASES = [
     (256, 128, 4, 2),          # prefix of exactly one tile
     (1024, 516, 32, 8),        # the paper's defaults: chunk 1024, sink 4 + window 512
     (300, 1000, 4, 4),         # long prefix, no grouping
+    (200, 130, 28, 4),         # seven query heads per kv head: one head per CTA
+    (2048, 516, 8, 2),         # 16 query tiles, up to 21 key tiles: the K/V ring wraps many times
 ]
 
 
