@@ -91,15 +91,16 @@ fill_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ C
 
   if (warp == 0) {
     if (lane == 0 && run) {
-      uint32_t it = 0;
+      // ring position kept as (stage, phase) counters: a division by the run-time stage count
+      // per 64-channel block would cost this thread more than the block's TMA issue
+      int s = 0;
+      uint32_t phase = 0;
       for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
         const int m0 = static_cast<int>(tile / n_ntiles) * kFillTileM;
         const int n0 = static_cast<int>(tile % n_ntiles) * NT;
         bool ok = true;
-        for (int kb = 0; kb < k_blocks && ok; ++kb, ++it) {
-          const int s = it % p.stages;
-          const uint32_t use = it / p.stages;
-          ok = mbar_wait(smem_u32(&tail->empty[s]), (use & 1u) ^ 1u, abort_flag, p.status,
+        for (int kb = 0; kb < k_blocks && ok; ++kb) {
+          ok = mbar_wait(smem_u32(&tail->empty[s]), phase ^ 1u, abort_flag, p.status,
                          kDevWaitKEmpty);
           if (!ok) break;
           const uint32_t bar = smem_u32(&tail->full[s]);
@@ -107,6 +108,7 @@ fill_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ C
           const uint32_t dst = smem_base + s * kStageBytes;
           tma_load_2d(dst, &map_x, kb * kFillBlockK, m0, bar);
           tma_load_2d(dst + kStageBytesA, &map_w, kb * kFillBlockK, n0, bar);
+          if (++s == p.stages) { s = 0; phase ^= 1u; }
         }
         if (!ok) break;
       }
@@ -114,7 +116,11 @@ fill_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ C
   } else if (warp == 1) {
     if (lane == 0 && run) {
       constexpr uint32_t idesc = umma_idesc_bf16(kFillTileM, NT);
-      uint32_t it = 0, local = 0;
+      // (stage, phase) counters instead of a division per block: the tensor pipe idles while
+      // this thread does anything but issue
+      uint32_t local = 0;
+      int s = 0;
+      uint32_t phase = 0;
       bool ok = true;
       for (long long tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++local) {
         const uint32_t buf = local & 1u, use = local >> 1;
@@ -122,10 +128,8 @@ fill_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ C
                        kDevWaitAccEmpty);
         if (!ok) break;
         tc_fence_after();
-        for (int kb = 0; kb < k_blocks; ++kb, ++it) {
-          const int s = it % p.stages;
-          const uint32_t kuse = it / p.stages;
-          ok = mbar_wait(smem_u32(&tail->full[s]), kuse & 1u, abort_flag, p.status, kDevWaitKFull);
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          ok = mbar_wait(smem_u32(&tail->full[s]), phase, abort_flag, p.status, kDevWaitKFull);
           if (!ok) break;
           tc_fence_after();
           const uint32_t a0 = smem_base + s * kStageBytes;
@@ -134,6 +138,7 @@ fill_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ C
             umma_bf16(tmem_base + buf * NT, umma_desc_sw128(a0 + ks * 32),
                       umma_desc_sw128(a0 + kStageBytesA + ks * 32), idesc, (kb | ks) != 0);
           umma_commit(smem_u32(&tail->empty[s]));
+          if (++s == p.stages) { s = 0; phase ^= 1u; }
         }
         if (ok) umma_commit(smem_u32(&tail->acc_full[buf]));
       }
