@@ -94,17 +94,18 @@ __device__ __forceinline__ void producer_loop(const CUtensorMap* tmapK, const CU
     for (int mt = 0; mt < p.rb_rows / 128; ++mt)
       tma_load_2d(q_s + kb * p.rb_rows * 128 + mt * 16384, tmapQ, kb * 64,
                   it.group * p.rb_rows + mt * 128, qf);
+  // ring position as (stage, phase) counters: no division by the run-time stage count
+  int s = 0;
+  uint32_t phase = 0;
   for (int i = 0; i < it.n_tiles; ++i) {
-    const int s = i % p.stages;
-    const uint32_t use = static_cast<uint32_t>(i / p.stages);
-    if (!mbar_wait(smem_u32(&tail->k_empty[s]), (use & 1u) ^ 1u, abort_flag, p.status,
-                   kDevWaitKEmpty))
+    if (!mbar_wait(smem_u32(&tail->k_empty[s]), phase ^ 1u, abort_flag, p.status, kDevWaitKEmpty))
       break;
     const uint32_t kf = smem_u32(&tail->k_full[s]);
     mbar_arrive_expect_tx(kf, kStageBytes);
     const int row = (it.tile_begin + i) * kTileKeys;
     tma_load_2d(k_s + s * kStageBytes, tmapK, it.g * 128, row, kf);
     tma_load_2d(k_s + s * kStageBytes + 16384, tmapK, it.g * 128 + 64, row, kf);
+    if (++s == p.stages) { s = 0; phase ^= 1u; }
   }
 }
 
@@ -187,11 +188,10 @@ row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
       bool ok = mbar_wait(smem_u32(&tail->q_full), 0, abort_flag, p.status, kDevWaitQFull);
       tc_fence_after();
       uint32_t u = 0;
+      int s = 0;
+      uint32_t kphase = 0;
       for (int i = 0; i < it.n_tiles && ok; ++i) {
-        const int s = i % p.stages;
-        const uint32_t kuse = static_cast<uint32_t>(i / p.stages);
-        ok = mbar_wait(smem_u32(&tail->k_full[s]), kuse & 1u, abort_flag, p.status,
-                       kDevWaitKFull);
+        ok = mbar_wait(smem_u32(&tail->k_full[s]), kphase, abort_flag, p.status, kDevWaitKFull);
         if (!ok) break;
         tc_fence_after();
         for (int mt = 0; mt < MT; ++mt, ++u) {
@@ -211,6 +211,7 @@ row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
           umma_commit(smem_u32(&tail->acc_full[b]));
         }
         umma_commit(smem_u32(&tail->k_empty[s]));
+        if (++s == p.stages) { s = 0; kphase ^= 1u; }
       }
     }
   } else if (warp >= 2) {
@@ -404,12 +405,13 @@ scores_kernel(const __grid_constant__ CUtensorMap tmapK,
       bool ok = mbar_wait(smem_u32(&tail->q_full), 0, abort_flag, p.status, kDevWaitQFull);
       tc_fence_after();
       uint32_t u = 0;
+      int s = -1;
+      uint32_t kphase = 1;
       for (int i = 0; i < it.n_tiles && ok; ++i) {
+        if (++s == p.stages) s = 0;                      // stage and phase of key tile i
+        if (s == 0) kphase ^= 1u;
         if (n_nh == 1 && ((static_cast<uint32_t>(i) & 1u) != mine)) { ++u; continue; }
-        const int s = i % p.stages;
-        const uint32_t kuse = static_cast<uint32_t>(i / p.stages);
-        ok = mbar_wait(smem_u32(&tail->k_full[s]), kuse & 1u, abort_flag, p.status,
-                       kDevWaitKFull);
+        ok = mbar_wait(smem_u32(&tail->k_full[s]), kphase, abort_flag, p.status, kDevWaitKFull);
         if (!ok) break;
         tc_fence_after();
         for (int nh = 0; nh < n_nh; ++nh, ++u) {
