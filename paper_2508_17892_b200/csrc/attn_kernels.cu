@@ -5,9 +5,11 @@
 //
 // One CTA per (128 query tokens, pair of query heads that share a kv head).  Both contractions
 // run on the tensor cores: S = Q K^T into tensor memory, and O += P V with P written to shared
-// memory as bf16 by the softmax warps (four per head, one thread per query row).  The two heads are two independent streams over the
-// same key/value tiles (one TMA ring feeds both): while the softmax warpgroup of one stream
-// works on its S tile, the tensor cores serve the other stream.  One sweep over the key tiles
+// memory as bf16 by the softmax warps (four per head, one thread per query row).  The two heads
+// are two independent streams over the same key/value tiles (one TMA ring feeds both): while
+// the softmax warps of one stream work on their S tile, the tensor cores serve the other
+// stream.  Two threads issue the MMAs, one every S and one every O += P V, because an issuing
+// thread is held until the tensor pipe takes its instruction.  One sweep over the key tiles
 // with an online softmax: probabilities are taken against a per-row reference maximum, O
 // accumulates in tensor memory and is rescaled there only when a row's maximum has run ahead
 // of its reference by more than 2^8 (rare after the first tiles); the row sums divide the
