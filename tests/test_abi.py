@@ -63,6 +63,25 @@ def test_null_handle_calls_return_invalid_arg(lib):
     assert lib.ilre_recall_set_profiling(None, 1) == -1
     assert lib.ilre_recall_last_launch_count(None) == -1
     assert lib.ilre_recall_run(None, None, 1, None, 1, 0, None, None, None, None) == -1
+    assert lib.ilre_recall_run_host(None, None, 1, None, 1, 0, None, None, None, None) == -1
+    assert lib.ilre_recall_shard_stats(None, None, 1, None, 1, None, None) == -1
+    assert lib.ilre_recall_shard_scores(None, None, 1, None, 1, None, 1, None, None) == -1
+    assert lib.ilre_recall_allocate(None, None, 1, 0, None, None, None) == -1
+    assert lib.ilre_recall_fill_keys(None, None, 1, 64, None, None, 0, 500000.0, None, 1, None) == -1
+    assert lib.ilre_recall_rerope_keys(None, None, None, 1, 1, 0, 500000.0, None) == -1
+    assert lib.ilre_recall_rerope_sinks(None, None, None, 1, 1, 1, 500000.0, None) == -1
+    assert lib.ilre_recall_chunk_attention(None, None, None, None, 1, 0, None, None) == -1
+    assert lib.ilre_recall_copy_row_lse(None, None, 1, None) == -1
+    assert lib.ilre_recall_sm_clock(None, None) == -1
+    assert lib.ilre_recall_stage_times(None, None, 0) == -1
+
+
+def test_handle_free_calls_validate_their_arguments(lib):
+    # no device is touched before validation
+    assert lib.ilre_layer_recall(None, 0, 0, None, None, 0, None, None, None, None) == -1   # no layers
+    assert lib.ilre_layer_recall(None, 1, 4, None, None, 0, None, None, None, None) == -1   # no outputs
+    assert lib.ilre_gather_input_ids(None, 0, None, 0, None, 0, None, None) == -1
+    assert lib.ilre_topk_positions_noalloc(None, 16, 4, None, None) != 0
 
 
 def test_create_without_gpu_reports_cuda_error(lib):
