@@ -51,6 +51,8 @@ def _load():
         lib.ilre_oracle_winpool.argtypes = [c_f64p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
                                             c_f64p]
         lib.ilre_oracle_winpool.restype = None
+        lib.ilre_oracle_avg_precision.argtypes = [ctypes.c_int]
+        lib.ilre_oracle_avg_precision.restype = None
         lib.ilre_oracle_allocate.argtypes = [c_f64p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
                                              c_i32p, ctypes.c_int, c_i32p, ctypes.c_int,
                                              ctypes.c_int, c_i32p, c_i32p, c_i32p, c_f64p, c_f64p]
@@ -133,16 +135,28 @@ def maxpool(a: np.ndarray, m: int) -> np.ndarray:
     return out
 
 
-def winpool(p: np.ndarray, n: int, op: int) -> np.ndarray:
+def winpool(p: np.ndarray, n: int, op: int, avg_single: bool = False) -> np.ndarray:
+    """Stride-1 window pooling.  ``avg_single``: add and divide the averaging window in single
+    precision, left to right (see ``allocate``)."""
     p = np.ascontiguousarray(p, dtype=np.float64)
     out = np.empty(len(p), dtype=np.float64)
-    _load().ilre_oracle_winpool(_p(p, ctypes.c_double), len(p), n, op, _p(out, ctypes.c_double))
+    lib = _load()
+    lib.ilre_oracle_avg_precision(int(avg_single))
+    try:
+        lib.ilre_oracle_winpool(_p(p, ctypes.c_double), len(p), n, op, _p(out, ctypes.c_double))
+    finally:
+        lib.ilre_oracle_avg_precision(0)
     return out
 
 
 def allocate(A: np.ndarray, budget: int, max_sizes: Sequence[int], win_sizes: Sequence[int],
-             win_op: int, n_sink: int = 0, diagnostics: bool = False):
-    """Algorithm 1 on a score array: ascending positions [n_sink + budget] (int32)."""
+             win_op: int, n_sink: int = 0, diagnostics: bool = False, avg_single: bool = False):
+    """Algorithm 1 on a score array: ascending positions [n_sink + budget] (int32).
+
+    ``avg_single``: the averaging window is added left to right and divided in single precision
+    instead of double.  Which cells rank first is an integer decision taken from those sums; to
+    check such a decision of an implementation that averages in single precision (on scores
+    that are exact floats), both sides have to round alike."""
     a = np.ascontiguousarray(A, dtype=np.float64)
     ms = np.ascontiguousarray(np.asarray(max_sizes, dtype=np.int32))
     ws = np.ascontiguousarray(np.asarray(win_sizes, dtype=np.int32))
@@ -152,11 +166,16 @@ def allocate(A: np.ndarray, budget: int, max_sizes: Sequence[int], win_sizes: Se
     taken = np.zeros(nc, dtype=np.int32)
     last_v = np.zeros(nc, dtype=np.float64)
     kth_v = np.zeros(nc, dtype=np.float64)
-    rc = _load().ilre_oracle_allocate(_p(a, ctypes.c_double), len(a), n_sink, budget,
+    lib = _load()
+    lib.ilre_oracle_avg_precision(int(avg_single))
+    try:
+        rc = lib.ilre_oracle_allocate(_p(a, ctypes.c_double), len(a), n_sink, budget,
                                       _p(ms, ctypes.c_int32), len(ms), _p(ws, ctypes.c_int32),
                                       len(ws), win_op, _p(out, ctypes.c_int32),
                                       _p(quota, ctypes.c_int32), _p(taken, ctypes.c_int32),
                                       _p(last_v, ctypes.c_double), _p(kth_v, ctypes.c_double))
+    finally:
+        lib.ilre_oracle_avg_precision(0)
     if rc != 0:
         raise RuntimeError(f"ilre_oracle_allocate failed: {rc}")
     out = out[: n_sink + budget]

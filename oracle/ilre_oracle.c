@@ -191,13 +191,26 @@ int64_t ilre_oracle_maxpool(const double *a, int64_t n, int m, double *out)
     return len;
 }
 
+/* Precision of the averaging window (the only rounded step of Algorithm 1): 0 = double (the
+ * definition), 1 = single.  Which cells Algorithm 1 ranks first is an integer decision taken
+ * from these sums; to compare such a decision with an implementation that averages in
+ * single precision, both sides must round alike, so the oracle can also add the window left to
+ * right in float and divide in float (inputs that are exact floats stay exact). */
+static int g_avg_single = 0;
+void ilre_oracle_avg_precision(int single) { g_avg_single = single ? 1 : 0; }
+
 /* Algorithm 1, stride-1 window pooling of size n over p[0..len): op 0 = average, 1 = max
  * (R6, R7). */
 void ilre_oracle_winpool(const double *p, int64_t len, int n, int op, double *out)
 {
     for (int64_t c = 0; c < len; ++c) {
         const int64_t lo = c - n / 2;
-        if (op == 0) {
+        if (op == 0 && g_avg_single) {
+            float acc = 0.0f;
+            for (int64_t u = lo; u < lo + n; ++u)
+                if (u >= 0 && u < len) acc += (float)p[u];
+            out[c] = (double)(acc / (float)n);
+        } else if (op == 0) {
             double acc = 0.0;
             for (int64_t u = lo; u < lo + n; ++u)
                 if (u >= 0 && u < len) acc += p[u];

@@ -2,8 +2,10 @@
 
 scores: |gpu - oracle| <= 2e-3 * |oracle| + 1e-6 per position.
 indices: (a) selection logic -- Algorithm 1 run by the oracle on the GPU's own fp32 scores
-must give the GPU's index list, except at cells whose pooled value ties (rel 1e-6) with a
-combination's cut-off value (fp32 vs fp64 window sums); (b) end to end -- every position in
+must give the GPU's index list EXACTLY.  Which cells rank first is an integer decision taken
+from the pooled values, so both sides take it in the kernel's precision: the oracle adds the
+averaging window left to right and divides in single precision, as the kernel does (the
+maximum window is exact in any precision); (b) end to end -- every position in
 the symmetric difference with the oracle's list must sit, in some combination, within the
 score tolerance of that combination's cut-off (last accepted or K_m-th value), or the
 difference is a knock-on of such a flip, in which case (a) must still hold.
@@ -69,14 +71,12 @@ def check_recall(K, Q, w, gpu_idx, gpu_scores, ref_scores=None, ref_idx=None, sp
     assert rep["n_bad"] == 0, f"scores out of tolerance: {rep}"
     assert len(gpu_idx) == n_sink + budget
     assert np.all(np.diff(gpu_idx) > 0), "indices not strictly ascending"
-    # (a) selection logic on the GPU's own scores
-    own = oracle.allocate(gpu_scores, budget, max_sizes, win_sizes, win_op, n_sink)
-    tie = unexplained_differences(gpu_scores, gpu_idx, own, budget, max_sizes, win_sizes, win_op,
-                                  n_sink, 1e-6 if win_op == 0 else 0.0, 0.0)
-    rep["logic_diff"] = len(set(gpu_idx.tolist()) ^ set(own.tolist()))
-    assert not tie, f"selection logic differs from Algorithm 1 at {tie[:10]}"
-    if win_op == 1:
-        assert rep["logic_diff"] == 0
+    # (a) selection logic on the GPU's own scores, decided in the kernel's precision
+    own = oracle.allocate(gpu_scores, budget, max_sizes, win_sizes, win_op, n_sink,
+                          avg_single=True)
+    differ = sorted(set(gpu_idx.tolist()) ^ set(own.tolist()))
+    rep["logic_diff"] = len(differ)
+    assert not differ, f"selection logic differs from Algorithm 1 at {differ[:10]}"
     # (b) end to end against the oracle's own selection
     if ref_idx is None:
         ref_idx = oracle.allocate(ref_scores, budget, max_sizes, win_sizes, win_op, n_sink)

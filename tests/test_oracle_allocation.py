@@ -211,3 +211,40 @@ def test_multi_kernel_keeps_long_span_whole_single_small_kernel_does_not():
     multi = set(oracle.allocate(A, B, [1], [1, 15, 31], 1))
     assert len(single & set(span)) == 8
     assert set(span) <= multi
+
+
+# ---- the averaging window in single precision (the rounding an fp32 implementation applies) ----
+
+def test_single_precision_average_hand_example():
+    # window of 3 around cell 1 covers 1, 2^-24, 2^-24: in float 1 + 2^-24 rounds back to 1
+    # (tie to even) twice, so the sum is 1 and the average float(1) / float(3); in double the
+    # sum is 1 + 2^-23
+    p = np.array([1.0, 2.0 ** -24, 2.0 ** -24, 0.0, 0.0], dtype=np.float64)
+    w64 = oracle.winpool(p, 3, 0)
+    w32 = oracle.winpool(p, 3, 0, avg_single=True)
+    assert w64[1] == (1.0 + 2.0 ** -23) / 3.0
+    assert w32[1] == float(np.float32(1.0) / np.float32(3.0))
+    # the maximum window is exact either way
+    assert np.array_equal(oracle.winpool(p, 3, 1), oracle.winpool(p, 3, 1, avg_single=True))
+
+
+def test_single_precision_average_is_exact_on_small_integers_and_close_otherwise():
+    rng = np.random.default_rng(3)
+    ints = rng.integers(0, 64, size=500).astype(np.float64) * 8.0       # sums and /8 exact in float
+    assert np.array_equal(oracle.winpool(ints, 8, 0), oracle.winpool(ints, 8, 0, avg_single=True))
+    x = np.exp(rng.normal(-10, 3, size=2000)).astype(np.float32).astype(np.float64)
+    for n in (2, 7, 31, 200):
+        w64, w32 = oracle.winpool(x, n, 0), oracle.winpool(x, n, 0, avg_single=True)
+        assert np.all(np.abs(w32 - w64) <= (n + 1) * 2.0 ** -24 * w64)
+        assert np.array_equal(w32, w32.astype(np.float32).astype(np.float64))   # results are floats
+
+
+def test_single_precision_average_can_turn_a_near_tie_into_a_tie():
+    # cells 1 and 4 hold 1; cell 3, left neighbour of cell 4, holds 2^-25.  Window 2 covers
+    # [c - 1, c]: in double cell 4 averages 0.5 + 2^-26 and ranks first; in float both cells
+    # average exactly 0.5 and the lower index ranks first.
+    a = np.array([0.0, 1.0, 0.0, 2.0 ** -25, 1.0, 0.0, 0.0, 0.0], dtype=np.float64)
+    assert oracle.allocate(a, 1, (1,), (2,), 0).tolist() == [4]
+    assert oracle.allocate(a, 1, (1,), (2,), 0, avg_single=True).tolist() == [1]
+    # the switch does not leak into later calls
+    assert oracle.allocate(a, 1, (1,), (2,), 0).tolist() == [4]
