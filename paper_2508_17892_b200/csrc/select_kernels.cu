@@ -375,15 +375,20 @@ __device__ __forceinline__ unsigned long long fresh_tokens(const uint32_t* bm, i
     const int pos = n_sink + cell;
     return ((bitmap_word<kSmem>(bm, pos >> 5) >> (pos & 31)) & 1u) ^ 1u;
   }
-  unsigned long long fresh = 0ull;
+  // the cell's cnt <= 64 consecutive bits sit in at most three bitmap words (the bitmap has
+  // ceil(L / 32) words; words past its end are not read)
   const int t0 = cell * m;
   const int cnt = min(m, Lp - t0);
-  for (int j = 0; j < cnt; ++j) {
-    const int pos = n_sink + t0 + j;
-    const uint32_t taken = (bitmap_word<kSmem>(bm, pos >> 5) >> (pos & 31)) & 1u;
-    fresh |= static_cast<unsigned long long>(taken ^ 1u) << j;
-  }
-  return fresh;
+  const int pos0 = n_sink + t0;
+  const int w0 = pos0 >> 5, sh = pos0 & 31;
+  const int last_w = (pos0 + cnt - 1) >> 5;
+  unsigned long long taken = bitmap_word<kSmem>(bm, w0);
+  if (last_w > w0) taken |= static_cast<unsigned long long>(bitmap_word<kSmem>(bm, w0 + 1)) << 32;
+  taken >>= sh;
+  if (last_w > w0 + 1)                                    // only with sh > 0 and cnt > 64 - sh
+    taken |= static_cast<unsigned long long>(bitmap_word<kSmem>(bm, w0 + 2)) << (64 - sh);
+  const unsigned long long mask = (cnt >= 64) ? ~0ull : ((1ull << cnt) - 1ull);
+  return ~taken & mask;
 }
 
 // Exclusive prefix sum over the block with a single barrier: every warp scans the 32 warp
