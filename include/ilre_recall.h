@@ -305,7 +305,8 @@ int ilre_recall_destroy(ilre_recall_t* h);
  * synchronisation).  No handle is needed.  Returns the k positions with the highest scores,
  * equal scores ranked by lower position, as ascending int32 positions -- what
  * ilre_recall_run returns for one max kernel of size 1, one window of size 1 and no sink.
- *   scores_dev   fp32 [L] on the CURRENT device; 1 <= L <= ILRE_NOALLOC_MAX_L
+ *   scores_dev   fp32 [L] on the CURRENT device; 1 <= L <= ILRE_NOALLOC_MAX_L; no NaNs
+ *                (-0.0 and +0.0 count as equal; a NaN would rank by its bit pattern)
  *   out_idx_dev  int32 [k] on the current device; 0 <= k <= L
  * Larger L is rejected with ILRE_ERR_CAPACITY, k > L with ILRE_ERR_BUDGET; nothing is launched
  * then.  The call is asynchronous on cuda_stream and calls no cudaMalloc/cudaFree.  Its scratch

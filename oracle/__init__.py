@@ -55,7 +55,8 @@ def _load():
         lib.ilre_oracle_avg_precision.restype = None
         lib.ilre_oracle_allocate.argtypes = [c_f64p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
                                              c_i32p, ctypes.c_int, c_i32p, ctypes.c_int,
-                                             ctypes.c_int, c_i32p, c_i32p, c_i32p, c_f64p, c_f64p]
+                                             ctypes.c_int, c_i32p, c_i32p, c_i32p, c_f64p, c_f64p,
+                                             c_i32p]
         lib.ilre_oracle_dca_rerope.argtypes = [c_u16p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
                                                ctypes.c_int, ctypes.c_int, ctypes.c_double, c_f64p]
         _lib = lib
@@ -156,7 +157,9 @@ def allocate(A: np.ndarray, budget: int, max_sizes: Sequence[int], win_sizes: Se
     ``avg_single``: the averaging window is added left to right and divided in single precision
     instead of double.  Which cells rank first is an integer decision taken from those sums; to
     check such a decision of an implementation that averages in single precision (on scores
-    that are exact floats), both sides have to round alike."""
+    that are exact floats), both sides have to round alike.  ``diagnostics`` adds per
+    combination the quota, the tokens taken, the pooled value of the last contributing and of
+    the K_m-th cell, and per position the combination that allocated it (-1 = none)."""
     a = np.ascontiguousarray(A, dtype=np.float64)
     ms = np.ascontiguousarray(np.asarray(max_sizes, dtype=np.int32))
     ws = np.ascontiguousarray(np.asarray(win_sizes, dtype=np.int32))
@@ -166,6 +169,7 @@ def allocate(A: np.ndarray, budget: int, max_sizes: Sequence[int], win_sizes: Se
     taken = np.zeros(nc, dtype=np.int32)
     last_v = np.zeros(nc, dtype=np.float64)
     kth_v = np.zeros(nc, dtype=np.float64)
+    comb_of = np.empty(len(a), dtype=np.int32) if diagnostics else None
     lib = _load()
     lib.ilre_oracle_avg_precision(int(avg_single))
     try:
@@ -173,14 +177,16 @@ def allocate(A: np.ndarray, budget: int, max_sizes: Sequence[int], win_sizes: Se
                                       _p(ms, ctypes.c_int32), len(ms), _p(ws, ctypes.c_int32),
                                       len(ws), win_op, _p(out, ctypes.c_int32),
                                       _p(quota, ctypes.c_int32), _p(taken, ctypes.c_int32),
-                                      _p(last_v, ctypes.c_double), _p(kth_v, ctypes.c_double))
+                                      _p(last_v, ctypes.c_double), _p(kth_v, ctypes.c_double),
+                                      _p(comb_of, ctypes.c_int32) if diagnostics else None)
     finally:
         lib.ilre_oracle_avg_precision(0)
     if rc != 0:
         raise RuntimeError(f"ilre_oracle_allocate failed: {rc}")
     out = out[: n_sink + budget]
     if diagnostics:
-        return out, dict(quota=quota, taken=taken, last_value=last_v, kth_value=kth_v)
+        return out, dict(quota=quota, taken=taken, last_value=last_v, kth_value=kth_v,
+                         combination_of=comb_of)
     return out
 
 

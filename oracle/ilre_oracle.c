@@ -240,7 +240,9 @@ static int by_value_desc_then_cell(const void *x, const void *y)
  *   out_idx receives n_sink + budget ascending positions;
  *   optional per-combination diagnostics (arrays of n_max * n_win entries, may be NULL):
  *     quota[c], taken[c], last_value[c] = pooled value of the last cell that contributed a
- *     token, kth_value[c] = pooled value of the K_m-th ranked cell.
+ *     token, kth_value[c] = pooled value of the K_m-th ranked cell;
+ *   optional comb_out[L] (may be NULL): for every position the index of the combination that
+ *     allocated it, -1 for positions that were not allocated (sink positions included).
  * Returns 0; -1 allocation failure; -2 budget > L - n_sink or bad sizes; -3 if some
  * combination ran out of candidates before meeting its quota.
  */
@@ -249,7 +251,7 @@ int ilre_oracle_allocate(const double *A, int64_t L, int n_sink, int budget,
                          const int32_t *win_sizes, int n_win, int win_op,
                          int32_t *out_idx,
                          int32_t *quota_out, int32_t *taken_out,
-                         double *last_value_out, double *kth_value_out)
+                         double *last_value_out, double *kth_value_out, int32_t *comb_out)
 {
     if (n_sink < 0 || budget < 0 || n_max < 1 || n_win < 1) return -2;
     const int64_t Lp = L - n_sink;                 /* length without the sink part */
@@ -264,6 +266,7 @@ int ilre_oracle_allocate(const double *A, int64_t L, int n_sink, int budget,
     if (!in_I || !P || !W || !rk) { free(in_I); free(P); free(W); free(rk); return -1; }
 
     int rc = 0;
+    if (comb_out) for (int64_t t = 0; t < L; ++t) comb_out[t] = -1;
     for (int t = 0; t < n_sink; ++t) in_I[t] = 1;  /* I <- indices of the sink part */
     const double *Ap = A + n_sink;                 /* A^C without the sink part     */
     const int n_comb = n_max * n_win;
@@ -284,7 +287,10 @@ int ilre_oracle_allocate(const double *A, int64_t L, int n_sink, int budget,
                 const int64_t c = rk[r].c;
                 for (int64_t t = c * m; t < c * m + m && t < Lp && taken < quota; ++t) {
                     const int64_t posn = n_sink + t;
-                    if (!in_I[posn]) { in_I[posn] = 1; ++taken; last_v = rk[r].v; }
+                    if (!in_I[posn]) {
+                        in_I[posn] = 1; ++taken; last_v = rk[r].v;
+                        if (comb_out) comb_out[posn] = comb;
+                    }
                 }
             }
             if (taken < quota) rc = -3;

@@ -50,8 +50,11 @@ cudaError_t scratch_for(int device, uint32_t** out) {
   return cudaSuccess;
 }
 
+// Sort key of one score: value first, then lower position.  Adding +0.0 turns -0.0 into +0.0,
+// so that the two zeros tie like any other pair of equal scores.
 __device__ __forceinline__ unsigned long long key_of(float v, uint32_t pos) {
-  return (static_cast<unsigned long long>(ilre::float_to_ordered(v)) << 32) | (0xFFFFFFFFu - pos);
+  return (static_cast<unsigned long long>(ilre::float_to_ordered(v + 0.0f)) << 32) |
+         (0xFFFFFFFFu - pos);
 }
 
 // Exclusive block scan over 1024 threads; *total = block sum.

@@ -49,7 +49,7 @@ def test_benchmark_configs_match_oracle(cases, name):
     w = x.workload
     eng = _engine(w)
     idx, sc = _run(eng, x)
-    rep = parity.check_recall(x.K, x.Q, w, idx, sc, ref_scores=a)
+    rep = parity.check_recall(x.K, x.Q, w, idx, sc, ref_scores=a, strict=True)
     gpu_lse = eng.row_lse(w.q_len).cpu().numpy().reshape(-1)
     assert np.abs(gpu_lse - lse).max() < 5e-4
     assert eng.last_launch_count() > 0
@@ -283,50 +283,46 @@ def test_error_codes_on_device(cases):
     eng.close()
 
 
-def test_full_size_1m_config_sampled():
-    """L = 1M, q_len = 256 (the benchmark configuration, same launch geometry as bench.py).
-
-    The oracle cannot finish 4.4e12 fp64 flops in a test, so it checks: (1) row statistics of
-    sampled rows, computed in full by the oracle; (2) scores at sampled positions, computed by
-    the oracle from the definition with the device's row statistics; (3) the selection logic,
-    exactly, by running the oracle's Algorithm 1 on the device's scores."""
+def test_full_size_1m_config_against_the_full_oracle():
+    """L = 1M, q_len = 256 (the benchmark configuration, same launch geometry as bench.py),
+    against the oracle run in full: the statistics of all 8192 rows over all 1M keys, all 1M
+    scores from the oracle's own statistics, and the index list, which must be identical.
+    The oracle needs about two minutes of the host's cores for its 4.4e12 flops."""
     w = CONFIGS["cfg5_L1m"]
     x = make_inputs(w)
     eng = _engine(w)
     idx, sc = _run(eng, x)
     gpu_lse = eng.row_lse(w.q_len).cpu().numpy().reshape(-1).astype(np.float64)
+    a, m, z = oracle.scores(x.K, x.Q, with_stats=True)
+    lse = m + np.log(z)
+    assert np.abs(gpu_lse - lse).max() < 5e-4
+    rep = parity.check_recall(x.K, x.Q, w, idx, sc, ref_scores=a, strict=True)
+    print("cfg5_L1m", rep, "max lse error", np.abs(gpu_lse - lse).max())
+    assert np.all(np.isfinite(sc)) and sc.min() > 0 and sc.max() <= 1
     rng = np.random.default_rng(0)
     rows = np.unique(np.concatenate([rng.integers(0, w.q_len * w.n_q_heads, 40),
                                      [0, w.q_len * w.n_q_heads - 1]]))
-    m, z = oracle.row_stats(x.K, x.Q, rows.tolist())
-    assert np.abs(gpu_lse[rows] - (m + np.log(z))).max() < 5e-4
-    planted = x.planted_positions().numpy()
-    pos = np.unique(np.concatenate([rng.integers(0, w.L, 300), planted[::64],
-                                    [0, 127, 128, w.L - 1], idx[::97]]))
-    ref = oracle.scores_at(x.K, x.Q, gpu_lse, np.ones_like(gpu_lse), pos.tolist())
-    rep = parity.score_errors(sc[pos].astype(np.float64), ref)
-    assert rep["n_bad"] == 0, rep
-    assert np.all(np.isfinite(sc)) and sc.min() > 0 and sc.max() <= 1
-    own = oracle.allocate(sc.astype(np.float64), w.budget, w.max_sizes, w.win_sizes, w.win_op, 0)
-    np.testing.assert_array_equal(idx, own)
     # The same context as eight key shards of 131072 positions (the per-rank steps bench.py
-    # times with --shards 8): merged statistics, sampled scores and the selection logic
+    # times with --shards 8): merged statistics, all scores and the index list
     # against the oracle, and the scores against the unsharded run's.
     from paper_2508_17892_b200.sharded import shard_bounds
     K, Q = x.K.cuda(), x.Q.cuda()
     bounds = [shard_bounds(w.L, 8, r) for r in range(8)]
-    stats = torch.stack([eng.shard_stats(K[a:b], Q) for a, b in bounds])
-    sc8 = torch.cat([eng.shard_scores(K[a:b], Q, stats) for a, b in bounds])
+    stats = torch.stack([eng.shard_stats(K[lo:hi], Q) for lo, hi in bounds])
+    sc8 = torch.cat([eng.shard_scores(K[lo:hi], Q, stats) for lo, hi in bounds])
     idx8 = eng.allocate(sc8, w.budget, w.max_sizes, w.win_sizes, w.win_op, w.n_sink)
     torch.cuda.synchronize()
     eng.check_status()
     sc8, idx8 = sc8.cpu().numpy(), idx8.cpu().numpy()
     lse8 = eng.row_lse(w.q_len).cpu().numpy().reshape(-1).astype(np.float64)
-    assert np.abs(lse8[rows] - (m + np.log(z))).max() < 5e-4
+    assert np.abs(lse8 - lse).max() < 5e-4
     assert np.abs(lse8 - gpu_lse).max() < 1e-5
-    rep8 = parity.score_errors(sc8[pos].astype(np.float64), ref)
-    assert rep8["n_bad"] == 0, rep8
+    # per-shard statistics of sampled rows against the oracle on the same key range
+    a0, b0 = bounds[3]
+    m3, z3 = oracle.row_stats(x.K[a0:b0].contiguous(), x.Q, rows.tolist())
+    st3 = stats[3].cpu().numpy().astype(np.float64)[rows]
+    assert np.abs(st3[:, 0] * np.log(2.0) + np.log(st3[:, 1]) - (m3 + np.log(z3))).max() < 5e-4
+    rep8 = parity.check_recall(x.K, x.Q, w, idx8, sc8, ref_scores=a)
+    print("cfg5_L1m in 8 shards", rep8)
     assert np.abs(sc8 - sc).max() <= 2e-5 * sc.max() and np.all(np.abs(sc8 - sc) <= 1e-4 * sc)
-    own8 = oracle.allocate(sc8.astype(np.float64), w.budget, w.max_sizes, w.win_sizes, w.win_op, 0)
-    np.testing.assert_array_equal(idx8, own8)
     eng.close()

@@ -123,9 +123,10 @@ def test_algorithm1_against_set_transcription(seed):
 def test_hand_worked_example():
     g = _read_golden("alg1_worked_example.txt")
     A = np.array([float(x) for x in g["A"]])
-    got = oracle.allocate(A, int(g["budget"][0]), [int(x) for x in g["max_sizes"]],
-                          [int(x) for x in g["win_sizes"]], 0)
+    got, diag = oracle.allocate(A, int(g["budget"][0]), [int(x) for x in g["max_sizes"]],
+                                [int(x) for x in g["win_sizes"]], 0, diagnostics=True)
     assert list(got) == [int(x) for x in g["expected"]]
+    assert list(diag["combination_of"]) == [int(x) for x in g["combination_of"]]
 
 
 def test_hand_worked_tie_rule():

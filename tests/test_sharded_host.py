@@ -103,6 +103,9 @@ def test_sharded_recall_on_gloo_ranks_matches_the_unsharded_oracle(world, L, por
         # statistics and scores crossed the wire as fp32
         assert np.all(np.abs(sc - a) <= 2e-5 * a + 1e-12)
         assert len(idx) == w.n_sink + w.budget and idx == sorted(set(idx))
-        bad = parity.unexplained_differences(a, idx, ref, w.budget, w.max_sizes, w.win_sizes,
-                                             w.win_op, w.n_sink, 1e-4, 1e-12)
-        assert not bad
+        own, diag = oracle.allocate(sc, w.budget, w.max_sizes, w.win_sizes, w.win_op, w.n_sink,
+                                    diagnostics=True)
+        assert own.tolist() == idx
+        assert not parity.decisions_within_tolerance(a, diag["combination_of"], w.budget,
+                                                     w.max_sizes, w.win_sizes, w.win_op, w.n_sink,
+                                                     1e-4, 1e-12)

@@ -5,7 +5,8 @@ thread that must never hit cudaMalloc's implicit synchronisation).  For them the
 one call that needs no handle and keeps its scratch in a fixed array inside the library.  Here
 its result is compared, through the C ABI, with what ``ilre_recall_run`` returns for the
 equivalent pooling spec (one max kernel of size 1, one window of size 1, no sink), on two
-calls in a row -- the second call reuses the scratch the first one left behind.
+calls in a row -- the second call reuses the scratch the first one left behind -- and with
+the CPU oracle's Algorithm 1 for that spec.
 """
 import ctypes
 
@@ -13,6 +14,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from workloads import CONFIGS, make_inputs, small_workload
 
 pytestmark = pytest.mark.gpu
@@ -40,6 +42,10 @@ def test_noalloc_topk_matches_recall_run_twice_in_a_row():
     torch.cuda.synchronize()
     assert torch.equal(out_a, ref_a)                        # integer positions: bit-exact
     assert torch.equal(out_b, ref_b)
+    # and against the oracle: Algorithm 1 with one size-1 max kernel and one size-1 window
+    sc64 = scores.cpu().numpy().astype(np.float64)
+    assert np.array_equal(out_a.cpu().numpy(), oracle.allocate(sc64, 512, [1], [1], 1))
+    assert np.array_equal(out_b.cpu().numpy(), oracle.allocate(sc64, 100, [1], [1], 1))
     eng.close()
 
     # a ragged length with exact ties (scores quantised to few levels), k = 0 and k = L
@@ -52,6 +58,19 @@ def test_noalloc_topk_matches_recall_run_twice_in_a_row():
     got = topk_positions_noalloc(coarse, 700)
     torch.cuda.synchronize()
     assert torch.equal(got.long(), want)
+    assert np.array_equal(got.cpu().numpy(),
+                          oracle.allocate(coarse.cpu().numpy().astype(np.float64), 700, [1], [1], 1))
+    # zeros of either sign are one value: ties among them go to the lower position
+    zeros = coarse.clone()
+    zeros[::3] = 0.0
+    zeros[1::3] = -0.0
+    zeros[2::3] = torch.where(zeros[2::3] > 0.01, zeros[2::3], torch.zeros_like(zeros[2::3]))
+    n_pos = int((zeros > 0).sum())
+    got0 = topk_positions_noalloc(zeros, n_pos + 40)
+    torch.cuda.synchronize()
+    assert np.array_equal(got0.cpu().numpy(),
+                          oracle.allocate(zeros.cpu().numpy().astype(np.float64), n_pos + 40,
+                                          [1], [1], 1))
     assert topk_positions_noalloc(coarse, 0).numel() == 0
     assert torch.equal(topk_positions_noalloc(coarse, 5003).long().cpu(), torch.arange(5003))
     eng2.close()
