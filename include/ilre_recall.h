@@ -99,7 +99,7 @@ int ilre_recall_run(ilre_recall_t* h,
  * Same computation from HOST buffers (handle created with host_staging != 0): copies the
  * key cache and query to device staging, runs, copies the indices (and scores if asked)
  * back, and synchronises the stream before returning.  For throughput the host buffers
- * should be page-locked.  Contexts of 131072 positions or more are uploaded in up to 16 pieces
+ * should be page-locked.  Contexts of more than 65536 positions are uploaded in up to 16 pieces
  * on an internal stream while the row statistics of the pieces already on the device are
  * computed; the pieces' statistics are merged as those of key shards are, so the scores may
  * differ from ilre_recall_run's in the rounding order of the softmax denominator (a few fp32
@@ -183,7 +183,9 @@ int ilre_recall_chunk_attention(ilre_recall_t* h, const void* q_dev, const void*
  * (ILRE_ERR_CAPACITY), all three tensors 16-byte aligned.  bf16 x bf16 products accumulate in
  * fp32 on the tensor cores; bias, rotation in fp32 from angle tables built in double precision;
  * one rounding to bf16.  Asynchronous on cuda_stream; bounded waits report through
- * ilre_recall_status.
+ * ilre_recall_status.  The handle keeps the angle tables between calls (they depend on
+ * rope_theta only); a call on another stream than the one that built them waits for the build
+ * on the device, but calls with different rope_theta on one handle must not overlap.
  */
 int ilre_recall_fill_keys(ilre_recall_t* h, const void* x_dev, int64_t n_tok, int32_t d_model,
                           const void* w_k_dev, const void* bias_dev, int64_t pos0,
@@ -202,8 +204,9 @@ int ilre_recall_fill_keys(ilre_recall_t* h, const void* x_dev, int64_t n_tok, in
  *                which case the unrotated chunks are copied
  * Arithmetic: fp32 from an angle table computed in double precision, one rounding to bf16
  * (nearest even).  Asynchronous on cuda_stream.  At most 8192 + 2 chunks
- * (ILRE_ERR_CAPACITY beyond).  The handle keeps the angle table between calls, so calls on
- * one handle must not overlap.
+ * (ILRE_ERR_CAPACITY beyond).  The handle keeps the angle table between calls; a call on
+ * another stream waits on the device for the table's build, but calls that need different
+ * tables (chunk size, theta, more rows) must not overlap on one handle.
  */
 int ilre_recall_rerope_keys(ilre_recall_t* h, const void* k_cache_dev, void* k_out_dev,
                             int64_t L, int32_t chunk_size, int32_t n_sink, double rope_theta,

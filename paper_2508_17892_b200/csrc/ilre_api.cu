@@ -56,10 +56,14 @@ struct ilre_recall {
   float2* rope_table;                   // (cos, sin) per (chunk distance, channel pair)
   int rope_rows, rope_chunk;            // what the table currently holds
   double rope_theta;
+  cudaEvent_t rope_ready;               // recorded after the table's build, on rope_stream
+  cudaStream_t rope_stream;
   float2* pos_lo;                       // RoPE angle tables of the key-cache fill
   float2* pos_hi;
   int pos_hi_rows;
   double pos_theta;                     // theta the tables were built for (0 = none)
+  cudaEvent_t pos_ready;                // recorded after their build, on pos_stream
+  cudaStream_t pos_stream;
   unsigned long long* cand;
   uint32_t* cand_count;
   int* ranked;
@@ -139,6 +143,8 @@ void free_all(ilre_recall* h) {
   cudaFree(h->piece_stats);
   if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
   if (h->copy_begin) cudaEventDestroy(h->copy_begin);
+  if (h->rope_ready) cudaEventDestroy(h->rope_ready);
+  if (h->pos_ready) cudaEventDestroy(h->pos_ready);
   for (int i = 0; i < kHostPieces; ++i)
     if (h->piece_done[i]) cudaEventDestroy(h->piece_done[i]);
   for (int r = 0; r < kProfRing; ++r)
@@ -276,6 +282,8 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out) {
   for (int r = 0; ok && r < kProfRing; ++r)
     for (int i = 0; ok && i <= kNumStages; ++i)
       ok = (cudaEventCreate(&h->ev[r][i]) == cudaSuccess);
+  ok = ok && (cudaEventCreateWithFlags(&h->rope_ready, cudaEventDisableTiming) == cudaSuccess);
+  ok = ok && (cudaEventCreateWithFlags(&h->pos_ready, cudaEventDisableTiming) == cudaSuccess);
   if (ok) ok = (cudaMemset(h->status, 0, sizeof(int)) == cudaSuccess);
   if (ok) ok = (cudaMemset(h->clk, 0, 2 * sizeof(unsigned long long)) == cudaSuccess);
   if (ok) ok = (cudaMemset(h->grid_barrier, 0, sizeof(uint32_t)) == cudaSuccess);
@@ -611,8 +619,12 @@ int ilre_recall_fill_keys(ilre_recall_t* h, const void* x_dev, int64_t n_tok, in
   int launches = 0;
   if (h->pos_theta != rope_theta) {                    // tables depend on theta only
     ILRE_CUDA(launch_rope_pos_tables(h->pos_lo, h->pos_hi, h->pos_hi_rows, rope_theta, st));
+    ILRE_CUDA(cudaEventRecord(h->pos_ready, st));
     h->pos_theta = rope_theta;
+    h->pos_stream = st;
     ++launches;
+  } else if (st != h->pos_stream) {                    // built on another stream: wait for it
+    ILRE_CUDA(cudaStreamWaitEvent(st, h->pos_ready, 0));
   }
   const int n_out = h->cfg.n_kv_heads * kHeadDim;
   const long long m_tiles = (n_tok + kFillTileM - 1) / kFillTileM;
@@ -661,8 +673,12 @@ int ilre_recall_rerope_keys(ilre_recall_t* h, const void* k_cache_dev, void* k_o
   if (n_rows > 0 && (h->rope_chunk != chunk_size || h->rope_theta != rope_theta ||
                      h->rope_rows < n_rows)) {
     ILRE_CUDA(launch_rope_table(h->rope_table, static_cast<int>(n_rows), chunk_size, rope_theta, st));
+    ILRE_CUDA(cudaEventRecord(h->rope_ready, st));
     h->rope_chunk = chunk_size; h->rope_theta = rope_theta; h->rope_rows = static_cast<int>(n_rows);
+    h->rope_stream = st;
     ++launches;
+  } else if (n_rows > 0 && st != h->rope_stream) {     // built on another stream: wait for it
+    ILRE_CUDA(cudaStreamWaitEvent(st, h->rope_ready, 0));
   }
   ReropeParams rp;
   rp.k_in = static_cast<const uint4*>(k_cache_dev);
@@ -699,8 +715,12 @@ int ilre_recall_rerope_sinks(ilre_recall_t* h, const void* k_sink_dev, void* k_o
       while (want < turns) want *= 2;
       if (want > kRopeTableRows) want = kRopeTableRows;
       ILRE_CUDA(launch_rope_table(h->rope_table, static_cast<int>(want), chunk_size, rope_theta, st));
+      ILRE_CUDA(cudaEventRecord(h->rope_ready, st));
       h->rope_chunk = chunk_size; h->rope_theta = rope_theta; h->rope_rows = static_cast<int>(want);
+      h->rope_stream = st;
       ++launches;
+    } else if (st != h->rope_stream) {                 // built on another stream: wait for it
+      ILRE_CUDA(cudaStreamWaitEvent(st, h->rope_ready, 0));
     }
     row = h->rope_table + (turns - 1) * kRopeHalfDim;
   }
