@@ -11,7 +11,15 @@ the same metric through the host entry point (host buffers, copies inside the ti
 
 With N > 1 (under torchrun) every rank runs an independent replica of the same recall on its
 own GPU (the path has no exchange step); the value is the sum over ranks divided by the
-slowest rank's time.  `--impl reference` times the CPU oracle on a bounded sample.
+slowest rank's time; the same line then carries, under `sharded_recall`, ONE recall with the
+keys split by position over the ranks (its two all-gathers included).  `--impl reference`
+times the CPU oracle on a bounded sample.
+
+Beside the headline the line carries `configs`: the other benchmark configurations (L = 4K
+to 512K), an HBM-bound probe (L = 1M, q_len 16) and the L = 1M configuration under
+Algorithm 1's default pooling spec, each timed with a cold L2; and the steps around the
+recall (key fill, Eq. 7 re-rotation alone and followed by the recall, chunk attention, the
+per-rank steps of a sharded recall, the retrieval-layer sweep).
 """
 from __future__ import annotations
 
@@ -157,6 +165,65 @@ def pick_workload(args):
     return w
 
 
+SIDE_WORKLOADS = ("cfg1_L4k", "cfg2_L32k", "cfg3_L128k", "cfg4_L512k", "probe_L1m_q16",
+                  "cfg5_L1m_paper_pool")
+
+
+def time_side_workload(eng, dev, w, x, steps, flush, peaks, K=None, Q=None):
+    """One row of the `configs` block: `steps` recalls of workload `w`, each between its own
+    pair of CUDA events, with a write of `flush` (larger than L2) before every recall so that
+    no key is served from L2 left warm by the previous recall.  Returns ms per recall (median
+    and mean), key-cache GB/s, stage times and the roofline fractions."""
+    K = x.K.to(dev) if K is None else K
+    Q = x.Q.to(dev) if Q is None else Q
+    spec = (w.budget, w.max_sizes, w.win_sizes, w.win_op, w.n_sink)
+    out_idx = torch.empty(w.n_sink + w.budget, dtype=torch.int32, device=dev)
+    for _ in range(3):
+        eng.run(K, Q, *spec, out_idx=out_idx)
+    torch.cuda.synchronize()
+    eng.check_status()
+    eng.set_profiling(True)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+           for _ in range(steps)]
+    for a, b in evs:
+        flush.zero_()
+        a.record()
+        eng.run(K, Q, *spec, out_idx=out_idx)
+        b.record()
+    torch.cuda.synchronize()
+    ms_all = sorted(a.elapsed_time(b) for a, b in evs)
+    stages = eng.stage_times()
+    eng.set_profiling(False)
+    eng.check_status()
+    # the same loop back to back (keys of short contexts stay in L2), for comparison
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(steps):
+        eng.run(K, Q, *spec, out_idx=out_idx)
+    b.record()
+    torch.cuda.synchronize()
+    ms_warm = a.elapsed_time(b) / steps
+    ms = ms_all[len(ms_all) // 2]
+    k_bytes = K.numel() * 2
+    flops = 2.0 * w.q_len * w.n_q_heads * w.L * w.d
+    gbs = k_bytes / (ms * 1e-3) / 1e9
+    row = dict(workload=workload_string(w), ms_per_recall=ms, ms_mean=sum(ms_all) / len(ms_all),
+               ms_min=ms_all[0], ms_back_to_back=ms_warm, steps=steps,
+               l2="flushed before every recall (256 MiB write, untimed)",
+               key_cache_gbs=gbs, stages_ms=stages, launches_per_recall=eng.last_launch_count(),
+               hbm_frac_one_read_of_K=gbs / peaks["hbm_gbs"],
+               tensor_frac_one_qk_burst=flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+               tensor_frac_one_qk_sustained=flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+               per_pass=dict(
+                   row_stats_gbs=k_bytes / (stages["row_stats"] * 1e-3) / 1e9,
+                   row_stats_hbm_frac=k_bytes / (stages["row_stats"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                   row_stats_tflops=flops / (stages["row_stats"] * 1e-3) / 1e12,
+                   scores_gbs=k_bytes / (stages["scores"] * 1e-3) / 1e9,
+                   scores_hbm_frac=k_bytes / (stages["scores"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                   scores_tflops=flops / (stages["scores"] * 1e-3) / 1e12))
+    return row
+
+
 def oracle_sample_run(x, sample_keys: int):
     """One oracle recall on the first `sample_keys` positions of the workload."""
     import oracle
@@ -205,8 +272,9 @@ def run_reference(args, world, rank):
 
 
 def run_sharded(args, world, rank, dev, w, x, eng, spec):
-    """--sharded: ONE recall over keys split by position across the ranks (strong scaling):
-    per-rank kernels plus the two all-gathers of the exchange, timed together."""
+    """ONE recall over keys split by position across the ranks (strong scaling): per-rank
+    kernels plus the two all-gathers of the exchange, timed together.  Returns the result
+    line on rank 0 (None elsewhere)."""
     import torch.distributed as dist
     from paper_2508_17892_b200.sharded import shard_bounds, sharded_recall
     own_group = not dist.is_initialized()
@@ -244,6 +312,7 @@ def run_sharded(args, world, rank, dev, w, x, eng, spec):
     dist.broadcast(ref, src=0)
     assert torch.equal(ref, idx), "ranks disagree on the recalled indices"
     elapsed_max, units = aggregate(elapsed_ms, float(K.numel() * 2) * args.steps, dev)
+    line = None
     if rank == 0:
         ms = elapsed_max / args.steps
         line = dict(metric=METRIC, value=units / (elapsed_max * 1e-3) / 1e9, unit=UNIT, n_gpus=world,
@@ -254,10 +323,10 @@ def run_sharded(args, world, rank, dev, w, x, eng, spec):
                                 parallelism=f"key-range sharded over {world} rank(s), two all-gathers"),
                     clocks=clocks, e2e=None, gpu_launches=8 * args.steps, roofline=None,
                     cpu_baseline=None)
-        print(json.dumps(line), flush=True)
-    eng.close()
+    del K
     if own_group:
         dist.destroy_process_group()
+    return line
 
 
 def run_ours(args, world, rank, local):
@@ -274,7 +343,10 @@ def run_ours(args, world, rank, local):
                      n_q_heads=w.n_q_heads, device=local, host_staging=not (args.no_e2e or args.sharded))
     spec = (w.budget, w.max_sizes, w.win_sizes, w.win_op, w.n_sink)
     if args.sharded:
-        run_sharded(args, world, rank, dev, w, x, eng, spec)
+        line = run_sharded(args, world, rank, dev, w, x, eng, spec)
+        if rank == 0:
+            print(json.dumps(line), flush=True)
+        eng.close()
         return
     K, Q = x.K.to(dev), x.Q.to(dev)
     out_idx = torch.empty(w.n_sink + w.budget, dtype=torch.int32, device=dev)
@@ -359,6 +431,24 @@ def run_ours(args, world, rank, local):
                    algorithmic_bytes=moved, achieved=moved / (ms * 1e-3) / 1e9, unit="GB/s",
                    bound="hbm", peak=measured_peaks()["hbm_gbs"],
                    frac=moved / (ms * 1e-3) / 1e9 / measured_peaks()["hbm_gbs"])
+        # the recall with DCA on (Eq. 7 -> Eq. 4): the cache re-rotated into a second buffer,
+        # then the recall on the rotated keys, one stream, one timed region
+        def dca_recall():
+            eng.rerope_keys(K, args.dca_chunk, w.n_sink, out=Kc)
+            eng.run(Kc, Q, *spec, out_idx=out_idx)
+        for _ in range(3):
+            dca_recall()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(reps):
+            dca_recall()
+        e1.record()
+        torch.cuda.synchronize()
+        ms_on = e0.elapsed_time(e1) / reps
+        dca["recall_with_dca"] = dict(ms=ms_on, key_cache_gbs=k_bytes / (ms_on * 1e-3) / 1e9,
+                                      steps=reps, note="re-rotation out of place + recall, one "
+                                      "timed region; key cache larger than L2")
+        eng.check_status()
         del Kc
 
     # Key-cache fill (key projection + RoPE into the cache), timed on its own: a tensor-bound
@@ -518,6 +608,37 @@ def run_ours(args, world, rank, local):
         eng.check_status()
         del Kl, Ql
 
+    # The other workloads: benchmark configurations 1-4, the HBM-bound probe and the benchmark
+    # configuration under Algorithm 1's default pooling, each timed with a cold L2.
+    configs_block = None
+    if args.side_steps > 0 and rank == 0 and args.config == "cfg5_L1m" and not args.L:
+        from workloads import CONFIGS
+        peaks_now = measured_peaks()
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        configs_block = {}
+        for name in SIDE_WORKLOADS:
+            sw = CONFIGS[name]
+            same_cache = (sw.seed == w.seed and sw.L == w.L and sw.q_len == w.q_len)
+            if same_cache:                                   # same keys and query as the main workload
+                row = time_side_workload(eng, dev, sw, x, args.side_steps, flush, peaks_now, K=K, Q=Q)
+            else:
+                sx = make_inputs(sw)
+                row = time_side_workload(eng, dev, sw, sx, args.side_steps, flush, peaks_now)
+                del sx
+            if name.startswith("probe"):
+                row["note"] = ("not a BASELINE config: q_len 16 puts the key scan below the ridge, "
+                               "so per_pass.*_hbm_frac is the streaming efficiency of each pass")
+            configs_block[name] = row
+        del flush
+
+    # With more than one rank: also ONE recall over keys split by position across the ranks
+    # (the replica line above measures throughput, this one the latency of a sharded recall)
+    sharded_line = None
+    if world > 1 and not args.no_sharded_line:
+        del K
+        torch.cuda.empty_cache()
+        sharded_line = run_sharded(args, world, rank, dev, w, x, eng, spec)
+
     elapsed_max, units = aggregate(elapsed_ms, float(k_bytes) * args.steps, dev)
     if rank != 0:
         return
@@ -532,18 +653,26 @@ def run_ours(args, world, rank, local):
     ridge = peaks["bf16_tflops_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
     hbm_bound = (flops / k_bytes) < ridge
     dom_gbs = k_bytes / (stages[dom] * 1e-3) / 1e9
+    # A timed loop shorter than about a second runs before the board settles at its power cap:
+    # the burst bf16 figure is then the matching denominator, the sustained one otherwise.
+    loop_s = elapsed_max * 1e-3
+    regime = "burst" if loop_s < 1.0 else "sustained"
+    tensor_peak = peaks["bf16_tflops"] if regime == "burst" else peaks["bf16_tflops_sustained"]
     roofline = dict(bound="hbm" if hbm_bound else "tensor", kernel=f"{dom}_kernel",
                     achieved=dom_gbs if hbm_bound else dom_tflops,
-                    peak=peaks["hbm_gbs"] if hbm_bound else peaks["bf16_tflops_sustained"],
+                    peak=peaks["hbm_gbs"] if hbm_bound else tensor_peak,
                     unit="GB/s" if hbm_bound else "TFLOP/s",
-                    frac=(dom_gbs / peaks["hbm_gbs"] if hbm_bound
-                          else dom_tflops / peaks["bf16_tflops_sustained"]),
+                    frac=(dom_gbs / peaks["hbm_gbs"] if hbm_bound else dom_tflops / tensor_peak),
+                    frac_of_burst_bf16=dom_tflops / peaks["bf16_tflops"],
+                    frac_of_sustained_bf16=dom_tflops / peaks["bf16_tflops_sustained"],
+                    regime=f"{regime}: timed loop of {loop_s:.2f} s, in-kernel SM clock "
+                           f"{sm_mhz_in_kernel:.0f} MHz",
                     flop_per_key_byte=flops / k_bytes, ridge_flop_per_byte=ridge,
                     traffic=(ROW_STATS_DRAM_BYTES_PER_KEY * w.L
                              if dom == "row_stats" and w.q_len == 256 else None),
                     traffic_unit="bytes per launch (ncu at L=131072, scaled by L)",
                     peak_source=(f"{peaks['source']} (HBM copy)" if hbm_bound
-                                 else f"{peaks['source']} (sustained bf16)"),
+                                 else f"{peaks['source']} ({regime} bf16)"),
                     kernel_ms=stages[dom], algorithmic_flops_per_launch=flops,
                     algorithmic_bytes_per_launch=k_bytes,
                     kernel_hbm_gbs=k_bytes / (stages[dom] * 1e-3) / 1e9)
@@ -580,7 +709,8 @@ def run_ours(args, world, rank, local):
                 clocks=clocks, e2e=e2e, gpu_launches=launches, roofline=roofline,
                 cpu_baseline=cpu_baseline,
                 stages_ms=stages, dca_rerope=dca, key_fill=fill, chunk_attention=attn,
-                sharded_steps=shard, layer_sweep=sweep,
+                sharded_steps=shard, layer_sweep=sweep, configs=configs_block,
+                sharded_recall=sharded_line,
                 whole_step=dict(hbm_frac_one_read_of_K=step_hbm_frac,
                                 tensor_frac_one_qk=step_tensor_frac,
                                 hbm_frac_of_8TBps=(k_bytes / (ms_per_step * 1e-3) / 1e9) / 8000.0))
@@ -613,6 +743,11 @@ def main():
     ap.add_argument("--sweep-layers", type=int, default=8,
                     help="also time the offline retrieval-layer sweep over this many candidate "
                          "layers at L = 128K (0 = skip)")
+    ap.add_argument("--side-steps", type=int, default=20,
+                    help="recalls timed per workload of the `configs` block (benchmark "
+                         "configurations 1-4, the q_len 16 probe, the default pooling spec; 0 = skip)")
+    ap.add_argument("--no-sharded-line", action="store_true",
+                    help="with --gpus N > 1: skip the additional key-range sharded recall")
     ap.add_argument("--cpu-sample-keys", type=int, default=131072)
     ap.add_argument("--ref-sample-keys", type=int, default=4096)
     args = ap.parse_args()

@@ -296,6 +296,30 @@ int ilre_recall_sm_clock(ilre_recall_t* h, float* mhz_out_host);
 int ilre_recall_set_profiling(ilre_recall_t* h, int32_t on);
 int ilre_recall_stage_times(ilre_recall_t* h, float* ms_host, int32_t n);
 
+/*
+ * Failure-detection self test.  Every wait inside the kernels (mbarrier waits of the TMA /
+ * tensor-core pipelines, the grid barrier of the Algorithm 1 kernel) is bounded: a wait that
+ * runs past its spin budget records a code in the handle's status word, its CTA leaves the
+ * kernel in an orderly way (no trap, tensor memory released), and ilre_recall_status returns
+ * ILRE_ERR_DEVICE_WAIT after the caller's next synchronisation.  This call lets a test reach
+ * that path without faulting anything: it sets the spin budget of the following runs on this
+ * handle and makes ONE wait impossible to complete,
+ *   ILRE_SELFTEST_GRID_BARRIER      the grid barrier of the Algorithm 1 kernel waits for one
+ *                                   CTA more than the grid has;
+ *   ILRE_SELFTEST_MISSING_KEY_TILE  the TMA producer of the row-statistics kernel leaves out
+ *                                   the last key tile of every CTA, so the tensor-core thread
+ *                                   waits for a tile that never arrives;
+ *   ILRE_SELFTEST_OFF               normal operation.
+ * wait_cycle_limit is the spin budget in SM clock cycles (0 = the default of 2^31, about a
+ * second).  The outputs of a run with an injected failure are unspecified; after
+ * ilre_recall_selftest_wait(h, 0, ILRE_SELFTEST_OFF) the handle works as before.  The paper
+ * has no counterpart; host-side, changes only the handle.
+ */
+#define ILRE_SELFTEST_OFF 0
+#define ILRE_SELFTEST_GRID_BARRIER 1
+#define ILRE_SELFTEST_MISSING_KEY_TILE 2
+int ilre_recall_selftest_wait(ilre_recall_t* h, int64_t wait_cycle_limit, int32_t what);
+
 /* Number of kernel launches issued by the last run(). */
 int ilre_recall_last_launch_count(ilre_recall_t* h);
 

@@ -89,6 +89,8 @@ struct ilre_recall {
   cudaStream_t last_stream;
   int cand_stride;
   int select_max_grid;                  // co-resident CTAs of the selection kernel
+  long long wait_limit;                 // spin budget of the device waits, SM cycles
+  int inject;                           // failure-detection self test: which wait cannot complete
 };
 
 namespace {
@@ -228,6 +230,7 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out) {
   std::memset(h, 0, sizeof(*h));
   h->cfg = *cfg;
   h->n_sm = prop.multiProcessorCount;
+  h->wait_limit = kWaitCycleLimit;
 
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
@@ -394,6 +397,8 @@ int recall_impl(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const void
   qk.c2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(kHeadDim)));
   qk.partial = h->partial; qk.enc = h->enc; qk.status = h->status;
   qk.clk = h->profiling ? h->clk : nullptr;
+  qk.wait_limit = h->wait_limit;
+  qk.skip_tiles = (h->inject == ILRE_SELFTEST_MISSING_KEY_TILE) ? 1 : 0;
 
   PrepParams pp;
   std::memset(&pp, 0, sizeof(pp));
@@ -420,6 +425,8 @@ int recall_impl(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const void
   sp.cand_count = h->cand_count; sp.ranked = h->ranked; sp.bitmap = h->bitmap;
   sp.out_idx = out_idx_dev; sp.budget = budget; sp.barrier = h->grid_barrier;
   sp.status = h->status;
+  sp.wait_limit = h->wait_limit;
+  sp.barrier_extra = (h->inject == ILRE_SELFTEST_GRID_BARRIER) ? 1 : 0;
   int max_km = 1;
   for (int c = 0; c < tbl.n_comb; ++c) max_km = tbl.k_m[c] > max_km ? tbl.k_m[c] : max_km;
   const size_t select_smem = select_smem_bytes(L, max_km, &sp);
@@ -786,6 +793,14 @@ int ilre_recall_sm_clock(ilre_recall_t* h, float* mhz_out_host) {
   unsigned long long w[2] = {0, 0};
   ILRE_CUDA(cudaMemcpy(w, h->clk, sizeof(w), cudaMemcpyDeviceToHost));
   *mhz_out_host = (w[1] > 0) ? static_cast<float>(1e3 * static_cast<double>(w[0]) / static_cast<double>(w[1])) : 0.f;
+  return ILRE_OK;
+}
+
+int ilre_recall_selftest_wait(ilre_recall_t* h, int64_t wait_cycle_limit, int32_t what) {
+  if (!h || wait_cycle_limit < 0 || what < ILRE_SELFTEST_OFF || what > ILRE_SELFTEST_MISSING_KEY_TILE)
+    return ILRE_ERR_INVALID_ARG;
+  h->wait_limit = wait_cycle_limit > 0 ? wait_cycle_limit : kWaitCycleLimit;
+  h->inject = what;
   return ILRE_OK;
 }
 

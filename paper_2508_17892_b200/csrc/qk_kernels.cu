@@ -86,7 +86,8 @@ __device__ __forceinline__ void cta_teardown(uint32_t tmem_base) {
 // TMA producer: the resident Q block once, then the K tiles of this CTA's key range.
 __device__ __forceinline__ void producer_loop(const CUtensorMap* tmapK, const CUtensorMap* tmapQ,
                                               const QkParams& p, const CtaItem& it,
-                                              SmemTail* tail, uint32_t q_s, uint32_t k_s) {
+                                              SmemTail* tail, uint32_t q_s, uint32_t k_s,
+                                              int skip_tiles = 0) {
   volatile int* abort_flag = &tail->abort_flag;
   const uint32_t qf = smem_u32(&tail->q_full);
   mbar_arrive_expect_tx(qf, static_cast<uint32_t>(p.rb_rows) * 256u);
@@ -97,7 +98,7 @@ __device__ __forceinline__ void producer_loop(const CUtensorMap* tmapK, const CU
   // ring position as (stage, phase) counters: no division by the run-time stage count
   int s = 0;
   uint32_t phase = 0;
-  for (int i = 0; i < it.n_tiles; ++i) {
+  for (int i = 0; i < it.n_tiles - skip_tiles; ++i) {
     if (!mbar_wait(smem_u32(&tail->k_empty[s]), phase ^ 1u, abort_flag, p.status, kDevWaitKEmpty))
       break;
     const uint32_t kf = smem_u32(&tail->k_full[s]);
@@ -181,23 +182,23 @@ row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
   }
 
   if (warp == 0) {
-    if (lane == 0 && run) producer_loop(&tmapK, &tmapQ, p, it, tail, q_s, k_s);
+    if (lane == 0 && run) producer_loop(&tmapK, &tmapQ, p, it, tail, q_s, k_s, p.skip_tiles);
   } else if (warp == 1) {
     if (lane == 0 && run) {
       constexpr uint32_t idesc = umma_idesc_bf16(128, kTileKeys);
-      bool ok = mbar_wait(smem_u32(&tail->q_full), 0, abort_flag, p.status, kDevWaitQFull);
+      bool ok = mbar_wait(smem_u32(&tail->q_full), 0, abort_flag, p.status, kDevWaitQFull, p.wait_limit);
       tc_fence_after();
       uint32_t u = 0;
       int s = 0;
       uint32_t kphase = 0;
       for (int i = 0; i < it.n_tiles && ok; ++i) {
-        ok = mbar_wait(smem_u32(&tail->k_full[s]), kphase, abort_flag, p.status, kDevWaitKFull);
+        ok = mbar_wait(smem_u32(&tail->k_full[s]), kphase, abort_flag, p.status, kDevWaitKFull, p.wait_limit);
         if (!ok) break;
         tc_fence_after();
         for (int mt = 0; mt < MT; ++mt, ++u) {
           const uint32_t b = u & 3u, use = u >> 2;
           ok = mbar_wait(smem_u32(&tail->acc_empty[b]), (use & 1u) ^ 1u, abort_flag, p.status,
-                         kDevWaitAccEmpty);
+                         kDevWaitAccEmpty, p.wait_limit);
           if (!ok) break;
           tc_fence_after();
 #pragma unroll
@@ -237,7 +238,7 @@ row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
       const int valid = static_cast<int>(min(static_cast<long long>(kTileKeys), p.L - key0));
       const uint32_t b = u & 3u, use = u >> 2;
       if (!mbar_wait(smem_u32(&tail->acc_full[b]), use & 1u, abort_flag, p.status,
-                     kDevWaitAccFull))
+                     kDevWaitAccFull, p.wait_limit))
         break;
       tc_fence_after();
       float mr = m[0], zr = z[0];

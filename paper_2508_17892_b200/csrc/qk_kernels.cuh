@@ -51,6 +51,11 @@ struct QkParams {
   // in nanoseconds of the global timer: their ratio is the SM clock the kernel really ran at
   // (under the power cap it is well below what the driver reports).
   unsigned long long* clk;
+  // Failure-detection self test (see ilre_recall_selftest_wait): spin budget of the
+  // row-statistics kernel's waits in SM cycles, and how many of its last key tiles the
+  // producer leaves out (0 in normal operation).
+  long long wait_limit;
+  int skip_tiles;
 };
 
 struct PrepParams {

@@ -66,13 +66,13 @@ __device__ __forceinline__ bool grid_sync(const SelectParams& p, SelShared* sh, 
   __syncthreads();
   if (threadIdx.x == 0) {
     int ok = 1;
-    const uint32_t target = epoch * gridDim.x;
+    const uint32_t target = epoch * (gridDim.x + static_cast<uint32_t>(p.barrier_extra));
     __threadfence();
     atomicAdd(p.barrier, 1u);
     volatile uint32_t* arrivals = p.barrier;
     const long long t0 = clock64();
     for (uint32_t it = 1; *arrivals < target; ++it) {
-      if ((it & 0xFF) == 0 && clock64() - t0 > kWaitCycleLimit) {
+      if ((it & 0xFF) == 0 && clock64() - t0 > p.wait_limit) {
         atomicCAS(p.status, 0, kDevGridBarrier);
         ok = 0;
         break;

@@ -63,6 +63,11 @@ struct SelectParams {
   int budget;
   uint32_t* barrier;       // grid barrier arrival counter, zero when the kernel starts
   int* status;
+  // Failure-detection self test (see ilre_recall_selftest_wait): spin budget of a grid
+  // barrier in SM cycles, and how many CTAs more than the grid has the barrier waits for
+  // (0 in normal operation).
+  long long wait_limit;
+  int barrier_extra;
 };
 
 // Dynamic shared memory the kernel needs for a context of L positions.

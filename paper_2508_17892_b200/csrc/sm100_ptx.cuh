@@ -66,14 +66,15 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // CTA already raised *abort_flag (shared memory), or this wait ran past the cycle limit, in
 // which case it raises the flag and records `code` in the global status word.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int* status, int code) {
+                                          int* status, int code,
+                                          long long cycle_limit = kWaitCycleLimit) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 0x3FF) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitCycleLimit) {
+      if (clock64() - t0 > cycle_limit) {
         *abort_flag = 1;
         atomicCAS(status, 0, code);
         return false;

@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = (
     "ilre_gather_input_ids",
     "ilre_layer_recall",
     "ilre_recall_copy_row_lse",
-    "ilre_recall_status", "ilre_recall_set_profiling", "ilre_recall_stage_times",
+    "ilre_recall_status", "ilre_recall_selftest_wait", "ilre_recall_set_profiling", "ilre_recall_stage_times",
     "ilre_recall_sm_clock",
     "ilre_recall_last_launch_count", "ilre_recall_destroy", "ilre_strerror",
     "ilre_topk_positions_noalloc",
@@ -83,6 +83,7 @@ def load_library() -> ctypes.CDLL:
     lib.ilre_recall_status.argtypes = [vp]
     lib.ilre_recall_sm_clock.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     lib.ilre_recall_set_profiling.argtypes = [vp, i32]
+    lib.ilre_recall_selftest_wait.argtypes = [vp, i64, i32]
     lib.ilre_recall_stage_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float), i32]
     lib.ilre_recall_last_launch_count.argtypes = [vp]
     lib.ilre_recall_destroy.argtypes = [vp]
@@ -393,6 +394,14 @@ class IlreRecall:
         rc = self.status()
         if rc != 0:
             raise IlreError(rc, "ilre_recall_status")
+
+    def selftest_wait(self, wait_cycle_limit: int = 0, what: int = 0) -> None:
+        """Failure-detection self test: spin budget (SM cycles, 0 = default) of the kernels'
+        bounded waits for the following runs, and which wait is made impossible to complete
+        (0 none, 1 the Algorithm 1 kernel's grid barrier, 2 a key tile that never arrives)."""
+        rc = self._lib.ilre_recall_selftest_wait(self._h, int(wait_cycle_limit), int(what))
+        if rc != 0:
+            raise IlreError(rc, "ilre_recall_selftest_wait")
 
     def set_profiling(self, on: bool) -> None:
         self._lib.ilre_recall_set_profiling(self._h, int(on))

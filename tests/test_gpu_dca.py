@@ -112,6 +112,69 @@ def test_recall_on_rerotated_keys_matches_oracle():
     eng.close()
 
 
+@pytest.mark.parametrize("name,chunk,n_sink", [("cfg2_L32k", 1024, 0), ("cfg3_L128k", 4096, 4)])
+def test_recall_with_dca_against_the_oracle_pipeline(name, chunk, n_sink):
+    """DCA on (Eq. 7 -> Eq. 4, Eq. 5, Algorithm 1) as one path against the oracle's pipeline
+    `dca_rerope -> round to bf16 -> scores -> allocate`, position by position.
+
+    The device's re-rotated cache differs from the oracle's correctly rounded one in rare
+    elements by one bf16 unit.  What such a difference can do to a score is bounded from the
+    inputs alone: a logit of position t moves by at most
+    delta_t = max_r |q_r . (K_dev[t] - K_ref[t])| / sqrt(d), every row's lse by at most
+    delta_lse (taken from the oracle's statistics on the two caches), so a score moves by at
+    most the factor exp(delta_t + delta_lse).  Where the two caches agree (delta_t = 0) the
+    plain score tolerance (plus delta_lse) applies."""
+    from workloads import CONFIGS
+    from paper_2508_17892_b200 import IlreRecall
+    w = CONFIGS[name]
+    x = make_inputs(w)
+    ref_keys = torch.from_numpy(oracle.round_to_bf16(oracle.dca_rerope(x.K, chunk, n_sink))
+                                .view(np.int16)).view(torch.bfloat16).reshape(x.K.shape)
+    eng = IlreRecall(max_L=w.L, max_q_len=w.q_len, max_budget=w.budget)
+    Kd = torch.empty_like(x.K, device="cuda")
+    eng.rerope_keys(x.K.cuda(), chunk, n_sink, out=Kd)
+    spec = (w.budget, w.max_sizes, w.win_sizes, w.win_op, n_sink)
+    idx, sc = eng.run(Kd, x.Q.cuda(), *spec, want_scores=True)
+    torch.cuda.synchronize()
+    eng.check_status()
+    idx, sc, Kd = idx.cpu().numpy(), sc.cpu().numpy().astype(np.float64), Kd.cpu()
+    same_rows = (Kd.view(torch.int16) == ref_keys.view(torch.int16)).all(dim=2).all(dim=1).numpy()
+    assert same_rows.mean() > 0.1                     # plenty of positions with identical keys
+    # the recall itself, exactly, on the device's own cache
+    a_dev, m_d, z_d = oracle.scores(Kd, x.Q, with_stats=True)
+    parity.check_recall(Kd, x.Q, w, idx, sc, ref_scores=a_dev, spec=spec)
+    # the whole path against the oracle's pipeline
+    a_ref, m_r, z_r = oracle.scores(ref_keys, x.Q, with_stats=True)
+    delta_lse = np.abs((m_d + np.log(z_d)) - (m_r + np.log(z_r))).max()
+    diff = Kd.to(torch.float64) - ref_keys.to(torch.float64)             # [L, n_kv, d], sparse
+    q = x.Q.to(torch.float64)
+    group = w.n_q_heads // w.n_kv_heads
+    delta = np.zeros(w.L)
+    touched = np.flatnonzero(~same_rows)
+    for g in range(w.n_kv_heads):
+        qg = q[:, g * group:(g + 1) * group, :].reshape(-1, w.d)        # rows of this kv head
+        dl = (diff[touched, g, :] @ qg.T).abs().max(dim=1).values.numpy() / np.sqrt(w.d)
+        delta[touched] = np.maximum(delta[touched], dl)
+    assert delta.max() < 0.05
+    bound = parity.SCORE_RTOL * a_ref + parity.SCORE_ATOL + a_ref * np.expm1(delta + delta_lse)
+    err = np.abs(sc - a_ref)
+    assert np.all(err <= bound), (int(np.argmax(err / bound)), float((err / bound).max()))
+    assert np.all(err[same_rows] <= (parity.SCORE_RTOL + 2 * delta_lse) * a_ref[same_rows]
+                  + parity.SCORE_ATOL)
+    # the index list: every combination's choice judged on the oracle pipeline's pooled
+    # values, near-ties widened by what the differing cache elements can move a score
+    own, diag = oracle.allocate(sc, *spec, avg_single=True, diagnostics=True)
+    assert np.array_equal(own, idx)
+    bad = parity.decisions_within_tolerance(
+        a_ref, diag["combination_of"], *spec,
+        rtol=parity.SCORE_RTOL + float(np.expm1(delta.max() + delta_lse)))
+    assert not bad, bad[:10]
+    ref_idx = oracle.allocate(a_ref, *spec)
+    print(name, "positions with identical keys", same_rows.mean(), "max delta", delta.max(),
+          "delta_lse", delta_lse, "index differences", len(set(idx.tolist()) ^ set(ref_idx.tolist())))
+    eng.close()
+
+
 # ---- Eq. 6: sink keys of the layers before the retrieval layer ----
 
 SINK_CASES = [
