@@ -66,6 +66,7 @@ struct ilre_recall {
   cudaStream_t pos_stream;
   unsigned long long* cand;
   uint32_t* cand_count;
+  unsigned long long* pending;
   int* ranked;
   uint32_t* bitmap;
   int* status;
@@ -140,7 +141,7 @@ void free_all(ilre_recall* h) {
   cudaFree(h->qp); cudaFree(h->partial); cudaFree(h->row_lse);
   cudaFree(h->enc); cudaFree(h->scores); cudaFree(h->pooled); cudaFree(h->maxpooled); cudaFree(h->hist);
   cudaFree(h->tile_ties); cudaFree(h->grid_barrier); cudaFree(h->rope_table); cudaFree(h->pos_lo); cudaFree(h->pos_hi);
-  cudaFree(h->cand); cudaFree(h->cand_count); cudaFree(h->ranked); cudaFree(h->bitmap);
+  cudaFree(h->cand); cudaFree(h->cand_count); cudaFree(h->pending); cudaFree(h->ranked); cudaFree(h->bitmap);
   cudaFree(h->status); cudaFree(h->clk); cudaFree(h->stage_k); cudaFree(h->stage_q); cudaFree(h->stage_idx);
   cudaFree(h->piece_stats);
   if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
@@ -266,7 +267,8 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out) {
   ok = ok && dev_alloc(&h->pos_lo, static_cast<size_t>(kRopeLoRows) * 64);
   ok = ok && dev_alloc(&h->pos_hi, static_cast<size_t>(h->pos_hi_rows) * 64);
   ok = ok && dev_alloc(&h->cand, ncomb * h->cand_stride);
-  ok = ok && dev_alloc(&h->cand_count, ncomb);
+  ok = ok && dev_alloc(&h->cand_count, 4 * static_cast<size_t>(kMaxCombos));
+  ok = ok && dev_alloc(&h->pending, ncomb * kPendCap);
   ok = ok && dev_alloc(&h->ranked, ncomb * h->cand_stride);
   ok = ok && dev_alloc(&h->bitmap, (maxL + 31) / 32);
   ok = ok && dev_alloc(&h->status, 1);
@@ -408,6 +410,7 @@ int recall_impl(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const void
   pp.n_comb = tbl.n_comb;
   pp.hist_words = static_cast<long long>(kSelectPasses) * tbl.n_comb * kHistBins;
   pp.cand_count = h->cand_count; pp.grid_barrier = h->grid_barrier;
+  pp.sel_state_words = 4 * kMaxCombos;
 
   MergeParams mp;
   mp.n_groups = g.n_groups; mp.n_rb = g.n_rb; mp.rb_rows = g.rb_rows; mp.cpg = g.cpg;
@@ -422,7 +425,7 @@ int recall_impl(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const void
   sp.maxpooled = h->maxpooled; sp.maxpooled_stride = h->cfg.max_L / 2 + 1;
   sp.tile_ties = h->tile_ties;
   sp.cand = h->cand; sp.cand_stride = h->cand_stride;
-  sp.cand_count = h->cand_count; sp.ranked = h->ranked; sp.bitmap = h->bitmap;
+  sp.cand_count = h->cand_count; sp.pending = h->pending; sp.ranked = h->ranked; sp.bitmap = h->bitmap;
   sp.out_idx = out_idx_dev; sp.budget = budget; sp.barrier = h->grid_barrier;
   sp.status = h->status;
   sp.wait_limit = h->wait_limit;

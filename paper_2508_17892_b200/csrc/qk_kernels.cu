@@ -520,9 +520,7 @@ __global__ void prepare_kernel(const uint4* __restrict__ q, uint4* __restrict__ 
   }
   for (long long e = tid; e < p.hist_words; e += nthreads) p.hist[e] = 0u;
   if (tid == 0) *p.grid_barrier = 0u;
-  for (long long c = tid; c < p.n_comb; c += nthreads) {
-    p.cand_count[c] = 0u;
-  }
+  for (long long c = tid; c < p.sel_state_words; c += nthreads) p.cand_count[c] = 0u;
 }
 
 // ---------------------------------------------------------------------------------------

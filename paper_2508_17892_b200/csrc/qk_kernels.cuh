@@ -67,7 +67,8 @@ struct PrepParams {
   uint32_t* hist;
   long long hist_words;     // words of the radix histograms to clear
   int n_comb;
-  uint32_t* cand_count;
+  uint32_t* cand_count;     // per-run state words of the selection kernel, cleared here
+  int sel_state_words;
   uint32_t* grid_barrier;   // arrival counter of the selection kernel's grid barrier
 };
 

@@ -55,6 +55,8 @@ struct SelShared {
   unsigned long long prefix[kMaxCombos];   // per combination: radix prefix found so far
   uint32_t state[kMaxCombos];              // per combination: threshold settled / candidate count
   uint32_t krem[kMaxCombos];               // per combination: keys still wanted inside the prefix
+  uint8_t mode[kMaxCombos];                // per combination, after the first pass: 0 settled,
+                                           // 1 threshold bin handed to one CTA, 2 full-scan passes
   uint32_t tot[2][32];                     // warp totals of the one-barrier block scan
 };
 
@@ -285,6 +287,18 @@ __device__ __forceinline__ void bin_search(const SelectParams& p, int n_comb, in
         sh->prefix[combo] = prefix | (static_cast<unsigned long long>(bin) << shift);
         sh->krem[combo] = new_k;
         sh->state[combo] = (h[j] == new_k) ? 1u : 0u;
+        if (pass == 0 && h[j] != new_k) {
+          // The threshold bin holds more cells than are wanted from it.  Few enough: they are
+          // set aside during the gather and one CTA picks the new_k highest of them; too many
+          // (a plateau across the bin): the remaining passes scan the whole array.
+          if (h[j] <= static_cast<uint32_t>(kPendCap)) {
+            sh->mode[combo] = 1;
+            p.cand_count[2 * kMaxCombos + combo] = new_k;
+          } else {
+            sh->mode[combo] = 2;
+            p.cand_count[3 * kMaxCombos] = 1u;
+          }
+        }
       }
       cum += h[j];
     }
@@ -343,6 +357,89 @@ __device__ __forceinline__ void rank_range(const SelectParams& p, int combo, int
     if (lane == 0 && mine < n)
       ranked[above] = static_cast<int>(0xFFFFFFFFu - static_cast<uint32_t>(key & 0xFFFFFFFFull));
   }
+}
+
+// One CTA picks the `wanted` highest of the n_p keys that the gather set aside for `combo`
+// (all of them share the top 11 bits) and appends them to the combination's candidates.
+// Radix select over the remaining 53 bits, 11/10/11/11/10 per pass, histograms in shared memory.
+__device__ __forceinline__ void resolve_pending(const SelectParams& p, const ComboTable& tbl,
+                                                int combo, int n_p, SelShared* sh) {
+  constexpr int kPer = kPendCap / kSelThreads;
+  const unsigned long long* pend = p.pending + static_cast<long long>(combo) * kPendCap;
+  unsigned long long* cand = p.cand + static_cast<long long>(combo) * p.cand_stride;
+  const uint32_t wanted = __ldcg(&p.cand_count[2 * kMaxCombos + combo]);
+  const uint32_t base = __ldcg(&p.cand_count[combo]);
+  __shared__ unsigned long long s_prefix;
+  __shared__ uint32_t s_krem, s_slot;
+  __shared__ int s_done;
+  unsigned long long key[kPer];
+#pragma unroll
+  for (int j = 0; j < kPer; ++j) {
+    const int i = j * kSelThreads + threadIdx.x;
+    key[j] = (i < n_p) ? __ldcg(&pend[i]) : 0ull;
+  }
+  __syncthreads();                                         // earlier users of the shared words are done
+  if (threadIdx.x == 0) {
+    s_prefix = (key[0] >> 53) << 53;                       // thread 0 holds key 0 (n_p >= 1)
+    s_krem = wanted;
+    s_done = (wanted >= static_cast<uint32_t>(n_p)) || wanted == 0u;
+    s_slot = 0u;
+  }
+  for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) sh->hist[b] = 0u;
+  __syncthreads();
+  const int shifts[5] = {42, 32, 21, 10, 0};
+  const int widths[5] = {11, 10, 11, 11, 10};
+  for (int pass = 0; pass < 5; ++pass) {
+    if (s_done) break;                                     // uniform: read after a barrier
+    const int shift = shifts[pass], bits = widths[pass];
+    const unsigned long long prefix = s_prefix;
+    const uint32_t k_rem = s_krem;
+#pragma unroll
+    for (int j = 0; j < kPer; ++j) {
+      if (j * kSelThreads >= n_p) break;                   // uniform
+      const int i = j * kSelThreads + threadIdx.x;
+      uint32_t digit = 0xFFFFFFFFu;
+      if (i < n_p && ((key[j] ^ prefix) >> (shift + bits)) == 0ull)
+        digit = static_cast<uint32_t>(key[j] >> shift) & ((1u << bits) - 1u);
+      hist_add(sh->hist, digit);
+    }
+    __syncthreads();
+    const uint32_t h0 = sh->hist[kHistBins - 1 - 2 * threadIdx.x];   // bins in descending order
+    const uint32_t h1 = sh->hist[kHistBins - 2 - 2 * threadIdx.x];
+    uint32_t total;
+    const uint32_t excl = block_exclusive_scan(h0 + h1, sh->scan, &total);
+    sh->hist[kHistBins - 1 - 2 * threadIdx.x] = 0u;
+    sh->hist[kHistBins - 2 - 2 * threadIdx.x] = 0u;
+    if (k_rem > excl && k_rem <= excl + h0 + h1) {
+      const bool first = k_rem <= excl + h0;
+      const uint32_t bin = first ? kHistBins - 1 - 2 * threadIdx.x : kHistBins - 2 - 2 * threadIdx.x;
+      const uint32_t above = first ? excl : excl + h0;
+      const uint32_t cnt = first ? h0 : h1;
+      s_prefix = prefix | (static_cast<unsigned long long>(bin) << shift);
+      s_krem = k_rem - above;
+      s_done = (cnt == k_rem - above) || pass == 4;
+    }
+    __syncthreads();
+  }
+  // every key at or above the threshold is wanted: exactly `wanted` of them (keys are distinct)
+  const unsigned long long threshold = (wanted >= static_cast<uint32_t>(n_p)) ? 0ull : s_prefix;
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int j = 0; j < kPer; ++j) {
+    if (j * kSelThreads >= n_p) break;                     // uniform
+    const int i = j * kSelThreads + threadIdx.x;
+    const bool take = wanted != 0u && i < n_p && key[j] >= threshold;
+    const uint32_t votes = __ballot_sync(0xFFFFFFFFu, take);
+    if (votes) {
+      uint32_t slot = 0;
+      if (lane == __ffs(votes) - 1) slot = atomicAdd(&s_slot, __popc(votes));
+      slot = base + __shfl_sync(0xFFFFFFFFu, slot, __ffs(votes) - 1) + __popc(votes & ((1u << lane) - 1u));
+      if (take && slot < static_cast<uint32_t>(tbl.k_m[combo])) cand[slot] = key[j];
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) p.cand_count[combo] = base + s_slot;
+  __syncthreads();
 }
 
 // Bitmap word access of the quota walk.  The bitmap lives in shared memory on the common path;
@@ -444,27 +541,34 @@ __device__ __forceinline__ void allocate(const ComboTable& tbl, const SelectPara
     return min(static_cast<int>(min(sh->state[combo], static_cast<uint32_t>(kMaxKm))),
                tbl.k_m[combo]);
   };
-  // The ranked cells of a combination are copied to shared memory asynchronously; with two
-  // staging buffers the copy of the next combination runs under the walk of the current one.
-  int* const stage_odd = p.stage_double ? staged + p.stage_capacity : staged;
+  // The ranked cells of a combination are copied to shared memory asynchronously, up to
+  // stage_depth combinations ahead in a ring of staging buffers, so that the copies' latency
+  // hides behind the walks of the combinations before them.
+  const int depth = p.stage_depth;
   auto issue_copy = [&](int combo) {
     const int K = candidates(combo);
     const int* ranked = p.ranked + static_cast<long long>(combo) * p.cand_stride;
-    int* dst = (combo & 1) ? stage_odd : staged;
+    int* dst = staged + (combo % depth) * p.stage_capacity;
     for (int r = threadIdx.x; r < K; r += kSelThreads)
       asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst + r)),
                    "l"(ranked + r) : "memory");
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
-  if (tbl.n_comb > 0) issue_copy(0);
+  int issued = 0;                                          // copies issued so far (uniform)
   for (int combo = 0; combo < tbl.n_comb; ++combo) {
     const int m = tbl.m[combo];
     const uint32_t quota = static_cast<uint32_t>(tbl.quota[combo]);
     const int K = candidates(combo);
-    const int* cells = (combo & 1) ? stage_odd : staged;
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    const int* cells = staged + (combo % depth) * p.stage_capacity;
+    // the buffer of copy q last served combination q - depth, which has finished by now
+    while (issued < tbl.n_comb && issued < combo + depth) issue_copy(issued++);
+    switch (issued - 1 - combo) {                            // younger copies may stay in flight
+      case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
+      case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
+      case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
+      default: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+    }
     __syncthreads();
-    if (p.stage_double && combo + 1 < tbl.n_comb) issue_copy(combo + 1);
     const int per = (K + kSelThreads - 1) / kSelThreads;
     const int r0 = min(K, static_cast<int>(threadIdx.x) * per), r1 = min(K, r0 + per);
     uint32_t mine = 0;
@@ -485,7 +589,6 @@ __device__ __forceinline__ void allocate(const ComboTable& tbl, const SelectPara
     }
     if (total < quota && threadIdx.x == 0) atomicCAS(p.status, 0, kDevQuota);
     __syncthreads();                                         // bitmap updates visible to the block
-    if (!p.stage_double && combo + 1 < tbl.n_comb) issue_copy(combo + 1);
   }
 
   // Ascending output.  Every warp owns a contiguous run of bitmap words and reads it 32
@@ -599,85 +702,16 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
     sh.prefix[combo] = 0ull;
     sh.krem[combo] = static_cast<uint32_t>(tbl.k_m[combo]);
     sh.state[combo] = 0u;
+    sh.mode[combo] = 0;
   }
   __syncthreads();
   for (int combo = c_lo; combo <= c_hi; ++combo) bin_search(p, tbl.n_comb, combo, 0, &sh);
-  for (int pass = 1; pass < kSelectPasses; ++pass) {
-    int shift, bits;
-    pass_bits(pass, shift, bits);
-    const uint32_t mask = (1u << bits) - 1u;
-    uint32_t* hist_pass = p.hist + static_cast<long long>(pass) * tbl.n_comb * kHistBins;
-    int cur = -1, load_cursor = 0, cursor = 0;
-    for (int t0 = t_begin; t0 < t_end; t0 += kScanGroup) {
-      float wv[kScanGroup][kTilePer];
-#pragma unroll
-      for (int g = 0; g < kScanGroup; ++g)
-        if (t0 + g < t_end) fetch_tile(tbl, p, t0 + g, load_cursor, sh.state, wv[g]);
-#pragma unroll
-      for (int g = 0; g < kScanGroup; ++g) {
-        const int tile = t0 + g;
-        if (tile >= t_end) break;
-        const int combo = combo_of_tile(tbl, tile, cursor);
-        if (sh.state[combo]) continue;
-        if (combo != cur && cur >= 0)
-          hist_flush(sh.hist, hist_pass + static_cast<long long>(cur) * kHistBins);
-        cur = combo;
-        const unsigned long long prefix = sh.prefix[combo];
-        const int c0 = (tile - tbl.tile_begin[combo]) * kSelTile;
-        const int c1 = min(tbl.len[combo], c0 + kSelTile);
-#pragma unroll
-        for (int k = 0; k < kTilePer; ++k) {
-          const int c = c0 + k * kSelThreads + threadIdx.x;
-          uint32_t digit = 0xFFFFFFFFu;                    // sentinel: does not take part
-          if (c < c1) {
-            const unsigned long long key = make_key(wv[g][k], static_cast<uint32_t>(c));
-            if (((key ^ prefix) >> (shift + bits)) == 0ull)
-              digit = static_cast<uint32_t>(key >> shift) & mask;
-          }
-          hist_add(sh.hist, digit);
-        }
-      }
-    }
-    if (cur >= 0) hist_flush(sh.hist, hist_pass + static_cast<long long>(cur) * kHistBins);
-    if (!grid_sync(p, &sh, epoch)) return;
-    SEL_TRACE("histogram");
-    for (int combo = c_lo; combo <= c_hi; ++combo)
-      if (sh.state[combo] == 0u) bin_search(p, tbl.n_comb, combo, pass, &sh);
-  }
 
-  // ---- D: ties at the K_m-th value, then the gather ----
-  // A combination that is not settled by now has its K_m-th value v (upper half of the
-  // prefix) and wants krem of the cells that hold exactly v: the ones with the lowest index.
-  {
-    int load_cursor = 0, cursor = 0;
-    for (int t0 = t_begin; t0 < t_end; t0 += kScanGroup) {
-      float wv[kScanGroup][kTilePer];
-#pragma unroll
-      for (int g = 0; g < kScanGroup; ++g)
-        if (t0 + g < t_end) fetch_tile(tbl, p, t0 + g, load_cursor, sh.state, wv[g]);
-#pragma unroll
-      for (int g = 0; g < kScanGroup; ++g) {
-        const int tile = t0 + g;
-        if (tile >= t_end) break;
-        const int combo = combo_of_tile(tbl, tile, cursor);
-        if (sh.state[combo]) continue;
-        const uint32_t v_star = static_cast<uint32_t>(sh.prefix[combo] >> 32);
-        const int c0 = (tile - tbl.tile_begin[combo]) * kSelTile;
-        const int c1 = min(tbl.len[combo], c0 + kSelTile);
-        int mine = 0;
-#pragma unroll
-        for (int k = 0; k < kTilePer; ++k) {
-          const int c = c0 + k * kSelThreads + threadIdx.x;
-          mine += (c < c1 && float_to_ordered(wv[g][k]) == v_star) ? 1 : 0;
-        }
-        const int holders = __syncthreads_count(mine & 1) + 2 * __syncthreads_count(mine & 2) +
-                            4 * __syncthreads_count(mine & 4);
-        if (threadIdx.x == 0) p.tile_ties[tile] = holders;
-      }
-    }
-  }
-  if (!grid_sync(p, &sh, epoch)) return;
-  SEL_TRACE("tie count");
+  // ---- D: the gather.  After the first pass a combination knows the bin (top 11 bits of the
+  // key) that holds its K_m-th value.  One scan settles almost everything: cells above that
+  // bin are candidates; where every cell of the bin is wanted too (or few cells exist), the
+  // bin's cells are candidates as well; otherwise the bin's cells are set aside (at most
+  // kPendCap of them) and one CTA picks the wanted number of highest keys among them.
   {
     const int lane = threadIdx.x & 31;
     int load_cursor = 0, cursor = 0;
@@ -691,43 +725,28 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
         const int tile = t0 + g;
         if (tile >= t_end) break;
         const int combo = combo_of_tile(tbl, tile, cursor);
-        const bool settled = sh.state[combo] != 0u;
+        const int mode = sh.mode[combo];
+        if (mode == 2) continue;                             // left to the full-scan passes
         const unsigned long long threshold = sh.prefix[combo];
-        const uint32_t v_star = static_cast<uint32_t>(threshold >> 32);
-        const uint32_t wanted = sh.krem[combo];
+        const uint32_t bin = static_cast<uint32_t>(threshold >> 53);
         unsigned long long* cand = p.cand + static_cast<long long>(combo) * p.cand_stride;
+        unsigned long long* pend = p.pending + static_cast<long long>(combo) * kPendCap;
         const int c0 = (tile - tbl.tile_begin[combo]) * kSelTile;
         const int c1 = min(tbl.len[combo], c0 + kSelTile);
-        // holders of v in the earlier tiles of this combination (tiles are in cell order)
-        uint32_t before = 0;
-        bool ties_here = false;
-        if (!settled) {
-          ties_here = __ldcg(&p.tile_ties[tile]) > 0;      // uniform
-          if (ties_here) {
-            uint32_t part = 0;
-            for (int t = tbl.tile_begin[combo] + threadIdx.x; t < tile; t += kSelThreads)
-              part += static_cast<uint32_t>(__ldcg(&p.tile_ties[t]));
-            block_exclusive_scan_1(part, sh.tot, 0, &before);
-            __syncthreads();
-          }
-        }
 #pragma unroll
         for (int k = 0; k < kTilePer; ++k) {
           const int c = c0 + k * kSelThreads + threadIdx.x;
           unsigned long long key = 0ull;
-          bool take = false, holder = false;
+          bool take = false, aside = false;
           if (c < c1) {
             key = make_key(wv[g][k], static_cast<uint32_t>(c));
-            const uint32_t v = static_cast<uint32_t>(key >> 32);
-            if (settled) take = key >= threshold;
-            else { take = v > v_star; holder = v == v_star; }
-          }
-          if (ties_here) {                                 // uniform
-            uint32_t in_row;
-            const uint32_t rank = before + block_exclusive_scan_1(holder ? 1u : 0u, sh.tot, 1, &in_row);
-            __syncthreads();
-            if (holder && rank < wanted) take = true;
-            before += in_row;
+            if (mode == 0) {
+              take = key >= threshold;
+            } else {
+              const uint32_t digit = static_cast<uint32_t>(key >> 53);
+              take = digit > bin;
+              aside = digit == bin;
+            }
           }
           const uint32_t votes = __ballot_sync(0xFFFFFFFFu, take);
           if (votes) {
@@ -737,12 +756,181 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
                    __popc(votes & ((1u << lane) - 1u));
             if (take && slot < static_cast<uint32_t>(tbl.k_m[combo])) cand[slot] = key;
           }
+          const uint32_t held = __ballot_sync(0xFFFFFFFFu, aside);
+          if (held) {
+            uint32_t slot = 0;
+            if (lane == __ffs(held) - 1)
+              slot = atomicAdd(&p.cand_count[kMaxCombos + combo], __popc(held));
+            slot = __shfl_sync(0xFFFFFFFFu, slot, __ffs(held) - 1) +
+                   __popc(held & ((1u << lane) - 1u));
+            if (aside && slot < static_cast<uint32_t>(kPendCap)) pend[slot] = key;
+          }
         }
       }
     }
   }
   if (!grid_sync(p, &sh, epoch)) return;
   SEL_TRACE("gather");
+
+  // The cells set aside: one CTA per combination selects the highest `wanted` keys among them
+  // (radix select over the remaining 53 bits of the key in shared memory) and appends them.
+  for (int combo = blockIdx.x; combo < tbl.n_comb; combo += gridDim.x) {
+    const int n_p = static_cast<int>(min(__ldcg(&p.cand_count[kMaxCombos + combo]),
+                                         static_cast<uint32_t>(kPendCap)));
+    if (n_p == 0) continue;                                  // uniform
+    resolve_pending(p, tbl, combo, n_p, &sh);
+  }
+  SEL_TRACE("resolve");
+
+  // A plateau across a whole bin (more than kPendCap equal-digit cells): the remaining passes
+  // over the array, for those combinations only.  The flag is the same for every CTA.
+  if (__ldcg(&p.cand_count[3 * kMaxCombos]) != 0u) {
+    for (int combo = c_lo + threadIdx.x; combo <= c_hi; combo += kSelThreads)
+      if (sh.mode[combo] != 2) sh.state[combo] = 1u;         // nothing left to do for these
+    __syncthreads();
+    for (int pass = 1; pass < kSelectPasses; ++pass) {
+      int shift, bits;
+      pass_bits(pass, shift, bits);
+      const uint32_t mask = (1u << bits) - 1u;
+      uint32_t* hist_pass = p.hist + static_cast<long long>(pass) * tbl.n_comb * kHistBins;
+      int cur = -1, load_cursor = 0, cursor = 0;
+      for (int t0 = t_begin; t0 < t_end; t0 += kScanGroup) {
+        float wv[kScanGroup][kTilePer];
+#pragma unroll
+        for (int g = 0; g < kScanGroup; ++g)
+          if (t0 + g < t_end) fetch_tile(tbl, p, t0 + g, load_cursor, sh.state, wv[g]);
+#pragma unroll
+        for (int g = 0; g < kScanGroup; ++g) {
+          const int tile = t0 + g;
+          if (tile >= t_end) break;
+          const int combo = combo_of_tile(tbl, tile, cursor);
+          if (sh.state[combo]) continue;
+          if (combo != cur && cur >= 0)
+            hist_flush(sh.hist, hist_pass + static_cast<long long>(cur) * kHistBins);
+          cur = combo;
+          const unsigned long long prefix = sh.prefix[combo];
+          const int c0 = (tile - tbl.tile_begin[combo]) * kSelTile;
+          const int c1 = min(tbl.len[combo], c0 + kSelTile);
+#pragma unroll
+          for (int k = 0; k < kTilePer; ++k) {
+            const int c = c0 + k * kSelThreads + threadIdx.x;
+            uint32_t digit = 0xFFFFFFFFu;                    // sentinel: does not take part
+            if (c < c1) {
+              const unsigned long long key = make_key(wv[g][k], static_cast<uint32_t>(c));
+              if (((key ^ prefix) >> (shift + bits)) == 0ull)
+                digit = static_cast<uint32_t>(key >> shift) & mask;
+            }
+            hist_add(sh.hist, digit);
+          }
+        }
+      }
+      if (cur >= 0) hist_flush(sh.hist, hist_pass + static_cast<long long>(cur) * kHistBins);
+      if (!grid_sync(p, &sh, epoch)) return;
+      SEL_TRACE("histogram");
+      for (int combo = c_lo; combo <= c_hi; ++combo)
+        if (sh.state[combo] == 0u) bin_search(p, tbl.n_comb, combo, pass, &sh);
+    }
+
+    // ---- D: ties at the K_m-th value, then the gather ----
+    // A combination that is not settled by now has its K_m-th value v (upper half of the
+    // prefix) and wants krem of the cells that hold exactly v: the ones with the lowest index.
+    {
+      int load_cursor = 0, cursor = 0;
+      for (int t0 = t_begin; t0 < t_end; t0 += kScanGroup) {
+        float wv[kScanGroup][kTilePer];
+#pragma unroll
+        for (int g = 0; g < kScanGroup; ++g)
+          if (t0 + g < t_end) fetch_tile(tbl, p, t0 + g, load_cursor, sh.state, wv[g]);
+#pragma unroll
+        for (int g = 0; g < kScanGroup; ++g) {
+          const int tile = t0 + g;
+          if (tile >= t_end) break;
+          const int combo = combo_of_tile(tbl, tile, cursor);
+          if (sh.state[combo]) continue;
+          const uint32_t v_star = static_cast<uint32_t>(sh.prefix[combo] >> 32);
+          const int c0 = (tile - tbl.tile_begin[combo]) * kSelTile;
+          const int c1 = min(tbl.len[combo], c0 + kSelTile);
+          int mine = 0;
+#pragma unroll
+          for (int k = 0; k < kTilePer; ++k) {
+            const int c = c0 + k * kSelThreads + threadIdx.x;
+            mine += (c < c1 && float_to_ordered(wv[g][k]) == v_star) ? 1 : 0;
+          }
+          const int holders = __syncthreads_count(mine & 1) + 2 * __syncthreads_count(mine & 2) +
+                              4 * __syncthreads_count(mine & 4);
+          if (threadIdx.x == 0) p.tile_ties[tile] = holders;
+        }
+      }
+    }
+    if (!grid_sync(p, &sh, epoch)) return;
+    SEL_TRACE("tie count");
+    {
+      const int lane = threadIdx.x & 31;
+      int load_cursor = 0, cursor = 0;
+      for (int t0 = t_begin; t0 < t_end; t0 += kScanGroup) {
+        float wv[kScanGroup][kTilePer];
+#pragma unroll
+        for (int g = 0; g < kScanGroup; ++g)
+          if (t0 + g < t_end) fetch_tile(tbl, p, t0 + g, load_cursor, nullptr, wv[g]);
+#pragma unroll
+        for (int g = 0; g < kScanGroup; ++g) {
+          const int tile = t0 + g;
+          if (tile >= t_end) break;
+          const int combo = combo_of_tile(tbl, tile, cursor);
+          if (sh.mode[combo] != 2) continue;                   // gathered in the first scan
+          const bool settled = sh.state[combo] != 0u;
+          const unsigned long long threshold = sh.prefix[combo];
+          const uint32_t v_star = static_cast<uint32_t>(threshold >> 32);
+          const uint32_t wanted = sh.krem[combo];
+          unsigned long long* cand = p.cand + static_cast<long long>(combo) * p.cand_stride;
+          const int c0 = (tile - tbl.tile_begin[combo]) * kSelTile;
+          const int c1 = min(tbl.len[combo], c0 + kSelTile);
+          // holders of v in the earlier tiles of this combination (tiles are in cell order)
+          uint32_t before = 0;
+          bool ties_here = false;
+          if (!settled) {
+            ties_here = __ldcg(&p.tile_ties[tile]) > 0;      // uniform
+            if (ties_here) {
+              uint32_t part = 0;
+              for (int t = tbl.tile_begin[combo] + threadIdx.x; t < tile; t += kSelThreads)
+                part += static_cast<uint32_t>(__ldcg(&p.tile_ties[t]));
+              block_exclusive_scan_1(part, sh.tot, 0, &before);
+              __syncthreads();
+            }
+          }
+#pragma unroll
+          for (int k = 0; k < kTilePer; ++k) {
+            const int c = c0 + k * kSelThreads + threadIdx.x;
+            unsigned long long key = 0ull;
+            bool take = false, holder = false;
+            if (c < c1) {
+              key = make_key(wv[g][k], static_cast<uint32_t>(c));
+              const uint32_t v = static_cast<uint32_t>(key >> 32);
+              if (settled) take = key >= threshold;
+              else { take = v > v_star; holder = v == v_star; }
+            }
+            if (ties_here) {                                 // uniform
+              uint32_t in_row;
+              const uint32_t rank = before + block_exclusive_scan_1(holder ? 1u : 0u, sh.tot, 1, &in_row);
+              __syncthreads();
+              if (holder && rank < wanted) take = true;
+              before += in_row;
+            }
+            const uint32_t votes = __ballot_sync(0xFFFFFFFFu, take);
+            if (votes) {
+              uint32_t slot = 0;
+              if (lane == __ffs(votes) - 1) slot = atomicAdd(&p.cand_count[combo], __popc(votes));
+              slot = __shfl_sync(0xFFFFFFFFu, slot, __ffs(votes) - 1) +
+                     __popc(votes & ((1u << lane) - 1u));
+              if (take && slot < static_cast<uint32_t>(tbl.k_m[combo])) cand[slot] = key;
+            }
+          }
+        }
+      }
+    }
+  }
+  if (!grid_sync(p, &sh, epoch)) return;
+  SEL_TRACE("plateau passes");
 
   // ---- E: ranking ----
   {
@@ -799,17 +987,19 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
 // ---------------------------------------------------------------------------------------
 size_t select_smem_bytes(long long L, int max_km, SelectParams* p) {
   size_t bytes = 2 * static_cast<size_t>(kSelTile + kMaxWin) * sizeof(float);  // pooling tiles
-  static_assert(kSrcTileTokens * sizeof(float) <= kRankChunk * sizeof(unsigned long long), "");
-  const size_t rank_bytes = kRankChunk * sizeof(unsigned long long);           // ranking chunk
-  if (rank_bytes > bytes) bytes = rank_bytes;
-  // quota walk: bitmap (when it fits) + one or two staging buffers of max_km cell ids
+  if (kSrcTileTokens * sizeof(float) > bytes) bytes = kSrcTileTokens * sizeof(float);
+  if (kRankChunk * sizeof(unsigned long long) > bytes) bytes = kRankChunk * sizeof(unsigned long long);
+  // quota walk: bitmap (when it fits) + a ring of up to four staging buffers of max_km cell ids
   const size_t cap = (static_cast<size_t>(max_km < 1 ? 1 : max_km) + 3) & ~size_t(3);
   const size_t bm_bytes = (static_cast<size_t>((L + 31) / 32) * sizeof(uint32_t) + 15) & ~size_t(15);
   p->bitmap_in_smem = bm_bytes <= static_cast<size_t>(kSelBitmapSmemBytes) ? 1 : 0;
   const size_t base = p->bitmap_in_smem ? bm_bytes : 0;
   p->stage_capacity = static_cast<int>(cap);
-  p->stage_double = (base + 2 * cap * sizeof(int) <= static_cast<size_t>(kSelMaxDynSmemBytes)) ? 1 : 0;
-  const size_t alloc_bytes = base + (p->stage_double ? 2 : 1) * cap * sizeof(int);
+  size_t depth = (static_cast<size_t>(kSelMaxDynSmemBytes) - base) / (cap * sizeof(int));
+  if (depth > 4) depth = 4;
+  if (depth < 1) depth = 1;
+  p->stage_depth = static_cast<int>(depth);
+  const size_t alloc_bytes = base + depth * cap * sizeof(int);
   if (alloc_bytes > bytes) bytes = alloc_bytes;
   return bytes;
 }

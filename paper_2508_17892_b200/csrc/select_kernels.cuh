@@ -16,6 +16,7 @@ static constexpr int kSelThreads = 1024;    // threads per CTA of the selection 
 static constexpr int kSelTile = 4096;       // cells of one combination per work tile
 static constexpr int kSrcTileTokens = 8192; // tokens per work tile of the strided max-pool
 static constexpr int kRankKeysPerItem = kSelThreads / 32;   // candidates ranked per work item
+static constexpr int kPendCap = 8192;        // cells of the threshold bin resolved by one CTA (else: more passes)
 static constexpr int kSelBitmapSmemBytes = 136 * 1024;   // bitmap kept in shared memory up to this
 static constexpr int kSelMaxDynSmemBytes = kSelBitmapSmemBytes + kMaxKm * 4;
 
@@ -53,12 +54,16 @@ struct SelectParams {
   int* tile_ties;          // [work tiles]: cells of a tile that hold the K_m-th value
   unsigned long long* cand;   // [n_comb][cand_stride] selected 64-bit keys
   int cand_stride;
-  uint32_t* cand_count;
+  uint32_t* cand_count;    // [4 * kMaxCombos]: candidates gathered per combination; then, at
+                           // kMaxCombos, 2 kMaxCombos and 3 kMaxCombos: cells pending in the
+                           // threshold bin, keys still wanted from it, and one flag word
+                           // (some combination needs the full-scan passes); zero on entry
+  unsigned long long* pending;   // [n_comb][kPendCap] keys of the threshold bin
   int* ranked;             // [n_comb][cand_stride] cell ids in rank order
   uint32_t* bitmap;        // [ceil(L/32)] in global memory, used when it does not fit shared memory
   int bitmap_in_smem;
   int stage_capacity;      // cell ids per staging buffer of the quota walk (>= largest K_m)
-  int stage_double;        // two staging buffers fit shared memory
+  int stage_depth;         // staging buffers in the ring (1..4, as shared memory allows)
   int* out_idx;            // [n_sink + budget]
   int budget;
   uint32_t* barrier;       // grid barrier arrival counter, zero when the kernel starts
@@ -71,7 +76,7 @@ struct SelectParams {
 };
 
 // Dynamic shared memory the kernel needs for a context of L positions.
-// Also fills p->bitmap_in_smem, p->stage_capacity and p->stage_double.
+// Also fills p->bitmap_in_smem, p->stage_capacity and p->stage_depth.
 size_t select_smem_bytes(long long L, int max_km, SelectParams* p);
 // Largest grid that is co-resident on the device (the kernel's CTAs wait on one another).
 cudaError_t select_max_grid(int n_sm, int* max_grid);

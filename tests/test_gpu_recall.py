@@ -134,13 +134,17 @@ def test_selection_kernel_edge_paths(case):
     eng.close()
 
 
-@pytest.mark.parametrize("pattern", ["all_equal", "two_levels", "blocks_of_equal"])
+@pytest.mark.parametrize("pattern", ["all_equal", "two_levels", "blocks_of_equal", "all_equal_40k",
+                                     "blocks_of_equal_40k"])
 @pytest.mark.parametrize("win_op", [0, 1])
 def test_massive_ties_follow_the_cell_order(pattern, win_op):
     """Keys that repeat make whole stretches of the scores bit-identical, so the K_m-th value
-    is held by thousands of cells and the lower cell index has to decide (reading 11)."""
+    is held by thousands of cells and the lower cell index has to decide (reading 11).  The
+    plateaus are shorter (one CTA sorts the tied cells out) or longer (further passes over the
+    whole array) than what the selection sets aside for one CTA, sometimes both in one call."""
     import dataclasses
-    L, q_len = 9000, 3
+    L, q_len = (40000, 2) if pattern.endswith("_40k") else (9000, 3)
+    pattern = pattern.replace("_40k", "")
     w = small_workload(L, q_len, seed=3, n_spans=0, budget=700, max_sizes=(1, 2), win_sizes=(1, 3),
                        win_op=win_op, n_sink=2)
     x = make_inputs(w)
@@ -154,7 +158,7 @@ def test_massive_ties_follow_the_cell_order(pattern, win_op):
     else:
         protos = torch.randn(9, 8, 128, generator=g).to(torch.bfloat16)
         for b in range(9):
-            K[b * 1000:(b + 1) * 1000] = protos[b]
+            K[b * (L // 9):(b + 1) * (L // 9)] = protos[b]
     x = dataclasses.replace(x, K=K.contiguous())
     eng = _engine(w)
     idx, sc = _run(eng, x)
