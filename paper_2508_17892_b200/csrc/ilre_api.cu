@@ -430,9 +430,7 @@ int recall_impl(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const void
   sp.status = h->status;
   sp.wait_limit = h->wait_limit;
   sp.barrier_extra = (h->inject == ILRE_SELFTEST_GRID_BARRIER) ? 1 : 0;
-  int max_km = 1;
-  for (int c = 0; c < tbl.n_comb; ++c) max_km = tbl.k_m[c] > max_km ? tbl.k_m[c] : max_km;
-  const size_t select_smem = select_smem_bytes(L, max_km, &sp);
+  const size_t select_smem = select_smem_bytes(L, &sp);
   // Grid of the selection kernel: enough CTAs for the scan tiles and for the ranking
   // (K_m^2 comparisons per combination), but no more, since every grid barrier pays for them.
   long long want_grid = tbl.tile_begin[tbl.n_comb];

@@ -514,9 +514,8 @@ __device__ __forceinline__ uint32_t block_exclusive_scan_1(uint32_t v, uint32_t 
 }
 
 // Phase F (one CTA): quota walk over the ranked cells of every combination, then the
-// ascending list of allocated positions.  `bm` is the bitmap (shared or global memory),
-// `staged` room for kMaxKm cell ids in shared memory.  Every thread owns a run of consecutive
-// ranks; the cells of one combination are disjoint, so the new-token counts of all its cells
+// ascending list of allocated positions.  The bitmap lives in shared memory when it fits,
+// else in global memory.  Every thread owns a run of consecutive ranks; the cells of one combination are disjoint, so the new-token counts of all its cells
 // can be taken before any of them is marked.
 template <bool kBitmapInSmem>
 __device__ __forceinline__ void allocate(const ComboTable& tbl, const SelectParams& p,
@@ -524,13 +523,10 @@ __device__ __forceinline__ void allocate(const ComboTable& tbl, const SelectPara
   // Two instantiations, so that the compiler knows the bitmap's address space on the common
   // path (shared memory) instead of going through generic loads and atomics.
   uint32_t* bm;
-  int* staged;
   if constexpr (kBitmapInSmem) {
     bm = reinterpret_cast<uint32_t*>(dyn_smem);
-    staged = reinterpret_cast<int*>(dyn_smem + ((((p.L + 31) / 32) * 4 + 15) & ~15ll));
   } else {
     bm = p.bitmap;
-    staged = reinterpret_cast<int*>(dyn_smem);
   }
   __shared__ uint32_t warp_totals[2][32];
   const int Lp = static_cast<int>(p.L - p.n_sink);
@@ -541,54 +537,63 @@ __device__ __forceinline__ void allocate(const ComboTable& tbl, const SelectPara
     return min(static_cast<int>(min(sh->state[combo], static_cast<uint32_t>(kMaxKm))),
                tbl.k_m[combo]);
   };
-  // The ranked cells of a combination are copied to shared memory asynchronously, up to
-  // stage_depth combinations ahead in a ring of staging buffers, so that the copies' latency
-  // hides behind the walks of the combinations before them.
-  const int depth = p.stage_depth;
-  auto issue_copy = [&](int combo) {
+  // Thread t owns the ranks [t * per, (t + 1) * per) of a combination.  The first kWalkRegs of
+  // its ranked cells are fetched into registers one combination ahead, so that their latency
+  // hides behind the walk of the combination before; a combination costs one block scan and
+  // two barriers.
+  constexpr int kWalkRegs = 4;
+  auto fetch_cells = [&](int combo, int (&dst)[kWalkRegs]) {
     const int K = candidates(combo);
+    const int per = (K + kSelThreads - 1) / kSelThreads;
+    const int r0 = min(K, static_cast<int>(threadIdx.x) * per), r1 = min(K, r0 + per);
     const int* ranked = p.ranked + static_cast<long long>(combo) * p.cand_stride;
-    int* dst = staged + (combo % depth) * p.stage_capacity;
-    for (int r = threadIdx.x; r < K; r += kSelThreads)
-      asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst + r)),
-                   "l"(ranked + r) : "memory");
-    asm volatile("cp.async.commit_group;" ::: "memory");
+#pragma unroll
+    for (int j = 0; j < kWalkRegs; ++j) dst[j] = (r0 + j < r1) ? __ldcg(&ranked[r0 + j]) : -1;
   };
-  int issued = 0;                                          // copies issued so far (uniform)
+  int cur[kWalkRegs];
+  if (tbl.n_comb > 0) fetch_cells(0, cur);
   for (int combo = 0; combo < tbl.n_comb; ++combo) {
     const int m = tbl.m[combo];
     const uint32_t quota = static_cast<uint32_t>(tbl.quota[combo]);
     const int K = candidates(combo);
-    const int* cells = staged + (combo % depth) * p.stage_capacity;
-    // the buffer of copy q last served combination q - depth, which has finished by now
-    while (issued < tbl.n_comb && issued < combo + depth) issue_copy(issued++);
-    switch (issued - 1 - combo) {                            // younger copies may stay in flight
-      case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
-      case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
-      case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
-      default: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
-    }
-    __syncthreads();
     const int per = (K + kSelThreads - 1) / kSelThreads;
     const int r0 = min(K, static_cast<int>(threadIdx.x) * per), r1 = min(K, r0 + per);
+    const int* ranked = p.ranked + static_cast<long long>(combo) * p.cand_stride;
+    // tokens of every owned cell that are not allocated yet (the cells of one combination are
+    // disjoint, so these masks stay valid while the combination is walked)
+    unsigned long long fresh[kWalkRegs];
     uint32_t mine = 0;
-    for (int r = r0; r < r1; ++r)
-      mine += __popcll(fresh_tokens<kBitmapInSmem>(bm, cells[r], m, Lp, p.n_sink));
+#pragma unroll
+    for (int j = 0; j < kWalkRegs; ++j) {
+      fresh[j] = (cur[j] >= 0) ? fresh_tokens<kBitmapInSmem>(bm, cur[j], m, Lp, p.n_sink) : 0ull;
+      mine += __popcll(fresh[j]);
+    }
+    for (int r = r0 + kWalkRegs; r < r1; ++r)                  // K > kWalkRegs * kSelThreads only
+      mine += __popcll(fresh_tokens<kBitmapInSmem>(bm, __ldcg(&ranked[r]), m, Lp, p.n_sink));
+    int nxt[kWalkRegs];
+    if (combo + 1 < tbl.n_comb) fetch_cells(combo + 1, nxt);   // in flight during the scan
     uint32_t total;
     uint32_t ord = block_exclusive_scan_1(mine, warp_totals, combo & 1, &total);
-    for (int r = r0; r < r1 && ord < quota; ++r) {
-      const int cell = cells[r];
-      unsigned long long fresh = fresh_tokens<kBitmapInSmem>(bm, cell, m, Lp, p.n_sink);
-      while (fresh && ord < quota) {                         // ascending position inside the cell
-        const int j = __ffsll(static_cast<long long>(fresh)) - 1;
-        fresh &= fresh - 1;
+    auto take = [&](int cell, unsigned long long f) {          // ascending position inside the cell
+      while (f && ord < quota) {
+        const int j = __ffsll(static_cast<long long>(f)) - 1;
+        f &= f - 1;
         const int pos = p.n_sink + cell * m + j;
         bitmap_set<kBitmapInSmem>(bm, pos >> 5, 1u << (pos & 31));
         ++ord;
       }
+    };
+#pragma unroll
+    for (int j = 0; j < kWalkRegs; ++j)
+      if (cur[j] >= 0) take(cur[j], fresh[j]);
+    for (int r = r0 + kWalkRegs; r < r1 && ord < quota; ++r) {
+      const int cell = __ldcg(&ranked[r]);
+      take(cell, fresh_tokens<kBitmapInSmem>(bm, cell, m, Lp, p.n_sink));
     }
     if (total < quota && threadIdx.x == 0) atomicCAS(p.status, 0, kDevQuota);
     __syncthreads();                                         // bitmap updates visible to the block
+#pragma unroll
+    for (int j = 0; j < kWalkRegs; ++j) cur[j] = nxt[j];
   }
 
   // Ascending output.  Every warp owns a contiguous run of bitmap words and reads it 32
@@ -611,6 +616,7 @@ __device__ __forceinline__ void allocate(const ComboTable& tbl, const SelectPara
   for (long long k = 0; k < rounds; ++k) {
     const long long w = w_begin + k * 32 + lane;
     uint32_t bits = (w < n_words) ? bitmap_word<kBitmapInSmem>(bm, static_cast<int>(w)) : 0u;
+    if (__ballot_sync(0xFFFFFFFFu, bits != 0u) == 0u) continue;      // nothing allocated in these 1024 positions
     uint32_t incl = __popc(bits);
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -985,22 +991,14 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
 // ---------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------
-size_t select_smem_bytes(long long L, int max_km, SelectParams* p) {
+size_t select_smem_bytes(long long L, SelectParams* p) {
   size_t bytes = 2 * static_cast<size_t>(kSelTile + kMaxWin) * sizeof(float);  // pooling tiles
   if (kSrcTileTokens * sizeof(float) > bytes) bytes = kSrcTileTokens * sizeof(float);
   if (kRankChunk * sizeof(unsigned long long) > bytes) bytes = kRankChunk * sizeof(unsigned long long);
-  // quota walk: bitmap (when it fits) + a ring of up to four staging buffers of max_km cell ids
-  const size_t cap = (static_cast<size_t>(max_km < 1 ? 1 : max_km) + 3) & ~size_t(3);
+  // quota walk: the bitmap, when it fits
   const size_t bm_bytes = (static_cast<size_t>((L + 31) / 32) * sizeof(uint32_t) + 15) & ~size_t(15);
   p->bitmap_in_smem = bm_bytes <= static_cast<size_t>(kSelBitmapSmemBytes) ? 1 : 0;
-  const size_t base = p->bitmap_in_smem ? bm_bytes : 0;
-  p->stage_capacity = static_cast<int>(cap);
-  size_t depth = (static_cast<size_t>(kSelMaxDynSmemBytes) - base) / (cap * sizeof(int));
-  if (depth > 4) depth = 4;
-  if (depth < 1) depth = 1;
-  p->stage_depth = static_cast<int>(depth);
-  const size_t alloc_bytes = base + depth * cap * sizeof(int);
-  if (alloc_bytes > bytes) bytes = alloc_bytes;
+  if (p->bitmap_in_smem && bm_bytes > bytes) bytes = bm_bytes;
   return bytes;
 }
 
