@@ -249,7 +249,7 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out) {
   const size_t max_items = max_groups > static_cast<size_t>(h->n_sm) ? max_groups : h->n_sm;
   const size_t maxL = static_cast<size_t>(cfg->max_L);
   const size_t ncomb = static_cast<size_t>(cfg->max_combinations);
-  h->cand_stride = cfg->max_budget + 2;
+  h->cand_stride = (cfg->max_budget + 2 + 3) & ~3;    // rows of the ranked lists start 16-byte aligned
 
   bool ok = true;
   ok = ok && dev_alloc(reinterpret_cast<uint8_t**>(&h->qp), cfg->n_kv_heads * rows_pad * 256);
@@ -430,7 +430,9 @@ int recall_impl(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const void
   sp.status = h->status;
   sp.wait_limit = h->wait_limit;
   sp.barrier_extra = (h->inject == ILRE_SELFTEST_GRID_BARRIER) ? 1 : 0;
-  const size_t select_smem = select_smem_bytes(L, &sp);
+  int max_km = 1;
+  for (int c = 0; c < tbl.n_comb; ++c) max_km = tbl.k_m[c] > max_km ? tbl.k_m[c] : max_km;
+  const size_t select_smem = select_smem_bytes(L, max_km, &sp);
   // Grid of the selection kernel: enough CTAs for the scan tiles and for the ranking
   // (K_m^2 comparisons per combination), but no more, since every grid barrier pays for them.
   long long want_grid = tbl.tile_begin[tbl.n_comb];

@@ -142,6 +142,7 @@ __device__ __forceinline__ int combo_of_tile(const ComboTable& tbl, int tile, in
 }
 
 static constexpr int kTilePer = kSelTile / kSelThreads;
+static constexpr int kMaxWalkWarps = kSelThreads / 32;
 static constexpr int kScanGroup = 4;      // tiles whose loads are issued together
 
 // Pooled values of one tile, kTilePer per thread, all loads in flight together.
@@ -472,12 +473,20 @@ __device__ __forceinline__ unsigned long long fresh_tokens(const uint32_t* bm, i
     const int pos = n_sink + cell;
     return ((bitmap_word<kSmem>(bm, pos >> 5) >> (pos & 31)) & 1u) ^ 1u;
   }
-  // the cell's cnt <= 64 consecutive bits sit in at most three bitmap words (the bitmap has
-  // ceil(L / 32) words; words past its end are not read)
   const int t0 = cell * m;
   const int cnt = min(m, Lp - t0);
   const int pos0 = n_sink + t0;
   const int w0 = pos0 >> 5, sh = pos0 & 31;
+  if (m <= 32) {
+    // at most 32 consecutive bits: two bitmap words, one funnel shift (the bitmap has
+    // ceil(L / 32) words; a word past its end is not read)
+    const uint32_t lo = bitmap_word<kSmem>(bm, w0);
+    const uint32_t hi = (sh + cnt > 32) ? bitmap_word<kSmem>(bm, w0 + 1) : 0u;
+    const uint32_t taken32 = __funnelshift_r(lo, hi, sh);
+    const uint32_t mask32 = (cnt >= 32) ? 0xFFFFFFFFu : ((1u << cnt) - 1u);
+    return static_cast<unsigned long long>(~taken32 & mask32);
+  }
+  // up to 64 consecutive bits sit in at most three bitmap words
   const int last_w = (pos0 + cnt - 1) >> 5;
   unsigned long long taken = bitmap_word<kSmem>(bm, w0);
   if (last_w > w0) taken |= static_cast<unsigned long long>(bitmap_word<kSmem>(bm, w0 + 1)) << 32;
@@ -523,78 +532,121 @@ __device__ __forceinline__ void allocate(const ComboTable& tbl, const SelectPara
   // Two instantiations, so that the compiler knows the bitmap's address space on the common
   // path (shared memory) instead of going through generic loads and atomics.
   uint32_t* bm;
+  int* staged;
   if constexpr (kBitmapInSmem) {
     bm = reinterpret_cast<uint32_t*>(dyn_smem);
+    staged = reinterpret_cast<int*>(dyn_smem + ((((p.L + 31) / 32) * 4 + 15) & ~15ll));
   } else {
     bm = p.bitmap;
+    staged = reinterpret_cast<int*>(dyn_smem);
   }
-  __shared__ uint32_t warp_totals[2][32];
+  __shared__ uint32_t warp_totals[2][kMaxWalkWarps];
+  const int n_walk = p.walk_threads;                       // multiple of 32, <= kSelThreads
   const int Lp = static_cast<int>(p.L - p.n_sink);
   for (int combo = threadIdx.x; combo < tbl.n_comb; combo += kSelThreads)
     sh->state[combo] = __ldcg(&p.cand_count[combo]);
   __syncthreads();
-  auto candidates = [&](int combo) {
-    return min(static_cast<int>(min(sh->state[combo], static_cast<uint32_t>(kMaxKm))),
-               tbl.k_m[combo]);
-  };
-  // Thread t owns the ranks [t * per, (t + 1) * per) of a combination.  The first kWalkRegs of
-  // its ranked cells are fetched into registers one combination ahead, so that their latency
-  // hides behind the walk of the combination before; a combination costs one block scan and
-  // two barriers.
-  constexpr int kWalkRegs = 4;
-  auto fetch_cells = [&](int combo, int (&dst)[kWalkRegs]) {
-    const int K = candidates(combo);
-    const int per = (K + kSelThreads - 1) / kSelThreads;
-    const int r0 = min(K, static_cast<int>(threadIdx.x) * per), r1 = min(K, r0 + per);
-    const int* ranked = p.ranked + static_cast<long long>(combo) * p.cand_stride;
-#pragma unroll
-    for (int j = 0; j < kWalkRegs; ++j) dst[j] = (r0 + j < r1) ? __ldcg(&ranked[r0 + j]) : -1;
-  };
-  int cur[kWalkRegs];
-  if (tbl.n_comb > 0) fetch_cells(0, cur);
-  for (int combo = 0; combo < tbl.n_comb; ++combo) {
-    const int m = tbl.m[combo];
-    const uint32_t quota = static_cast<uint32_t>(tbl.quota[combo]);
-    const int K = candidates(combo);
-    const int per = (K + kSelThreads - 1) / kSelThreads;
-    const int r0 = min(K, static_cast<int>(threadIdx.x) * per), r1 = min(K, r0 + per);
-    const int* ranked = p.ranked + static_cast<long long>(combo) * p.cand_stride;
-    // tokens of every owned cell that are not allocated yet (the cells of one combination are
-    // disjoint, so these masks stay valid while the combination is walked)
-    unsigned long long fresh[kWalkRegs];
-    uint32_t mine = 0;
-#pragma unroll
-    for (int j = 0; j < kWalkRegs; ++j) {
-      fresh[j] = (cur[j] >= 0) ? fresh_tokens<kBitmapInSmem>(bm, cur[j], m, Lp, p.n_sink) : 0ull;
-      mine += __popcll(fresh[j]);
-    }
-    for (int r = r0 + kWalkRegs; r < r1; ++r)                  // K > kWalkRegs * kSelThreads only
-      mine += __popcll(fresh_tokens<kBitmapInSmem>(bm, __ldcg(&ranked[r]), m, Lp, p.n_sink));
-    int nxt[kWalkRegs];
-    if (combo + 1 < tbl.n_comb) fetch_cells(combo + 1, nxt);   // in flight during the scan
-    uint32_t total;
-    uint32_t ord = block_exclusive_scan_1(mine, warp_totals, combo & 1, &total);
-    auto take = [&](int cell, unsigned long long f) {          // ascending position inside the cell
-      while (f && ord < quota) {
-        const int j = __ffsll(static_cast<long long>(f)) - 1;
-        f &= f - 1;
-        const int pos = p.n_sink + cell * m + j;
-        bitmap_set<kBitmapInSmem>(bm, pos >> 5, 1u << (pos & 31));
-        ++ord;
-      }
+  // The walk is a chain of short dependent steps per combination, so what it costs is the
+  // number of warps that have to issue them: walk_threads threads walk (about two ranked
+  // cells each for the longest list, at least 256), the others wait for the output pass.  The ranked cells of a combination reach shared memory by 16-byte
+  // asynchronous copies, one combination ahead when two staging buffers fit.
+  if (static_cast<int>(threadIdx.x) < n_walk) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    auto walk_barrier = [&] { asm volatile("bar.sync 1, %0;" ::"r"(n_walk) : "memory"); };
+    auto candidates = [&](int combo) {
+      return min(static_cast<int>(min(sh->state[combo], static_cast<uint32_t>(kMaxKm))),
+                 tbl.k_m[combo]);
     };
+    const bool two = p.stage_double != 0;
+    auto issue_copy = [&](int combo) {
+      const int K = candidates(combo);
+      const int* ranked = p.ranked + static_cast<long long>(combo) * p.cand_stride;
+      int* dst = staged + ((two && (combo & 1)) ? p.stage_capacity : 0);
+      for (int r = 4 * threadIdx.x; r < K; r += 4 * n_walk)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst + r)),
+                     "l"(ranked + r) : "memory");
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    if (tbl.n_comb > 0) issue_copy(0);
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    walk_barrier();
+    for (int combo = 0; combo < tbl.n_comb; ++combo) {
+      const int m = tbl.m[combo];
+      const uint32_t quota = static_cast<uint32_t>(tbl.quota[combo]);
+      const int K = candidates(combo);
+      const int* cells = staged + ((two && (combo & 1)) ? p.stage_capacity : 0);
+      // the other buffer last served combination combo - 1, which every thread has left
+      if (two && combo + 1 < tbl.n_comb) issue_copy(combo + 1);
+      // thread t owns the ranks [t * per, (t + 1) * per)
+      const int per = (K + n_walk - 1) / n_walk;
+      const int r0 = min(K, static_cast<int>(threadIdx.x) * per), r1 = min(K, r0 + per);
+      uint32_t mine = 0;
+      int r = r0;
+      for (; r + 4 <= r1; r += 4) {                            // four cells' loads in flight together
+        const int c0 = cells[r], c1 = cells[r + 1], c2 = cells[r + 2], c3 = cells[r + 3];
+        const unsigned long long f0 = fresh_tokens<kBitmapInSmem>(bm, c0, m, Lp, p.n_sink);
+        const unsigned long long f1 = fresh_tokens<kBitmapInSmem>(bm, c1, m, Lp, p.n_sink);
+        const unsigned long long f2 = fresh_tokens<kBitmapInSmem>(bm, c2, m, Lp, p.n_sink);
+        const unsigned long long f3 = fresh_tokens<kBitmapInSmem>(bm, c3, m, Lp, p.n_sink);
+        mine += __popcll(f0) + __popcll(f1) + __popcll(f2) + __popcll(f3);
+      }
+      for (; r < r1; ++r)
+        mine += __popcll(fresh_tokens<kBitmapInSmem>(bm, cells[r], m, Lp, p.n_sink));
+      // exclusive prefix over the walking threads: tokens that higher-ranked cells bring
+      uint32_t incl = mine;
 #pragma unroll
-    for (int j = 0; j < kWalkRegs; ++j)
-      if (cur[j] >= 0) take(cur[j], fresh[j]);
-    for (int r = r0 + kWalkRegs; r < r1 && ord < quota; ++r) {
-      const int cell = __ldcg(&ranked[r]);
-      take(cell, fresh_tokens<kBitmapInSmem>(bm, cell, m, Lp, p.n_sink));
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += t;
+      }
+      if (lane == 31) warp_totals[combo & 1][warp] = incl;
+      walk_barrier();
+      const uint32_t wt = (lane < n_walk / 32) ? warp_totals[combo & 1][lane] : 0u;
+      uint32_t wi = wt;
+#pragma unroll
+      for (int o = 1; o < kMaxWalkWarps; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, wi, o);
+        if (lane >= o) wi += t;
+      }
+      const uint32_t total = __shfl_sync(0xFFFFFFFFu, wi, 31);
+      uint32_t ord = __shfl_sync(0xFFFFFFFFu, wi - wt, warp) + incl - mine;
+      // accept in rank order while the quota lasts; inside a cell in ascending position; the
+      // tokens of a cell are marked with one atomic per bitmap word (at most three words)
+      for (r = r0; r < r1 && ord < quota; ++r) {
+        const int cell = cells[r];
+        unsigned long long f = fresh_tokens<kBitmapInSmem>(bm, cell, m, Lp, p.n_sink);
+        if (f == 0ull) continue;
+        uint32_t n_new = __popcll(f);
+        if (ord + n_new > quota) {                             // the quota ends inside this cell
+          unsigned long long kept = 0ull;
+          for (uint32_t k = quota - ord; k > 0; --k) {
+            const unsigned long long lowest = f & (0ull - f);
+            kept |= lowest;
+            f ^= lowest;
+          }
+          f = kept;
+          n_new = quota - ord;
+        }
+        ord += n_new;
+        const int pos0 = p.n_sink + cell * m;
+        const int w0 = pos0 >> 5, sft = pos0 & 31;
+        const unsigned long long shifted = f << sft;
+        const uint32_t b0 = static_cast<uint32_t>(shifted), b1 = static_cast<uint32_t>(shifted >> 32);
+        const uint32_t b2 = sft ? static_cast<uint32_t>(f >> (64 - sft)) : 0u;
+        if (b0) bitmap_set<kBitmapInSmem>(bm, w0, b0);
+        if (b1) bitmap_set<kBitmapInSmem>(bm, w0 + 1, b1);
+        if (b2) bitmap_set<kBitmapInSmem>(bm, w0 + 2, b2);
+      }
+      if (total < quota && threadIdx.x == 0) atomicCAS(p.status, 0, kDevQuota);
+      if (!two) {                                              // one buffer: copy only once it is free
+        walk_barrier();
+        if (combo + 1 < tbl.n_comb) issue_copy(combo + 1);
+      }
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      walk_barrier();                                          // bitmap updates and the next cells visible
     }
-    if (total < quota && threadIdx.x == 0) atomicCAS(p.status, 0, kDevQuota);
-    __syncthreads();                                         // bitmap updates visible to the block
-#pragma unroll
-    for (int j = 0; j < kWalkRegs; ++j) cur[j] = nxt[j];
   }
+  __syncthreads();
 
   // Ascending output.  Every warp owns a contiguous run of bitmap words and reads it 32
   // consecutive words at a time (one per lane).
@@ -991,14 +1043,21 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
 // ---------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------
-size_t select_smem_bytes(long long L, SelectParams* p) {
+size_t select_smem_bytes(long long L, int max_km, SelectParams* p) {
   size_t bytes = 2 * static_cast<size_t>(kSelTile + kMaxWin) * sizeof(float);  // pooling tiles
   if (kSrcTileTokens * sizeof(float) > bytes) bytes = kSrcTileTokens * sizeof(float);
   if (kRankChunk * sizeof(unsigned long long) > bytes) bytes = kRankChunk * sizeof(unsigned long long);
-  // quota walk: the bitmap, when it fits
+  // quota walk: bitmap (when it fits) + one or two staging buffers of max_km cell ids
+  const size_t cap = (static_cast<size_t>(max_km < 1 ? 1 : max_km) + 3) & ~size_t(3);
   const size_t bm_bytes = (static_cast<size_t>((L + 31) / 32) * sizeof(uint32_t) + 15) & ~size_t(15);
   p->bitmap_in_smem = bm_bytes <= static_cast<size_t>(kSelBitmapSmemBytes) ? 1 : 0;
-  if (p->bitmap_in_smem && bm_bytes > bytes) bytes = bm_bytes;
+  const size_t base = p->bitmap_in_smem ? bm_bytes : 0;
+  int walkers = ((max_km + 1) / 2 + 31) & ~31;               // about two ranked cells per thread
+  p->walk_threads = walkers < 256 ? 256 : (walkers > kSelThreads ? kSelThreads : walkers);
+  p->stage_capacity = static_cast<int>(cap);
+  p->stage_double = (base + 2 * cap * sizeof(int) <= static_cast<size_t>(kSelMaxDynSmemBytes)) ? 1 : 0;
+  const size_t alloc_bytes = base + (p->stage_double ? 2 : 1) * cap * sizeof(int);
+  if (alloc_bytes > bytes) bytes = alloc_bytes;
   return bytes;
 }
 

@@ -18,7 +18,7 @@ static constexpr int kSrcTileTokens = 8192; // tokens per work tile of the strid
 static constexpr int kRankKeysPerItem = kSelThreads / 32;   // candidates ranked per work item
 static constexpr int kPendCap = 8192;        // cells of the threshold bin resolved by one CTA (else: more passes)
 static constexpr int kSelBitmapSmemBytes = 136 * 1024;   // bitmap kept in shared memory up to this
-static constexpr int kSelMaxDynSmemBytes = kSelBitmapSmemBytes;
+static constexpr int kSelMaxDynSmemBytes = kSelBitmapSmemBytes + kMaxKm * 4;
 
 // One entry per (m_i, n_j) combination, in Algorithm 1's loop order.
 struct ComboTable {
@@ -59,9 +59,12 @@ struct SelectParams {
                            // threshold bin, keys still wanted from it, and one flag word
                            // (some combination needs the full-scan passes); zero on entry
   unsigned long long* pending;   // [n_comb][kPendCap] keys of the threshold bin
-  int* ranked;             // [n_comb][cand_stride] cell ids in rank order
+  int* ranked;             // [n_comb][cand_stride] cell ids in rank order (cand_stride: multiple of 4)
   uint32_t* bitmap;        // [ceil(L/32)] in global memory, used when it does not fit shared memory
   int bitmap_in_smem;
+  int stage_capacity;      // cell ids per staging buffer of the quota walk (>= largest K_m, multiple of 4)
+  int stage_double;        // two staging buffers fit shared memory
+  int walk_threads;        // threads that walk the combinations in the allocation phase
   int* out_idx;            // [n_sink + budget]
   int budget;
   uint32_t* barrier;       // grid barrier arrival counter, zero when the kernel starts
@@ -74,8 +77,8 @@ struct SelectParams {
 };
 
 // Dynamic shared memory the kernel needs for a context of L positions.
-// Also fills p->bitmap_in_smem.
-size_t select_smem_bytes(long long L, SelectParams* p);
+// Also fills p->bitmap_in_smem, p->stage_capacity, p->stage_double and p->walk_threads.
+size_t select_smem_bytes(long long L, int max_km, SelectParams* p);
 // Largest grid that is co-resident on the device (the kernel's CTAs wait on one another).
 cudaError_t select_max_grid(int n_sm, int* max_grid);
 // One cooperative launch: A^C from the encoded maxima, then all of Algorithm 1.
