@@ -24,10 +24,7 @@ namespace ilre {
 static constexpr int kAttnStages = 3;
 static constexpr int kAttnTileBytes = 128 * 128 * 2;       // one 128 x 128 bf16 tile
 static constexpr int kAttnTailBytes = 256;
-#ifndef ILRE_ATTN_POLY_PAIRS
-#define ILRE_ATTN_POLY_PAIRS 2
-#endif
-static constexpr int kAttnPolyPairs = ILRE_ATTN_POLY_PAIRS;   // of every 16 pairs of exponentials
+static constexpr int kAttnPolyPairs = 2;                   // of every 16 pairs of exponentials
 static constexpr int kAttnSoftmaxWarps = 4;                // per stream: one per TMEM lane quadrant
 
 struct AttnTail {

@@ -15,10 +15,7 @@ static constexpr int kQkThreads = 384;             // scores: warp 0 TMA, warps 
 static constexpr int kConsumerWarps = 8;
 // Row statistics: warp 0 TMA, warp 1 MMA, then kStatsWarpgroups consumer warpgroups of four
 // warps (one per TMEM lane quadrant); accumulator buffer u belongs to warpgroup u % kStatsWarpgroups.
-#ifndef ILRE_STATS_WARPGROUPS
-#define ILRE_STATS_WARPGROUPS 4
-#endif
-static constexpr int kStatsWarpgroups = ILRE_STATS_WARPGROUPS;
+static constexpr int kStatsWarpgroups = 4;
 // A warpgroup's first accumulator must be one of the first four (the number of TMEM buffers):
 // a parity wait on a buffer that has not completed its first phase yet would pass at once.
 static_assert(kStatsWarpgroups >= 1 && kStatsWarpgroups <= 4, "at most one warpgroup per TMEM buffer");
@@ -29,10 +26,7 @@ static constexpr int kMaxDynSmem = 232448;         // 227 KB per CTA on sm_100
 
 // Row statistics: how many of every 16 logit pairs take 2^x from the FMA-pipe polynomial
 // instead of the special-function unit (0 = none).  Balances the two pipes.
-#ifndef ILRE_ROW_STATS_POLY_PAIRS
-#define ILRE_ROW_STATS_POLY_PAIRS 4
-#endif
-static constexpr int kRowStatsPolyPairs = ILRE_ROW_STATS_POLY_PAIRS;
+static constexpr int kRowStatsPolyPairs = 4;
 
 // Geometry of one recall, shared by both passes.
 struct QkParams {

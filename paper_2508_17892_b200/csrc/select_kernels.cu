@@ -3,14 +3,18 @@
 //
 //   A  A^C[t] = exp2(max_r log2 p_rt) from the scores pass' encoded maxima (Eq. 5);
 //   B  MaxPooling(size = stride = m), once per distinct m, then the stride-1 window pooling
-//      (average or max) of every (m, n) combination, and the first radix histogram;
-//   C  radix select of the K_m-th largest pooled value, 11/11/10 bits per pass, all
-//      combinations at once: the histograms are global, but every CTA works out the bin of
-//      the combinations it scans by itself, so a pass costs one grid barrier;
-//   D  where that value has more holders than are still wanted, the ones with the lowest cell
-//      index win (Algorithm 1's order: value descending, cell ascending): the tiles are in
-//      cell order, so a count of the holders per tile plus an ordered rank inside the tile
-//      settle it; then the gather of the selected keys;
+//      (average or max) of every (m, n) combination, and a histogram of the top 11 bits of
+//      the 64-bit key (pooled value, then lower cell index first);
+//   C  every CTA finds, for the combinations it scans, the histogram bin that holds the
+//      K_m-th largest key;
+//   D  one scan gathers the candidates: cells above that bin, the bin's cells too when all of
+//      them are wanted; otherwise the bin's cells (at most kPendCap) are set aside and one CTA
+//      per combination picks the wanted number of highest keys among them with a radix select
+//      over the remaining 53 bits in shared memory.  Only a plateau of more than kPendCap
+//      cells in the bin (exactly equal pooled values, mostly) takes the long way: two more
+//      histogram passes over the array, then the ties in cell order (the tiles are in cell
+//      order, so a count of the holders per tile plus an ordered rank inside the tile settle
+//      which cells win);
 //   E  ranking (value descending, cell ascending) by counting, spread over the grid;
 //   F  one CTA walks the combinations in loop order: maps cells back to tokens, skips tokens
 //      already allocated, stops each combination at its quota B_c, then writes the allocated
@@ -20,20 +24,6 @@
 // contiguous run of tiles, the same in every phase.
 #include "select_kernels.cuh"
 #include "sm100_ptx.cuh"
-
-// Build with -DILRE_SELECT_TRACE to have CTA 0 print the time spent in every phase.
-#ifdef ILRE_SELECT_TRACE
-#include <cstdio>
-#define SEL_TRACE(tag)                                                              \
-  do {                                                                              \
-    if (blockIdx.x == 0 && threadIdx.x == 0 && trace_n < 32) {                      \
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(trace_t[trace_n]));          \
-      trace_tag[trace_n++] = tag;                                                   \
-    }                                                                               \
-  } while (0)
-#else
-#define SEL_TRACE(tag) do { } while (0)
-#endif
 
 namespace ilre {
 
@@ -696,12 +686,6 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
   const int t_end = static_cast<int>(static_cast<long long>(blockIdx.x + 1) * n_tiles / gridDim.x);
   for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) sh.hist[b] = 0u;
   uint32_t epoch = 0;
-#ifdef ILRE_SELECT_TRACE
-  __shared__ unsigned long long trace_t[32];
-  __shared__ const char* trace_tag[32];
-  int trace_n = 0;
-  SEL_TRACE("start");
-#endif
 
   // ---- A: scores from the encoded maxima, one exp per position ----
   if (!p.scores_given) {
@@ -714,7 +698,6 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
     }
   }
   if (!grid_sync(p, &sh, epoch)) return;
-  SEL_TRACE("scores");
 
   // ---- B1: strided max-pool arrays, one per distinct m > 1 ----
   if (tbl.n_src > 0) {
@@ -728,7 +711,6 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
       maxpool_tile(tbl, p, src, tile - tbl.src_tile_begin[src], buf);
     }
     if (!grid_sync(p, &sh, epoch)) return;
-    SEL_TRACE("maxpool");
   }
 
   // ---- B2: window pooling of every combination + first histogram ----
@@ -746,7 +728,6 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
     if (cur >= 0) hist_flush(sh.hist, p.hist + static_cast<long long>(cur) * kHistBins);
   }
   if (!grid_sync(p, &sh, epoch)) return;
-  SEL_TRACE("pool+hist0");
 
   // ---- C: radix select of the K_m-th largest value ----
   // combinations whose tiles this CTA scans
@@ -828,7 +809,6 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
     }
   }
   if (!grid_sync(p, &sh, epoch)) return;
-  SEL_TRACE("gather");
 
   // The cells set aside: one CTA per combination selects the highest `wanted` keys among them
   // (radix select over the remaining 53 bits of the key in shared memory) and appends them.
@@ -838,7 +818,6 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
     if (n_p == 0) continue;                                  // uniform
     resolve_pending(p, tbl, combo, n_p, &sh);
   }
-  SEL_TRACE("resolve");
 
   // A plateau across a whole bin (more than kPendCap equal-digit cells): the remaining passes
   // over the array, for those combinations only.  The flag is the same for every CTA.
@@ -884,7 +863,6 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
       }
       if (cur >= 0) hist_flush(sh.hist, hist_pass + static_cast<long long>(cur) * kHistBins);
       if (!grid_sync(p, &sh, epoch)) return;
-      SEL_TRACE("histogram");
       for (int combo = c_lo; combo <= c_hi; ++combo)
         if (sh.state[combo] == 0u) bin_search(p, tbl.n_comb, combo, pass, &sh);
     }
@@ -921,7 +899,6 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
       }
     }
     if (!grid_sync(p, &sh, epoch)) return;
-    SEL_TRACE("tie count");
     {
       const int lane = threadIdx.x & 31;
       int load_cursor = 0, cursor = 0;
@@ -988,7 +965,6 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
     }
   }
   if (!grid_sync(p, &sh, epoch)) return;
-  SEL_TRACE("plateau passes");
 
   // ---- E: ranking ----
   {
@@ -1013,7 +989,6 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
     }
   }
   if (!grid_sync(p, &sh, epoch)) return;
-  SEL_TRACE("rank");
 
   // ---- F: allocation and ascending output (one CTA) ----
   if (blockIdx.x != 0) return;
@@ -1027,17 +1002,10 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
       bm[w] = bits;
     }
     __syncthreads();
-    SEL_TRACE("bitmap init");
     allocate<true>(tbl, p, dyn_smem, &sh);
   } else {
     allocate<false>(tbl, p, dyn_smem, &sh);
   }
-  SEL_TRACE("allocate");
-#ifdef ILRE_SELECT_TRACE
-  if (threadIdx.x == 0)
-    for (int i = 1; i < trace_n; ++i)
-      printf("select phase %-12s %8.2f us\n", trace_tag[i], (trace_t[i] - trace_t[i - 1]) * 1e-3);
-#endif
 }
 
 // ---------------------------------------------------------------------------------------
