@@ -433,13 +433,12 @@ int recall_impl(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const void
   int max_km = 1;
   for (int c = 0; c < tbl.n_comb; ++c) max_km = tbl.k_m[c] > max_km ? tbl.k_m[c] : max_km;
   const size_t select_smem = select_smem_bytes(L, max_km, &sp);
-  // Grid of the selection kernel: enough CTAs for the scan tiles and for the ranking
-  // (K_m^2 comparisons per combination), but no more, since every grid barrier pays for them.
+  // Grid of the selection kernel: enough CTAs for the scan tiles and for the ranking (about a
+  // hundred candidates per CTA), but no more, since every grid barrier pays for them.
   long long want_grid = tbl.tile_begin[tbl.n_comb];
-  long long rank_items = 0;
-  for (int c = 0; c < tbl.n_comb; ++c)
-    rank_items += (tbl.k_m[c] + kRankKeysPerItem - 1) / kRankKeysPerItem;
-  if (rank_items / 2 > want_grid) want_grid = rank_items / 2;
+  long long n_cand = 0;
+  for (int c = 0; c < tbl.n_comb; ++c) n_cand += tbl.k_m[c];
+  if (n_cand / 96 > want_grid) want_grid = n_cand / 96;
   if (want_grid < 1) want_grid = 1;
   if (want_grid > h->select_max_grid) want_grid = h->select_max_grid;
   const int select_grid = static_cast<int>(want_grid);

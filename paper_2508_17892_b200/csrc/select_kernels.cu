@@ -52,25 +52,28 @@ struct SelShared {
 
 // Grid-wide barrier (all CTAs are co-resident: cooperative launch).  The arrival counter is
 // zero when the kernel starts and only grows: the k-th barrier completes when it reaches
-// k * gridDim.x.  The wait is bounded; a CTA that gives up records it and leaves the kernel.
+// k * gridDim.x.  One thread per CTA arrives with a release at device scope (cumulative over the
+// CTA's writes, which the block barrier before it orders) and polls with acquire loads; no
+// value comes back from the arrival, so a barrier costs one trip to the L2 instead of two.
+// The wait is bounded; a CTA that gives up records it and leaves the kernel.
 __device__ __forceinline__ bool grid_sync(const SelectParams& p, SelShared* sh, uint32_t& epoch) {
   ++epoch;
   __syncthreads();
   if (threadIdx.x == 0) {
     int ok = 1;
     const uint32_t target = epoch * (gridDim.x + static_cast<uint32_t>(p.barrier_extra));
-    __threadfence();
-    atomicAdd(p.barrier, 1u);
-    volatile uint32_t* arrivals = p.barrier;
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.barrier) : "memory");
     const long long t0 = clock64();
-    for (uint32_t it = 1; *arrivals < target; ++it) {
+    for (uint32_t it = 1;; ++it) {
+      uint32_t arrived;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(arrived) : "l"(p.barrier) : "memory");
+      if (arrived >= target) break;
       if ((it & 0xFF) == 0 && clock64() - t0 > p.wait_limit) {
         atomicCAS(p.status, 0, kDevGridBarrier);
         ok = 0;
         break;
       }
     }
-    __threadfence();
     sh->flag = ok;
   }
   __syncthreads();
@@ -299,54 +302,60 @@ __device__ __forceinline__ void bin_search(const SelectParams& p, int n_comb, in
   __syncthreads();
 }
 
-// Phase E: ranks the candidates [32 * kb_begin, 32 * kb_end) of `combo` among all of its n
-// candidates by counting the keys above each (keys are distinct).  One warp per candidate,
-// its lanes split the comparison range; the candidates are staged in shared memory, at most
-// kRankChunk at a time (one staging serves all items when n fits).
+// Phase E: ranks the candidates [lo, hi) of `combo` among all of its n candidates by counting
+// the keys above each (keys are distinct).  The combination's keys are staged in shared memory
+// (at most kRankChunk at a time).  A thread owns one candidate and one slice of the keys: the
+// threads of a warp share the slice, so every key is one broadcast read for 32 comparisons;
+// the slices' counts meet in shared-memory counters.
 static constexpr int kRankChunk = 8192;
 
-__device__ __forceinline__ void rank_range(const SelectParams& p, int combo, int n, int kb_begin,
-                                           int kb_end, unsigned long long* chunk) {
+__device__ __forceinline__ void rank_range(const SelectParams& p, int combo, int n, int lo, int hi,
+                                           unsigned long long* chunk, int* count_s) {
   const unsigned long long* cand = p.cand + static_cast<long long>(combo) * p.cand_stride;
   int* ranked = p.ranked + static_cast<long long>(combo) * p.cand_stride;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const bool whole = n <= kRankChunk;
-  for (int kb = kb_begin; kb < kb_end; ++kb) {
-    const int mine = kb * kRankKeysPerItem + warp;
-    const unsigned long long key = (mine < n) ? __ldcg(&cand[mine]) : 0ull;
+  for (int c0 = lo; c0 < hi; c0 += kSelThreads) {
+    const int nc = min(kSelThreads, hi - c0);               // candidates of this round
+    const int cpad = (nc + 31) & ~31;
+    const int n_slices = kSelThreads / cpad;                // >= 1; whole warps per slice
+    const int local = threadIdx.x % cpad, slice = threadIdx.x / cpad;
+    const bool active = slice < n_slices && local < nc;
+    const unsigned long long key = active ? __ldcg(&cand[c0 + local]) : ~0ull;
+    __syncthreads();                                        // previous users of count_s / chunk
+    if (threadIdx.x < cpad) count_s[threadIdx.x] = 0;
     int above = 0;
     for (int base = 0; base < n; base += kRankChunk) {
       const int cnt = min(kRankChunk, n - base);
-      const int padded = (cnt + 63) & ~63;
-      if (!whole || kb == kb_begin) {
-        __syncthreads();
-        constexpr int kLd = kRankChunk / kSelThreads;       // all loads in flight together
-        unsigned long long v[kLd];
+      if (base > 0) __syncthreads();
+      constexpr int kLd = kRankChunk / kSelThreads;         // all loads in flight together
+      unsigned long long v[kLd];
 #pragma unroll
-        for (int k = 0; k < kLd; ++k) {
-          const int i = k * kSelThreads + threadIdx.x;
-          v[k] = (i < cnt) ? __ldcg(&cand[base + i]) : 0ull;
-        }
-#pragma unroll
-        for (int k = 0; k < kLd; ++k) {
-          const int i = k * kSelThreads + threadIdx.x;
-          if (i < padded) chunk[i] = v[k];
-        }
-        __syncthreads();
+      for (int k = 0; k < kLd; ++k) {
+        const int i = k * kSelThreads + threadIdx.x;
+        v[k] = (i < cnt) ? __ldcg(&cand[base + i]) : 0ull;
       }
-      const ulonglong2* pairs = reinterpret_cast<const ulonglong2*>(chunk);
-      const int rounds = padded >> 6;                       // 32 lanes x 2 keys per round
-#pragma unroll 4
-      for (int j = 0; j < rounds; ++j) {
-        const ulonglong2 two = pairs[32 * j + lane];
-        above += (two.x > key) ? 1 : 0;
-        above += (two.y > key) ? 1 : 0;
+#pragma unroll
+      for (int k = 0; k < kLd; ++k) {
+        const int i = k * kSelThreads + threadIdx.x;
+        if (i < cnt) chunk[i] = v[k];
+      }
+      __syncthreads();
+      const int per = (cnt + n_slices - 1) / n_slices;
+      const int j0 = min(cnt, slice * per), j1 = min(cnt, j0 + per);
+      if (slice < n_slices) {                               // warp-uniform
+        int j = j0;
+        for (; j + 4 <= j1; j += 4) {
+          above += (chunk[j] > key) ? 1 : 0;
+          above += (chunk[j + 1] > key) ? 1 : 0;
+          above += (chunk[j + 2] > key) ? 1 : 0;
+          above += (chunk[j + 3] > key) ? 1 : 0;
+        }
+        for (; j < j1; ++j) above += (chunk[j] > key) ? 1 : 0;
       }
     }
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) above += __shfl_xor_sync(0xFFFFFFFFu, above, o);
-    if (lane == 0 && mine < n)
-      ranked[above] = static_cast<int>(0xFFFFFFFFu - static_cast<uint32_t>(key & 0xFFFFFFFFull));
+    if (active && above) atomicAdd(&count_s[local], above);
+    __syncthreads();
+    if (threadIdx.x < nc)                                   // slice 0 holds candidate c0 + threadIdx.x
+      ranked[count_s[threadIdx.x]] = static_cast<int>(0xFFFFFFFFu - static_cast<uint32_t>(key & 0xFFFFFFFFull));
   }
 }
 
@@ -969,23 +978,22 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
   // ---- E: ranking ----
   {
     unsigned long long* chunk = reinterpret_cast<unsigned long long*>(dyn_smem);
+    __shared__ int rank_count[kSelThreads];
     for (int combo = threadIdx.x; combo < tbl.n_comb; combo += kSelThreads)
       sh.state[combo] = min(min(__ldcg(&p.cand_count[combo]), static_cast<uint32_t>(kMaxKm)),
                             static_cast<uint32_t>(tbl.k_m[combo]));
     __syncthreads();
-    int n_items = 0;
-    for (int combo = 0; combo < tbl.n_comb; ++combo)
-      n_items += (static_cast<int>(sh.state[combo]) + kRankKeysPerItem - 1) / kRankKeysPerItem;
-    // every CTA takes a contiguous run of items, so that it stages few combinations
-    const int i_begin = static_cast<int>(static_cast<long long>(blockIdx.x) * n_items / gridDim.x);
-    const int i_end = static_cast<int>(static_cast<long long>(blockIdx.x + 1) * n_items / gridDim.x);
-    int item0 = 0;
+    long long n_cand = 0;
+    for (int combo = 0; combo < tbl.n_comb; ++combo) n_cand += sh.state[combo];
+    // every CTA takes a contiguous run of all candidates, so that it stages few combinations
+    const int i_begin = static_cast<int>(static_cast<long long>(blockIdx.x) * n_cand / gridDim.x);
+    const int i_end = static_cast<int>(static_cast<long long>(blockIdx.x + 1) * n_cand / gridDim.x);
+    int first = 0;
     for (int combo = 0; combo < tbl.n_comb; ++combo) {
       const int n = static_cast<int>(sh.state[combo]);
-      const int items = (n + kRankKeysPerItem - 1) / kRankKeysPerItem;
-      const int lo = max(i_begin, item0) - item0, hi = min(i_end, item0 + items) - item0;
-      if (lo < hi) rank_range(p, combo, n, lo, hi, chunk);
-      item0 += items;
+      const int lo = max(i_begin, first) - first, hi = min(i_end, first + n) - first;
+      if (lo < hi) rank_range(p, combo, n, lo, hi, chunk, rank_count);
+      first += n;
     }
   }
   if (!grid_sync(p, &sh, epoch)) return;
