@@ -64,9 +64,24 @@ chunk_attention_kernel(const __grid_constant__ CUtensorMap map_q,
   volatile int* abort_flag = &tail->abort_flag;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  const int j0 = (gridDim.x - 1 - blockIdx.x) * 128;    // first query token; heavy tiles first
-  const int n_streams = p.pair ? 2 : 1;
-  const int h0 = p.pair ? 2 * blockIdx.y : blockIdx.y;  // head of stream 0; stream 1 = h0 + 1
+  // Work items in launch order, heaviest first (later query tiles see more keys): the query
+  // tiles from split_from on with one CTA per head, then the others with one CTA per head pair.
+  int qt, h0, n_streams;
+  {
+    const int n_single = p.pair ? (p.n_qt - p.split_from) * p.n_q : p.n_qt * p.n_q;
+    const int b = blockIdx.x;
+    if (b < n_single) {
+      qt = p.n_qt - 1 - b / p.n_q;
+      h0 = b % p.n_q;
+      n_streams = 1;
+    } else {
+      const int n_pairs = p.n_q / 2, r = b - n_single;
+      qt = p.split_from - 1 - r / n_pairs;
+      h0 = 2 * (r % n_pairs);                            // head of stream 0; stream 1 = h0 + 1
+      n_streams = 2;
+    }
+  }
+  const int j0 = qt * 128;                               // first query token
   const int g = h0 / (p.n_q / p.n_kv);
   const int last_q = min(j0 + 128, p.c) - 1;
   const int n_tiles = (p.n_prefix + last_q) / 128 + 1;   // key tiles that hold a visible key
@@ -376,14 +391,24 @@ size_t attn_smem_bytes() {
 }
 
 cudaError_t launch_chunk_attention(const CUtensorMap& map_q, const CUtensorMap& map_k,
-                                   const CUtensorMap& map_v, const AttnParams& p, cudaStream_t st) {
+                                   const CUtensorMap& map_v, AttnParams p, int n_sm, cudaStream_t st) {
   const size_t smem = attn_smem_bytes();
   cudaError_t e = cudaFuncSetAttribute(chunk_attention_kernel,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(smem));
   if (e != cudaSuccess) return e;
-  dim3 grid((p.c + 127) / 128, p.pair ? p.n_q / 2 : p.n_q);
-  chunk_attention_kernel<<<grid, kAttnThreads, smem, st>>>(map_q, map_k, map_v, p);
+  p.n_qt = (p.c + 127) / 128;
+  p.split_from = p.n_qt;
+  long long n_cta = static_cast<long long>(p.n_qt) * (p.pair ? p.n_q / 2 : p.n_q);
+  if (p.pair) {
+    // A short chunk leaves SMs idle while the wave lasts as long as its heaviest CTA: give the
+    // heaviest query tiles one CTA per head for as long as everything still fits one wave.
+    while (p.split_from > 0 && n_cta + p.n_q / 2 <= n_sm) {
+      --p.split_from;
+      n_cta += p.n_q / 2;
+    }
+  }
+  chunk_attention_kernel<<<static_cast<unsigned>(n_cta), kAttnThreads, smem, st>>>(map_q, map_k, map_v, p);
   return cudaGetLastError();
 }
 

@@ -15,14 +15,17 @@ struct AttnParams {
   int n_prefix;      // rows of K/V visible to every query (sink + sliding window)
   int n_q, n_kv;     // query heads, kv heads
   int pair;          // 1: a CTA serves two query heads of one kv head; 0: one head
+  int n_qt;          // query tiles of 128 tokens
+  int split_from;    // query tiles >= split_from get one CTA per head (pair mode only; n_qt = none)
   float c2;          // log2(e) / sqrt(d)
   uint16_t* out;     // bf16 [c][n_q][128]
   int* status;
 };
 
 size_t attn_smem_bytes();
-// grid = (ceil(c / 128), n_q / 2 or n_q)
+// One CTA per (query tile, head pair) -- or per head, for the query tiles from split_from on;
+// fills p.n_qt and p.split_from (n_sm: SMs of the device).
 cudaError_t launch_chunk_attention(const CUtensorMap& map_q, const CUtensorMap& map_k,
-                                   const CUtensorMap& map_v, const AttnParams& p, cudaStream_t st);
+                                   const CUtensorMap& map_v, AttnParams p, int n_sm, cudaStream_t st);
 
 }  // namespace ilre

@@ -604,7 +604,7 @@ int ilre_recall_chunk_attention(ilre_recall_t* h, const void* q_dev, const void*
   ap.pair = ((h->cfg.n_q_heads / h->cfg.n_kv_heads) % 2 == 0) ? 1 : 0;   // two heads of one kv head per CTA
   ap.c2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(kHeadDim)));
   ap.out = static_cast<uint16_t*>(out_dev); ap.status = h->status;
-  ILRE_CUDA(launch_chunk_attention(map_q, map_k, map_v, ap, st));
+  ILRE_CUDA(launch_chunk_attention(map_q, map_k, map_v, ap, h->n_sm, st));
   h->last_launches = 1;
   return ILRE_OK;
 }

@@ -309,14 +309,18 @@ class IlreRecall:
         return out_idx, out_scores
 
     def chunk_attention(self, Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, n_prefix: int,
+                        out: Optional[torch.Tensor] = None,
                         stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
-        """Attention of one prefill chunk over n_prefix cached rows plus, causally, its own."""
+        """Attention of one prefill chunk over n_prefix cached rows plus, causally, its own.
+        Writes into ``out`` (bf16, Q's shape) when given."""
         for t in (Q, K, V):
             assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous() and t.dim() == 3
         c = Q.shape[0]
         assert Q.shape[1:] == (self.cfg.n_q_heads, self.cfg.head_dim)
         assert K.shape == (n_prefix + c, self.cfg.n_kv_heads, self.cfg.head_dim) and V.shape == K.shape
-        out = torch.empty_like(Q)
+        if out is None:
+            out = torch.empty_like(Q)
+        assert out.is_cuda and out.dtype == torch.bfloat16 and out.is_contiguous() and out.shape == Q.shape
         st = stream if stream is not None else torch.cuda.current_stream(self.device)
         rc = self._lib.ilre_recall_chunk_attention(self._h, Q.data_ptr(), K.data_ptr(), V.data_ptr(),
                                                    c, n_prefix, out.data_ptr(), st.cuda_stream)
