@@ -22,6 +22,8 @@ struct SmemTail {
   uint64_t acc_empty[4];
   uint32_t tmem_base;
   int abort_flag;
+  long long stamp_cycles;            // start of the optional clock stamp (kept out of registers)
+  unsigned long long stamp_ns;
 };
 static_assert(sizeof(SmemTail) <= kSmemTailBytes, "tail too large");
 
@@ -174,11 +176,11 @@ row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
   const uint32_t tmem_base = cta_setup(tail, smem_base, p.stages, 4, 4, p.status);
   const bool run = (it.n_tiles > 0) && (*abort_flag == 0);
   const bool stamp = (p.clk != nullptr) && blockIdx.x == 0 && threadIdx.x == 0;
-  long long cyc0 = 0;
-  unsigned long long ns0 = 0;
   if (stamp) {
-    cyc0 = clock64();
+    unsigned long long ns0;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns0));
+    tail->stamp_cycles = clock64();
+    tail->stamp_ns = ns0;
   }
 
   if (warp == 0) {
@@ -223,9 +225,13 @@ row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
     // the current one.
     const int wg = (warp - 2) >> 2;
     const int quad = warp & 3;               // TMEM lane quadrant this warp may read
-    float m[MT], z[MT];
+    // Accumulator u belongs to warpgroup u % 4 and holds row tile u % MT.  With 1, 2 or 4 row
+    // tiles a warpgroup therefore always meets the same row tile (wg % MT) and a thread keeps
+    // one (max, sum) pair; only with 3 row tiles does it meet all of them in turn.
+    constexpr int kStates = (MT == 3) ? 3 : 1;
+    float m[kStates], z[kStates];
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt) { m[mt] = -1e30f; z[mt] = 0.f; }
+    for (int j = 0; j < kStates; ++j) { m[j] = -1e30f; z[j] = 0.f; }
     const float c2 = p.c2;
     const uint32_t n_acc = run ? static_cast<uint32_t>(it.n_tiles) * MT : 0u;
     // One copy of the loop body serves every (key tile, row tile): the warpgroups run at
@@ -242,9 +248,11 @@ row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
         break;
       tc_fence_after();
       float mr = m[0], zr = z[0];
+      if (kStates > 1) {
 #pragma unroll
-      for (int j = 1; j < MT; ++j)
-        if (j == mt) { mr = m[j]; zr = z[j]; }
+        for (int j = 1; j < kStates; ++j)
+          if (j == mt) { mr = m[j]; zr = z[j]; }
+      }
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + b * 128;
       float va[32], vb[32];
       tmem_ld32(taddr, va);
@@ -264,21 +272,33 @@ row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
         row_chunk_update<NPOLY>(vb, 64 * h + 32, valid, c2, mr, zr);
         if (h == 0) tmem_ld_wait();
       }
+      if (kStates > 1) {
 #pragma unroll
-      for (int j = 0; j < MT; ++j)
-        if (j == mt) { m[j] = mr; z[j] = zr; }
+        for (int j = 0; j < kStates; ++j)
+          if (j == mt) { m[j] = mr; z[j] = zr; }
+      } else {
+        m[0] = mr; z[0] = zr;
+      }
     }
     // Merge the warpgroups' statistics through shared memory and write this CTA's partial
-    // statistics: (max in log2 units, sum).  The scratch aliases the first K stage, which is
-    // idle once every warpgroup has read its last accumulator (every MMA, hence every TMA
-    // load, has completed by then).
+    // statistics: (max in log2 units, sum).  Every warpgroup stores a pair for every row tile
+    // (a neutral one for the row tiles it never met); warpgroup 0 merges.  The scratch aliases
+    // the first K stage, which is idle once every warpgroup has read its last accumulator
+    // (every MMA, hence every TMA load, has completed by then).
     float2* scratch = reinterpret_cast<float2*>(smem + MT * 128 * 256);
     const int row_in_tile = quad * 32 + lane;
     asm volatile("bar.sync 1, %0;" ::"r"(kStatsConsumerWarps * 32) : "memory");
-    if (wg > 0) {
 #pragma unroll
-      for (int mt = 0; mt < MT; ++mt)
-        scratch[((wg - 1) * MT + mt) * 128 + row_in_tile] = make_float2(m[mt], z[mt]);
+    for (int mt = 0; mt < MT; ++mt) {
+      float2 mine = make_float2(-1e30f, 0.f);
+      if (kStates > 1) {
+#pragma unroll
+        for (int j = 0; j < kStates; ++j)
+          if (j == mt) mine = make_float2(m[j], z[j]);
+      } else if (mt == wg % MT) {
+        mine = make_float2(m[0], z[0]);
+      }
+      scratch[(wg * MT + mt) * 128 + row_in_tile] = mine;
     }
     asm volatile("bar.sync 1, %0;" ::"r"(kStatsConsumerWarps * 32) : "memory");
     if (wg == 0) {
@@ -286,14 +306,14 @@ row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
                     (static_cast<size_t>(it.group) * p.cpg + it.chunk) * (MT * 128);
 #pragma unroll
       for (int mt = 0; mt < MT; ++mt) {
-        float mm = m[mt];
+        float mm = -1e30f;
 #pragma unroll
-        for (int w = 1; w < kStatsWarpgroups; ++w)
-          mm = fmaxf(mm, scratch[((w - 1) * MT + mt) * 128 + row_in_tile].x);
-        float zz = z[mt] * exp2f((m[mt] - mm) * c2);
+        for (int w = 0; w < kStatsWarpgroups; ++w)
+          mm = fmaxf(mm, scratch[(w * MT + mt) * 128 + row_in_tile].x);
+        float zz = 0.f;
 #pragma unroll
-        for (int w = 1; w < kStatsWarpgroups; ++w) {
-          const float2 o = scratch[((w - 1) * MT + mt) * 128 + row_in_tile];
+        for (int w = 0; w < kStatsWarpgroups; ++w) {
+          const float2 o = scratch[(w * MT + mt) * 128 + row_in_tile];
           zz += o.y * exp2f((o.x - mm) * c2);
         }
         out[mt * 128 + row_in_tile] = make_float2(mm * c2, zz);
@@ -303,8 +323,8 @@ row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
   if (stamp) {
     unsigned long long ns1;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns1));
-    p.clk[0] = static_cast<unsigned long long>(clock64() - cyc0);
-    p.clk[1] = ns1 - ns0;
+    p.clk[0] = static_cast<unsigned long long>(clock64() - tail->stamp_cycles);
+    p.clk[1] = ns1 - tail->stamp_ns;
   }
   cta_teardown(tmem_base);
 }
