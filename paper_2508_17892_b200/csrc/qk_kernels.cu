@@ -153,8 +153,11 @@ __device__ __forceinline__ void row_chunk_update(float (&v)[32], int col0, int v
   const float m_new = fmaxf(fmax3(m, cm0, cm1), fmaxf(v[30], v[31]));
   const float nm = -m_new * c2;
   const float sum = chunk_sum_exp2<NPOLY>(v, c2, nm);
-  z = fmaf(z, ex2_approx((m - m_new) * c2), sum);
-  m = m_new;
+  if (m_new > m) {                         // rare once the first tiles have been seen
+    z *= ex2_approx((m - m_new) * c2);
+    m = m_new;
+  }
+  z += sum;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -257,7 +260,7 @@ row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
       float va[32], vb[32];
       tmem_ld32(taddr, va);
       tmem_ld_wait();
-#pragma unroll 1
+#pragma unroll
       for (int h = 0; h < 2; ++h) {
         tmem_ld32(taddr + 64 * h + 32, vb);
         row_chunk_update<NPOLY>(va, 64 * h, valid, c2, mr, zr);
