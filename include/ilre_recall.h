@@ -80,7 +80,8 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out);
  *   k_cache_dev   bf16 [L][n_kv_heads][128], RoPE already applied, 16-byte aligned; read only
  *   query_dev     bf16 [q_len][n_q_heads][128], 16-byte aligned; read only
  *   budget        B, 0 <= B <= L - n_sink
- *   out_idx_dev   int32 [n_sink + budget]: chosen context positions, ascending
+ *   out_idx_dev   int32 [n_sink + budget]: chosen context positions, ascending (may be NULL when
+ *                 n_sink + budget = 0: the result is empty)
  *   out_scores_dev  optional fp32 [L]: A^C of Eq. 5 (NULL to skip)
  * The call only encodes two tensor maps on the host and launches kernels on cuda_stream (no
  * allocation, no synchronisation), so it may be captured into a CUDA graph and replayed.

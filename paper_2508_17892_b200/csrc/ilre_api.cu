@@ -172,8 +172,9 @@ int validate_run(const ilre_recall* h, const void* k, long long L, const void* q
                  bool with_select) {
   if (!h || !spec) return ILRE_ERR_INVALID_ARG;
   if (with_qk && (!k || !q)) return ILRE_ERR_INVALID_ARG;
-  if (with_select && !out_idx) return ILRE_ERR_INVALID_ARG;
   if (L < 1 || q_len < 1 || budget < 0) return ILRE_ERR_INVALID_ARG;
+  // an empty result (no budget, no sink part) needs no output buffer
+  if (with_select && !out_idx && (budget > 0 || spec->n_sink > 0)) return ILRE_ERR_INVALID_ARG;
   if (spec->n_max < 1 || spec->n_win < 1 || !spec->max_sizes || !spec->win_sizes)
     return ILRE_ERR_INVALID_ARG;
   if (spec->n_sink < 0 || spec->win_op < 0 || spec->win_op > 1) return ILRE_ERR_INVALID_ARG;

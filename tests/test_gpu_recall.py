@@ -93,6 +93,7 @@ RAGGED = [
     (20000, 40, 1, 8, 999, (4,), (1, 2), 0, 3),
     (300, 5, 8, 32, 296, (8,), (1, 4), 0, 4),            # budget = L - n_sink with a partial cell
     (300, 5, 8, 32, 0, (2,), (3,), 0, 4),                # empty budget: sinks only
+    (50, 3, 8, 32, 0, (2,), (3,), 0, 0),                 # empty budget, no sinks: an empty list
 ]
 
 
