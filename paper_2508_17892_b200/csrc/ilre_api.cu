@@ -441,6 +441,8 @@ int recall_impl(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const void
   for (int c = 0; c < tbl.n_comb; ++c) n_cand += tbl.k_m[c];
   if (n_cand / 96 > want_grid) want_grid = n_cand / 96;
   if (want_grid < 1) want_grid = 1;
+  // a grid just above the cluster size: the cluster barrier is worth more than the extra CTAs
+  if (want_grid > kSelClusterMax && want_grid <= 2 * kSelClusterMax) want_grid = kSelClusterMax;
   if (want_grid > h->select_max_grid) want_grid = h->select_max_grid;
   const int select_grid = static_cast<int>(want_grid);
 

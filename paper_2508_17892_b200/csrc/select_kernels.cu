@@ -56,7 +56,14 @@ struct SelShared {
 // CTA's writes, which the block barrier before it orders) and polls with acquire loads; no
 // value comes back from the arrival, so a barrier costs one trip to the L2 instead of two.
 // The wait is bounded; a CTA that gives up records it and leaves the kernel.
+// kCluster: the whole grid is one thread-block cluster (short contexts): the hardware cluster
+// barrier takes the place of the counter, with release / acquire ordering at cluster scope.
+template <bool kCluster>
 __device__ __forceinline__ bool grid_sync(const SelectParams& p, SelShared* sh, uint32_t& epoch) {
+  if constexpr (kCluster) {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    return true;
+  }
   ++epoch;
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -686,6 +693,7 @@ __device__ __forceinline__ void allocate(const ComboTable& tbl, const SelectPara
   if (threadIdx.x == 0 && total != cap) atomicCAS(p.status, 0, kDevQuota);
 }
 
+template <bool kCluster>
 __global__ void __launch_bounds__(kSelThreads, 1)
 select_kernel(const ComboTable tbl, const SelectParams p) {
   extern __shared__ __align__(16) uint8_t dyn_smem[];
@@ -706,7 +714,7 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
       if (p.user_scores) p.user_scores[t] = a;
     }
   }
-  if (!grid_sync(p, &sh, epoch)) return;
+  if (!grid_sync<kCluster>(p, &sh, epoch)) return;
 
   // ---- B1: strided max-pool arrays, one per distinct m > 1 ----
   if (tbl.n_src > 0) {
@@ -719,7 +727,7 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
       while (src + 1 < tbl.n_src && tile >= tbl.src_tile_begin[src + 1]) ++src;
       maxpool_tile(tbl, p, src, tile - tbl.src_tile_begin[src], buf);
     }
-    if (!grid_sync(p, &sh, epoch)) return;
+    if (!grid_sync<kCluster>(p, &sh, epoch)) return;
   }
 
   // ---- B2: window pooling of every combination + first histogram ----
@@ -736,7 +744,7 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
     }
     if (cur >= 0) hist_flush(sh.hist, p.hist + static_cast<long long>(cur) * kHistBins);
   }
-  if (!grid_sync(p, &sh, epoch)) return;
+  if (!grid_sync<kCluster>(p, &sh, epoch)) return;
 
   // ---- C: radix select of the K_m-th largest value ----
   // combinations whose tiles this CTA scans
@@ -817,7 +825,7 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
       }
     }
   }
-  if (!grid_sync(p, &sh, epoch)) return;
+  if (!grid_sync<kCluster>(p, &sh, epoch)) return;
 
   // The cells set aside: one CTA per combination selects the highest `wanted` keys among them
   // (radix select over the remaining 53 bits of the key in shared memory) and appends them.
@@ -871,7 +879,7 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
         }
       }
       if (cur >= 0) hist_flush(sh.hist, hist_pass + static_cast<long long>(cur) * kHistBins);
-      if (!grid_sync(p, &sh, epoch)) return;
+      if (!grid_sync<kCluster>(p, &sh, epoch)) return;
       for (int combo = c_lo; combo <= c_hi; ++combo)
         if (sh.state[combo] == 0u) bin_search(p, tbl.n_comb, combo, pass, &sh);
     }
@@ -907,7 +915,7 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
         }
       }
     }
-    if (!grid_sync(p, &sh, epoch)) return;
+    if (!grid_sync<kCluster>(p, &sh, epoch)) return;
     {
       const int lane = threadIdx.x & 31;
       int load_cursor = 0, cursor = 0;
@@ -973,7 +981,7 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
       }
     }
   }
-  if (!grid_sync(p, &sh, epoch)) return;
+  if (!grid_sync<kCluster>(p, &sh, epoch)) return;
 
   // ---- E: ranking ----
   {
@@ -996,7 +1004,7 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
       first += n;
     }
   }
-  if (!grid_sync(p, &sh, epoch)) return;
+  if (!grid_sync<kCluster>(p, &sh, epoch)) return;
 
   // ---- F: allocation and ascending output (one CTA) ----
   if (blockIdx.x != 0) return;
@@ -1038,11 +1046,14 @@ size_t select_smem_bytes(long long L, int max_km, SelectParams* p) {
 }
 
 cudaError_t select_max_grid(int n_sm, int* max_grid) {
-  cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(select_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        kSelMaxDynSmemBytes);
   if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kSelMaxDynSmemBytes);
+  if (e != cudaSuccess) return e;
   int per_sm = 0;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, select_kernel, kSelThreads,
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, select_kernel<false>, kSelThreads,
                                                     kSelMaxDynSmemBytes);
   if (e != cudaSuccess) return e;
   if (per_sm < 1) return cudaErrorLaunchOutOfResources;
@@ -1052,8 +1063,26 @@ cudaError_t select_max_grid(int n_sm, int* max_grid) {
 
 cudaError_t launch_select(const ComboTable& tbl, const SelectParams& p, int grid, size_t smem,
                           cudaStream_t st) {
+  // Short contexts need few CTAs: up to kSelClusterMax of them run as one thread-block cluster,
+  // whose hardware barrier costs a fraction of a trip to the L2 (not with the self test's
+  // barrier that cannot complete: that one is the counter's).
+  if (grid <= kSelClusterMax && p.barrier_extra == 0) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kSelThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = grid;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, select_kernel<true>, tbl, p);
+  }
   void* args[2] = {const_cast<ComboTable*>(&tbl), const_cast<SelectParams*>(&p)};
-  return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(select_kernel), dim3(grid),
+  return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(select_kernel<false>), dim3(grid),
                                      dim3(kSelThreads), args, smem, st);
 }
 

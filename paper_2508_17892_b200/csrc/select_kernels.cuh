@@ -15,6 +15,7 @@ static constexpr int kSelectPasses = 3;     // 32 value bits of the key in 11/11
 static constexpr int kSelThreads = 1024;    // threads per CTA of the selection kernel
 static constexpr int kSelTile = 4096;       // cells of one combination per work tile
 static constexpr int kSrcTileTokens = 8192; // tokens per work tile of the strided max-pool
+static constexpr int kSelClusterMax = 8;     // grids up to this size run as one thread-block cluster
 static constexpr int kPendCap = 8192;        // cells of the threshold bin resolved by one CTA (else: more passes)
 static constexpr int kSelBitmapSmemBytes = 136 * 1024;   // bitmap kept in shared memory up to this
 static constexpr int kSelMaxDynSmemBytes = kSelBitmapSmemBytes + kMaxKm * 4;
