@@ -40,10 +40,10 @@ import numpy as np
 import torch
 
 # DRAM bytes per context position of the dominant kernel (row statistics), from one ncu
-# capture at L = 131072, q_len = 256: (270.60 MB read + 5.19 MB written, mean of two launches)
+# capture at L = 131072, q_len = 256: (270.60 MB read + 3.96 MB written, mean of two launches)
 # / 131072 keys.  Traffic grows in proportion to L (the query block is L2-resident), so it is
 # scaled by L.
-ROW_STATS_DRAM_BYTES_PER_KEY = 2104.0
+ROW_STATS_DRAM_BYTES_PER_KEY = 2095.0
 METRIC = "key_cache_GBps_per_recall_L1M"
 UNIT = "GB/s"
 CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
