@@ -310,16 +310,133 @@ __device__ __forceinline__ void bin_search(const SelectParams& p, int n_comb, in
 }
 
 // Phase E: ranks the candidates [lo, hi) of `combo` among all of its n candidates by counting
-// the keys above each (keys are distinct).  The combination's keys are staged in shared memory
-// (at most kRankChunk at a time).  A thread owns one candidate and one slice of the keys: the
-// threads of a warp share the slice, so every key is one broadcast read for 32 comparisons;
-// the slices' counts meet in shared-memory counters.
+// the keys above each (keys are distinct).
+//
+// Lists of kRankBucketMin..kRankChunk keys are first split into kRankBuckets value ranges, so
+// that a candidate is compared with its own range only: kRankSamples keys taken at even
+// strides are ranked among themselves, every fourth of them becomes a splitter, every key of
+// the list goes to the bucket "number of splitters above it" (bucket 0 holds the largest
+// keys) and is stored bucket by bucket in shared memory.  rank = keys in the buckets before
+// + keys above inside the bucket.  The result does not depend on which keys were sampled,
+// only the work per candidate does; every CTA samples for itself.
+//
+// Other lists take the plain form: the keys are staged in shared memory (at most kRankChunk
+// at a time), a thread owns one candidate and one slice of the keys, the threads of a warp
+// share the slice, so every key is one broadcast read for 32 comparisons; the slices' counts
+// meet in shared-memory counters.
 static constexpr int kRankChunk = 8192;
+static constexpr int kRankSamples = 128;
+static constexpr int kRankBuckets = 32;
+static constexpr int kRankBucketMin = 1024;
+
+struct RankScratch {
+  unsigned long long samp[kRankSamples];
+  unsigned long long spl[kRankBuckets];    // splitters, descending; the last entry is unused
+  uint32_t srank[kRankSamples];
+  uint32_t count[kRankBuckets];
+  uint32_t start[kRankBuckets + 1];
+};
+
+// Number of splitters above `key`.
+__device__ __forceinline__ int rank_bucket(const unsigned long long* spl, unsigned long long key) {
+  int b = 0;
+#pragma unroll
+  for (int step = kRankBuckets / 2; step >= 1; step >>= 1)
+    if (spl[b + step - 1] > key) b += step;
+  return b;
+}
+
+__device__ __forceinline__ void rank_range_bucketed(const unsigned long long* cand, int* ranked, int n,
+                                                    int lo, int hi, unsigned long long* grouped,
+                                                    RankScratch* rs) {
+  constexpr int kLd = kRankChunk / kSelThreads;
+  const int tid = threadIdx.x;
+  unsigned long long v[kLd];
+#pragma unroll
+  for (int k = 0; k < kLd; ++k) {
+    const int i = k * kSelThreads + tid;
+    v[k] = (i < n) ? __ldcg(&cand[i]) : 0ull;
+  }
+  __syncthreads();                                          // previous users of rs / grouped
+  if (tid < kRankSamples) {
+    rs->samp[tid] = __ldcg(&cand[static_cast<int>((static_cast<long long>(tid) * n) / kRankSamples)]);
+    rs->srank[tid] = 0;
+  }
+  if (tid < kRankBuckets) rs->count[tid] = 0;
+  __syncthreads();
+  {                                                         // rank the samples among themselves
+    constexpr int kPer = kRankSamples / (kSelThreads / kRankSamples);
+    const int si = tid % kRankSamples, j0 = (tid / kRankSamples) * kPer;
+    const unsigned long long mine = rs->samp[si];
+    uint32_t above = 0;
+#pragma unroll
+    for (int j = 0; j < kPer; ++j) above += (rs->samp[j0 + j] > mine) ? 1u : 0u;
+    if (above) atomicAdd(&rs->srank[si], above);
+  }
+  __syncthreads();
+  if (tid < kRankSamples) {
+    const uint32_t r = rs->srank[tid];
+    if ((r & 3u) == 3u) rs->spl[r >> 2] = rs->samp[tid];
+  }
+  __syncthreads();
+  uint32_t where[kLd];                                      // bucket << 16 | slot inside the bucket
+#pragma unroll
+  for (int k = 0; k < kLd; ++k) {
+    const int i = k * kSelThreads + tid;
+    if (i < n) {
+      const int b = rank_bucket(rs->spl, v[k]);
+      where[k] = (static_cast<uint32_t>(b) << 16) | atomicAdd(&rs->count[b], 1u);
+    }
+  }
+  __syncthreads();
+  if (tid < 32) {
+    const uint32_t c = rs->count[tid];
+    uint32_t incl = c;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+      if (tid >= d) incl += o;
+    }
+    rs->start[tid] = incl - c;
+    if (tid == 31) rs->start[32] = incl;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int k = 0; k < kLd; ++k) {
+    const int i = k * kSelThreads + tid;
+    if (i < n) grouped[rs->start[where[k] >> 16] + (where[k] & 0xFFFFu)] = v[k];
+  }
+  __syncthreads();
+  for (int c0 = lo; c0 < hi; c0 += kSelThreads) {
+    const int nc = min(kSelThreads, hi - c0);
+    int g = 1;                                              // threads per candidate
+    while (g < 32 && 2 * g * nc <= kSelThreads) g <<= 1;
+    const int local = tid / g, sub = tid % g;
+    const bool active = local < nc;
+    const unsigned long long key = active ? __ldcg(&cand[c0 + local]) : ~0ull;
+    int j = 0, j1 = 0, first = 0;
+    if (active) {
+      const int b = rank_bucket(rs->spl, key);
+      first = static_cast<int>(rs->start[b]);
+      j = first + sub;
+      j1 = static_cast<int>(rs->start[b + 1]);
+    }
+    int above = 0;
+    for (; j < j1; j += g) above += (grouped[j] > key) ? 1 : 0;
+    for (int d = 1; d < g; d <<= 1) above += __shfl_xor_sync(0xFFFFFFFFu, above, d);
+    if (active && sub == 0)
+      ranked[first + above] = static_cast<int>(0xFFFFFFFFu - static_cast<uint32_t>(key & 0xFFFFFFFFull));
+  }
+}
 
 __device__ __forceinline__ void rank_range(const SelectParams& p, int combo, int n, int lo, int hi,
-                                           unsigned long long* chunk, int* count_s) {
+                                           unsigned long long* chunk, int* count_s, RankScratch* rs) {
   const unsigned long long* cand = p.cand + static_cast<long long>(combo) * p.cand_stride;
   int* ranked = p.ranked + static_cast<long long>(combo) * p.cand_stride;
+  if (n >= kRankBucketMin && n <= kRankChunk) {
+    rank_range_bucketed(cand, ranked, n, lo, hi, chunk, rs);
+    return;
+  }
   for (int c0 = lo; c0 < hi; c0 += kSelThreads) {
     const int nc = min(kSelThreads, hi - c0);               // candidates of this round
     const int cpad = (nc + 31) & ~31;
@@ -987,21 +1104,36 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
   {
     unsigned long long* chunk = reinterpret_cast<unsigned long long*>(dyn_smem);
     __shared__ int rank_count[kSelThreads];
+    __shared__ RankScratch rank_scratch;
     for (int combo = threadIdx.x; combo < tbl.n_comb; combo += kSelThreads)
       sh.state[combo] = min(min(__ldcg(&p.cand_count[combo]), static_cast<uint32_t>(kMaxKm)),
                             static_cast<uint32_t>(tbl.k_m[combo]));
     __syncthreads();
-    long long n_cand = 0;
-    for (int combo = 0; combo < tbl.n_comb; ++combo) n_cand += sh.state[combo];
-    // every CTA takes a contiguous run of all candidates, so that it stages few combinations
-    const int i_begin = static_cast<int>(static_cast<long long>(blockIdx.x) * n_cand / gridDim.x);
-    const int i_end = static_cast<int>(static_cast<long long>(blockIdx.x + 1) * n_cand / gridDim.x);
-    int first = 0;
-    for (int combo = 0; combo < tbl.n_comb; ++combo) {
-      const int n = static_cast<int>(sh.state[combo]);
-      const int lo = max(i_begin, first) - first, hi = min(i_end, first + n) - first;
-      if (lo < hi) rank_range(p, combo, n, lo, hi, chunk, rank_count);
-      first += n;
+    const int grid = static_cast<int>(gridDim.x), bid = static_cast<int>(blockIdx.x);
+    if (tbl.rank_by_list) {
+      // Enough CTAs: each serves one combination only (a CTA that met two would stage and
+      // split both lists, and the whole grid would wait for it).  The host has dealt the CTAs
+      // out: combination c has [rank_cta_begin[c], rank_cta_begin[c + 1]).
+      for (int combo = 0; combo < tbl.n_comb; ++combo) {
+        const int b0 = tbl.rank_cta_begin[combo], b1 = tbl.rank_cta_begin[combo + 1];
+        if (bid < b0 || bid >= b1) continue;
+        const uint32_t n = sh.state[combo], share = b1 - b0, k = bid - b0;
+        const int lo = static_cast<int>(n * k / share), hi = static_cast<int>(n * (k + 1) / share);
+        if (lo < hi) rank_range(p, combo, static_cast<int>(n), lo, hi, chunk, rank_count, &rank_scratch);
+      }
+    } else {
+      // fewer CTAs than lists: every CTA takes a contiguous run of all candidates
+      long long n_cand = 0;
+      for (int combo = 0; combo < tbl.n_comb; ++combo) n_cand += sh.state[combo];
+      const int i_begin = static_cast<int>(static_cast<long long>(bid) * n_cand / grid);
+      const int i_end = static_cast<int>(static_cast<long long>(bid + 1) * n_cand / grid);
+      int first = 0;
+      for (int combo = 0; combo < tbl.n_comb; ++combo) {
+        const int n = static_cast<int>(sh.state[combo]);
+        const int lo = max(i_begin, first) - first, hi = min(i_end, first + n) - first;
+        if (lo < hi) rank_range(p, combo, n, lo, hi, chunk, rank_count, &rank_scratch);
+        first += n;
+      }
     }
   }
   if (!grid_sync<kCluster>(p, &sh, epoch)) return;
@@ -1061,8 +1193,37 @@ cudaError_t select_max_grid(int n_sm, int* max_grid) {
   return cudaSuccess;
 }
 
-cudaError_t launch_select(const ComboTable& tbl, const SelectParams& p, int grid, size_t smem,
+// Deals the CTAs of the grid out to the combinations for the ranking phase: each list gets
+// its share of the grid by candidates, at least one CTA, never past what the lists after it
+// still need.  With fewer CTAs than lists the kernel splits the candidates evenly instead.
+static void assign_ranking(ComboTable* t, int grid) {
+  long long n_cand = 0;
+  int n_lists = 0;
+  for (int c = 0; c < t->n_comb; ++c) {
+    n_cand += t->k_m[c];
+    n_lists += t->k_m[c] > 0 ? 1 : 0;
+  }
+  t->rank_by_list = (n_lists > 0 && grid >= n_lists) ? 1 : 0;
+  long long before = 0;
+  int b0 = 0, lists_left = n_lists;
+  for (int c = 0; c < t->n_comb; ++c) {
+    t->rank_cta_begin[c] = b0;
+    if (!t->rank_by_list || t->k_m[c] <= 0) continue;
+    --lists_left;
+    before += t->k_m[c];
+    int b1 = static_cast<int>((before * grid + n_cand / 2) / n_cand);
+    if (b1 < b0 + 1) b1 = b0 + 1;
+    if (b1 > grid - lists_left) b1 = grid - lists_left;
+    if (lists_left == 0) b1 = grid;
+    b0 = b1;
+  }
+  t->rank_cta_begin[t->n_comb] = b0;
+}
+
+cudaError_t launch_select(const ComboTable& table, const SelectParams& p, int grid, size_t smem,
                           cudaStream_t st) {
+  ComboTable tbl = table;
+  assign_ranking(&tbl, grid);
   // Short contexts need few CTAs: up to kSelClusterMax of them run as one thread-block cluster,
   // whose hardware barrier costs a fraction of a trip to the L2 (not with the self test's
   // barrier that cannot complete: that one is the counter's).
@@ -1081,7 +1242,7 @@ cudaError_t launch_select(const ComboTable& tbl, const SelectParams& p, int grid
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, select_kernel<true>, tbl, p);
   }
-  void* args[2] = {const_cast<ComboTable*>(&tbl), const_cast<SelectParams*>(&p)};
+  void* args[2] = {&tbl, const_cast<SelectParams*>(&p)};
   return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(select_kernel<false>), dim3(grid),
                                      dim3(kSelThreads), args, smem, st);
 }

@@ -36,6 +36,10 @@ struct ComboTable {
   int src_m[kMaxCombos];
   int src_len[kMaxCombos];
   int src_tile_begin[kMaxCombos + 1];   // tiles of kSrcTileTokens / m cells each
+  // Ranking phase (filled in by launch_select): with rank_by_list, combination c is ranked by
+  // the CTAs [rank_cta_begin[c], rank_cta_begin[c + 1]).
+  int rank_by_list;
+  int rank_cta_begin[kMaxCombos + 1];
 };
 
 struct SelectParams {
