@@ -271,7 +271,7 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out) {
   ok = ok && dev_alloc(&h->cand_count, 4 * static_cast<size_t>(kMaxCombos));
   ok = ok && dev_alloc(&h->pending, ncomb * kPendCap);
   ok = ok && dev_alloc(&h->ranked, ncomb * h->cand_stride);
-  ok = ok && dev_alloc(&h->bitmap, (maxL + 31) / 32);
+  ok = ok && dev_alloc(&h->bitmap, (maxL + 31) / 32 + 4);    // read four words at a time
   ok = ok && dev_alloc(&h->status, 1);
   ok = ok && dev_alloc(&h->clk, 2);
   if (ok && cfg->host_staging) {
@@ -433,7 +433,7 @@ int recall_impl(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const void
   sp.barrier_extra = (h->inject == ILRE_SELFTEST_GRID_BARRIER) ? 1 : 0;
   int max_km = 1;
   for (int c = 0; c < tbl.n_comb; ++c) max_km = tbl.k_m[c] > max_km ? tbl.k_m[c] : max_km;
-  const size_t select_smem = select_smem_bytes(L, max_km, &sp);
+  const size_t select_smem = select_smem_bytes(L, max_km, budget, &sp);
   // Grid of the selection kernel: enough CTAs for the scan tiles and for the ranking (about a
   // hundred candidates per CTA), but no more, since every grid barrier pays for them.
   long long want_grid = tbl.tile_begin[tbl.n_comb];

@@ -771,43 +771,110 @@ __device__ __forceinline__ void allocate(const ComboTable& tbl, const SelectPara
   }
   __syncthreads();
 
-  // Ascending output.  Every warp owns a contiguous run of bitmap words and reads it 32
-  // consecutive words at a time (one per lane).
+  // Ascending output.  One SM does this, so what counts is the number of instructions it has
+  // to issue.  Up to kSelThreads bitmap words (32K positions) a thread takes one word.  Longer
+  // contexts: the sink part is the identity; for the rest the bitmap is read four words per
+  // lane and load (a warp owns a contiguous run of words), twice: to count the words that hold
+  // an allocated position outside the sink part, then to list them in ascending order in
+  // shared memory (where the staged cells were; they are done with).  There are at most
+  // `budget` such words, usually a few hundred: the threads share them out evenly, take the
+  // prefix of their position counts and write the positions.
   const long long n_words = (p.L + 31) / 32;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const long long rounds = (n_words + kSelThreads - 1) / kSelThreads;       // per warp
-  const long long w_begin = static_cast<long long>(warp) * rounds * 32;
-  uint32_t count = 0;
-  for (long long k = 0; k < rounds; ++k) {
-    const long long w = w_begin + k * 32 + lane;
-    if (w < n_words) count += __popc(bitmap_word<kBitmapInSmem>(bm, static_cast<int>(w)));
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) count += __shfl_xor_sync(0xFFFFFFFFu, count, o);
-  uint32_t total;
-  uint32_t off = block_exclusive_scan(lane == 0 ? count : 0u, sh->scan, &total);
-  off = __shfl_sync(0xFFFFFFFFu, off, 0);                   // first output slot of this warp
   const uint32_t cap = static_cast<uint32_t>(p.n_sink + p.budget);
-  for (long long k = 0; k < rounds; ++k) {
-    const long long w = w_begin + k * 32 + lane;
-    uint32_t bits = (w < n_words) ? bitmap_word<kBitmapInSmem>(bm, static_cast<int>(w)) : 0u;
-    if (__ballot_sync(0xFFFFFFFFu, bits != 0u) == 0u) continue;      // nothing allocated in these 1024 positions
-    uint32_t incl = __popc(bits);
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-      if (lane >= o) incl += t;
-    }
-    uint32_t at = off + incl - __popc(bits);
+  if (n_words <= kSelThreads) {
+    // short context: a thread per bitmap word (sink bits included), one prefix sum
+    uint32_t bits = (static_cast<long long>(threadIdx.x) < n_words)
+                        ? bitmap_word<kBitmapInSmem>(bm, static_cast<int>(threadIdx.x)) : 0u;
+    uint32_t total;
+    uint32_t at = block_exclusive_scan(__popc(bits), sh->scan, &total);
     while (bits) {
       const int b = __ffs(bits) - 1;
       bits &= bits - 1;
-      if (at < cap) p.out_idx[at] = static_cast<int>(w * 32 + b);
+      if (at < cap) p.out_idx[at] = static_cast<int>(threadIdx.x) * 32 + b;
       ++at;
     }
-    off += __shfl_sync(0xFFFFFFFFu, incl, 31);
+    if (threadIdx.x == 0 && total != cap) atomicCAS(p.status, 0, kDevQuota);
+    return;
   }
-  if (threadIdx.x == 0 && total != cap) atomicCAS(p.status, 0, kDevQuota);
+  const int n_quads = static_cast<int>((n_words + 3) / 4);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rounds = (n_quads + kSelThreads - 1) / kSelThreads;      // per warp
+  const int q_begin = warp * rounds * 32;
+  int* list = staged;
+  // bits of word w that stand for allocated positions outside the sink part
+  auto outside_sink = [&](uint32_t bits, long long w) -> uint32_t {
+    const long long lo = w * 32;
+    if (lo >= p.n_sink) return bits;
+    return (p.n_sink - lo >= 32) ? 0u : (bits & ~((1u << (p.n_sink - lo)) - 1u));
+  };
+  auto load_quad = [&](int q) -> uint4 {
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (q >= n_quads) return v;
+    if constexpr (kBitmapInSmem) {
+      asm volatile("ld.volatile.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                   : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(smem_u32(bm + 4 * q)) : "memory");
+    } else {
+      v = __ldcg(reinterpret_cast<const uint4*>(bm) + q);
+    }
+    const long long w0 = 4ll * q;
+    if (w0 + 4 > n_words) {                                  // words past the end hold nothing
+      if (w0 + 1 >= n_words) v.y = 0u;
+      if (w0 + 2 >= n_words) v.z = 0u;
+      if (w0 + 3 >= n_words) v.w = 0u;
+    }
+    if (w0 * 32 < p.n_sink) {
+      v.x = outside_sink(v.x, w0); v.y = outside_sink(v.y, w0 + 1);
+      v.z = outside_sink(v.z, w0 + 2); v.w = outside_sink(v.w, w0 + 3);
+    }
+    return v;
+  };
+  for (int j = threadIdx.x; j < p.n_sink; j += kSelThreads) p.out_idx[j] = j;
+  uint32_t n_mine = 0;
+  for (int k = 0; k < rounds; ++k) {
+    const uint4 v = load_quad(q_begin + k * 32 + lane);
+    n_mine += (v.x != 0u) + (v.y != 0u) + (v.z != 0u) + (v.w != 0u);
+  }
+  uint32_t n_entries;
+  uint32_t running = block_exclusive_scan(n_mine, sh->scan, &n_entries);
+  running = __shfl_sync(0xFFFFFFFFu, running, 0);            // entries of the warps before this one
+  const uint32_t lt = (1u << lane) - 1u;
+  for (int k = 0; k < rounds; ++k) {
+    const int q = q_begin + k * 32 + lane;
+    const uint4 v = load_quad(q);
+    if (__ballot_sync(0xFFFFFFFFu, (v.x | v.y | v.z | v.w) != 0u) == 0u) continue;
+    const uint32_t b0 = __ballot_sync(0xFFFFFFFFu, v.x != 0u), b1 = __ballot_sync(0xFFFFFFFFu, v.y != 0u);
+    const uint32_t b2 = __ballot_sync(0xFFFFFFFFu, v.z != 0u), b3 = __ballot_sync(0xFFFFFFFFu, v.w != 0u);
+    uint32_t at = running + __popc(b0 & lt) + __popc(b1 & lt) + __popc(b2 & lt) + __popc(b3 & lt);
+    const uint32_t room = static_cast<uint32_t>(p.budget);  // the list's size; never short unless a quota was overrun
+    if (v.x) { if (at < room) list[at] = 4 * q; ++at; }
+    if (v.y) { if (at < room) list[at] = 4 * q + 1; ++at; }
+    if (v.z) { if (at < room) list[at] = 4 * q + 2; ++at; }
+    if (v.w) { if (at < room) list[at] = 4 * q + 3; ++at; }
+    running += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
+  }
+  __syncthreads();
+  n_entries = min(n_entries, static_cast<uint32_t>(p.budget));
+  const int per = static_cast<int>((n_entries + kSelThreads - 1) / kSelThreads);
+  const int e_begin = min(static_cast<int>(n_entries), static_cast<int>(threadIdx.x) * per);
+  const int e_end = min(static_cast<int>(n_entries), e_begin + per);
+  uint32_t mine = 0;
+  for (int e = e_begin; e < e_end; ++e) {
+    const int w = list[e];
+    mine += __popc(outside_sink(bitmap_word<kBitmapInSmem>(bm, w), w));
+  }
+  uint32_t total;
+  uint32_t at = static_cast<uint32_t>(p.n_sink) + block_exclusive_scan(mine, sh->scan, &total);
+  for (int e = e_begin; e < e_end; ++e) {
+    const int w = list[e];
+    uint32_t bits = outside_sink(bitmap_word<kBitmapInSmem>(bm, w), w);
+    while (bits) {
+      const int b = __ffs(bits) - 1;
+      bits &= bits - 1;
+      if (at < cap) p.out_idx[at] = w * 32 + b;
+      ++at;
+    }
+  }
+  if (threadIdx.x == 0 && total != static_cast<uint32_t>(p.budget)) atomicCAS(p.status, 0, kDevQuota);
 }
 
 template <bool kCluster>
@@ -1159,7 +1226,7 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
 // ---------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------
-size_t select_smem_bytes(long long L, int max_km, SelectParams* p) {
+size_t select_smem_bytes(long long L, int max_km, int budget, SelectParams* p) {
   size_t bytes = 2 * static_cast<size_t>(kSelTile + kMaxWin) * sizeof(float);  // pooling tiles
   if (kSrcTileTokens * sizeof(float) > bytes) bytes = kSrcTileTokens * sizeof(float);
   if (kRankChunk * sizeof(unsigned long long) > bytes) bytes = kRankChunk * sizeof(unsigned long long);
@@ -1172,7 +1239,14 @@ size_t select_smem_bytes(long long L, int max_km, SelectParams* p) {
   p->walk_threads = walkers < 256 ? 256 : (walkers > kSelThreads ? kSelThreads : walkers);
   p->stage_capacity = static_cast<int>(cap);
   p->stage_double = (base + 2 * cap * sizeof(int) <= static_cast<size_t>(kSelMaxDynSmemBytes)) ? 1 : 0;
-  const size_t alloc_bytes = base + (p->stage_double ? 2 : 1) * cap * sizeof(int);
+  size_t after_bitmap = (p->stage_double ? 2 : 1) * cap * sizeof(int);
+  // the output pass lists the bitmap words that hold allocated positions (at most `budget`)
+  // where the staged cells were
+  size_t list_bytes = static_cast<size_t>((L + 31) / 32);
+  if (list_bytes > static_cast<size_t>(budget < 0 ? 0 : budget)) list_bytes = budget < 0 ? 0 : budget;
+  list_bytes *= sizeof(int);
+  if (list_bytes > after_bitmap) after_bitmap = list_bytes;
+  const size_t alloc_bytes = base + after_bitmap;
   if (alloc_bytes > bytes) bytes = alloc_bytes;
   return bytes;
 }

@@ -80,9 +80,9 @@ struct SelectParams {
   int barrier_extra;
 };
 
-// Dynamic shared memory the kernel needs for a context of L positions.
+// Dynamic shared memory the kernel needs for a context of L positions and a budget.
 // Also fills p->bitmap_in_smem, p->stage_capacity, p->stage_double and p->walk_threads.
-size_t select_smem_bytes(long long L, int max_km, SelectParams* p);
+size_t select_smem_bytes(long long L, int max_km, int budget, SelectParams* p);
 // Largest grid that is co-resident on the device (the kernel's CTAs wait on one another).
 cudaError_t select_max_grid(int n_sm, int* max_grid);
 // One cooperative launch: A^C from the encoded maxima, then all of Algorithm 1.

@@ -118,6 +118,11 @@ BIG = [
     (60000, 2, 16382, (1,), (1,), 0, 0),           # largest budget: one staging buffer only
     (1200000, 1, 4096, (1,), (1, 15), 1, 4),       # bitmap too large for shared memory
     (1100000, 1, 2000, (2, 64), (1, 3), 0, 3),     # strided max-pool sources at 1M, m = 64
+    # ascending output pass: word list with a long sink part that ends inside a bitmap word,
+    # a word count that is no multiple of four, a context just past one word per thread
+    (70001, 1, 3000, (1, 4), (1, 7), 1, 5003),
+    (32801, 2, 1500, (1,), (3,), 0, 33),
+    (1200070, 1, 1000, (1,), (1,), 1, 40000),      # the same with the bitmap in global memory
 ]
 
 
