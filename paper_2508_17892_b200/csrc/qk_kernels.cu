@@ -7,6 +7,7 @@
 //                   max over rows of (logit - lse_row); exp is monotone, so one exp per position
 //                   is taken afterwards.
 #include "qk_kernels.cuh"
+#include <utility>
 #include "sm100_ptx.cuh"
 
 namespace ilre {
@@ -187,7 +188,13 @@ row_stats_kernel(const __grid_constant__ CUtensorMap tmapK,
   }
 
   if (warp == 0) {
-    if (lane == 0 && run) producer_loop(&tmapK, &tmapQ, p, it, tail, q_s, k_s, p.skip_tiles);
+    if (lane == 0 && run) {
+      // The packed query comes from the kernel before this one, which may still be running.
+      // After that the next kernel's CTAs may come in as SMs fall free.
+      grid_dep_wait();
+      grid_dep_launch();
+      producer_loop(&tmapK, &tmapQ, p, it, tail, q_s, k_s, p.skip_tiles);
+    }
   } else if (warp == 1) {
     if (lane == 0 && run) {
       constexpr uint32_t idesc = umma_idesc_bf16(128, kTileKeys);
@@ -407,10 +414,6 @@ scores_kernel(const __grid_constant__ CUtensorMap tmapK,
   const CtaItem it = decode_item(p);
   const int n_nh = (p.rb_rows + 255) / 256;
 
-  // Every CTA merges the per-key-chunk statistics of its own rows (a few KB from L2); the
-  // CTAs of the first key chunk also publish the natural-log lse.
-  for (int i = threadIdx.x; i < p.rb_rows; i += blockDim.x)
-    nl[i] = merged_neg_lse2(mp, it.group, i, it.chunk == 0);
   // Two MMA-issuing threads (warps 1 and 2), one per accumulator buffer: tcgen05.mma holds its
   // issuing thread until the tensor pipe takes the instruction, so the waits and commits of
   // one thread overlap the MMAs of the other.  With two row halves per key tile each thread
@@ -422,7 +425,11 @@ scores_kernel(const __grid_constant__ CUtensorMap tmapK,
   const bool run = (it.n_tiles > 0) && (*abort_flag == 0);
 
   if (warp == 0) {
-    if (lane == 0 && run) producer_loop(&tmapK, &tmapQ, p, it, tail, q_s, k_s);
+    if (lane == 0 && run) {
+      grid_dep_wait();                   // the kernel before this one (it packed the query or made the statistics) is done
+      grid_dep_launch();                 // the next kernel's CTAs may come in as SMs fall free
+      producer_loop(&tmapK, &tmapQ, p, it, tail, q_s, k_s);
+    }
   } else if (warp == 1 || warp == 2) {
     if (lane == 0 && run) {
       const uint32_t mine = static_cast<uint32_t>(warp - 1);          // accumulator buffer
@@ -462,6 +469,14 @@ scores_kernel(const __grid_constant__ CUtensorMap tmapK,
       }
     }
   } else if (warp >= 4) {
+    // The consumer warps merge the per-key-chunk statistics of the CTA's rows (a few KB from
+    // L2; the CTAs of the first key chunk also publish the natural-log lse).  The statistics
+    // come from the kernel before this one, which may still be running when this CTA starts
+    // (the set-up above does not wait for it).
+    grid_dep_wait();
+    for (int i = threadIdx.x - 128; i < p.rb_rows; i += kConsumerWarps * 32)
+      nl[i] = merged_neg_lse2(mp, it.group, i, it.chunk == 0);
+    asm volatile("bar.sync 2, %0;" ::"r"(kConsumerWarps * 32) : "memory");
     const int wg = (warp - 4) >> 2;
     const int quad = warp & 3;
     const float c2 = p.c2;
@@ -515,6 +530,7 @@ scores_kernel(const __grid_constant__ CUtensorMap tmapK,
 // and clears the per-run state (encoded scores, bitmap with the sink bits set, selection
 // state).
 __global__ void prepare_kernel(const uint4* __restrict__ q, uint4* __restrict__ qp, PrepParams p) {
+  grid_dep_launch();                     // the statistics kernel sets itself up meanwhile
   const long long tid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   const long long nthreads = static_cast<long long>(gridDim.x) * blockDim.x;
   // packed query: 16 x uint4 per 128-element row
@@ -549,6 +565,24 @@ __global__ void prepare_kernel(const uint4* __restrict__ q, uint4* __restrict__ 
 // ---------------------------------------------------------------------------------------
 // host-side launchers
 // ---------------------------------------------------------------------------------------
+// Launch that may overlap the end of the kernel before it in the stream (programmatic
+// dependent launch): the kernel itself waits (grid_dep_wait) before it touches that kernel's output.
+template <typename... Params, typename... Args>
+static cudaError_t launch_after_previous(void (*kernel)(Params...), int grid, int block, size_t smem,
+                                         cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 size_t row_stats_smem_bytes(int rb_rows, int stages) {
   return static_cast<size_t>(rb_rows) * 256 + static_cast<size_t>(stages) * kStageBytes +
          kSmemTailBytes;
@@ -564,8 +598,8 @@ static cudaError_t launch_row_stats_mt(const CUtensorMap& tk, const CUtensorMap&
   cudaError_t e = cudaFuncSetAttribute(row_stats_kernel<MT, kRowStatsPolyPairs>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  row_stats_kernel<MT, kRowStatsPolyPairs><<<p.n_groups * p.cpg, kStatsThreads, smem, st>>>(tk, tq, p);
-  return cudaGetLastError();
+  return launch_after_previous(row_stats_kernel<MT, kRowStatsPolyPairs>, p.n_groups * p.cpg,
+                               kStatsThreads, smem, st, tk, tq, p);
 }
 
 cudaError_t launch_row_stats(const CUtensorMap& tk, const CUtensorMap& tq, const QkParams& p,
@@ -596,8 +630,7 @@ cudaError_t launch_scores(const CUtensorMap& tk, const CUtensorMap& tq, const Qk
   cudaError_t e = cudaFuncSetAttribute(scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
-  scores_kernel<<<p.n_groups * p.cpg, kQkThreads, smem, st>>>(tk, tq, p, mp);
-  return cudaGetLastError();
+  return launch_after_previous(scores_kernel, p.n_groups * p.cpg, kQkThreads, smem, st, tk, tq, p, mp);
 }
 
 cudaError_t launch_prepare(const void* q, void* qp, const PrepParams& p, int n_sm,

@@ -887,6 +887,7 @@ select_kernel(const ComboTable tbl, const SelectParams p) {
   const int t_end = static_cast<int>(static_cast<long long>(blockIdx.x + 1) * n_tiles / gridDim.x);
   for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) sh.hist[b] = 0u;
   uint32_t epoch = 0;
+  grid_dep_wait();       // the kernel before this one (scores, state cleared for this run) is done
 
   // ---- A: scores from the encoded maxima, one exp per position ----
   if (!p.scores_given) {
@@ -1300,25 +1301,31 @@ cudaError_t launch_select(const ComboTable& table, const SelectParams& p, int gr
   assign_ranking(&tbl, grid);
   // Short contexts need few CTAs: up to kSelClusterMax of them run as one thread-block cluster,
   // whose hardware barrier costs a fraction of a trip to the L2 (not with the self test's
-  // barrier that cannot complete: that one is the counter's).
-  if (grid <= kSelClusterMax && p.barrier_extra == 0) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(kSelThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+  // barrier that cannot complete: that one is the counter's).  Longer ones: a cooperative
+  // launch (every CTA resident: they wait on one another).  Either way the launch may overlap
+  // the end of the kernel before it in the stream; the kernel waits before it reads anything.
+  const bool cluster = grid <= kSelClusterMax && p.barrier_extra == 0;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kSelThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  if (cluster) {
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = grid;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, select_kernel<true>, tbl, p);
+  } else {
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
   }
-  void* args[2] = {&tbl, const_cast<SelectParams*>(&p)};
-  return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(select_kernel<false>), dim3(grid),
-                                     dim3(kSelThreads), args, smem, st);
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  return cluster ? cudaLaunchKernelEx(&cfg, select_kernel<true>, tbl, p)
+                 : cudaLaunchKernelEx(&cfg, select_kernel<false>, tbl, p);
 }
 
 }  // namespace ilre

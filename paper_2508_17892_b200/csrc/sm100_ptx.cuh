@@ -190,6 +190,18 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
+// ---- programmatic dependent launch ----
+// A kernel launched with the programmatic-stream-serialization attribute may start while the
+// kernel before it in the stream still runs, once every CTA of that kernel has called
+// grid_dep_launch() (or exited).  grid_dep_wait() returns when the earlier kernel has completed
+// and its writes are visible; without the attribute both are no-ops.
+__device__ __forceinline__ void grid_dep_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void grid_dep_launch() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ---- packed fp32 arithmetic (two lanes per instruction) and three-input max ----
 __device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
   float2 d;
