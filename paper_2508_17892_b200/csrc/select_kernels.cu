@@ -796,36 +796,35 @@ __device__ __forceinline__ void allocate(const ComboTable& tbl, const SelectPara
     if (threadIdx.x == 0 && total != cap) atomicCAS(p.status, 0, kDevQuota);
     return;
   }
-  const int n_quads = static_cast<int>((n_words + 3) / 4);
+  const int n_w = static_cast<int>(n_words);                // L < 2^31: word and quad numbers fit an int
+  const int n_quads = (n_w + 3) / 4;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rounds = (n_quads + kSelThreads - 1) / kSelThreads;      // per warp
   const int q_begin = warp * rounds * 32;
   int* list = staged;
   // bits of word w that stand for allocated positions outside the sink part
-  auto outside_sink = [&](uint32_t bits, long long w) -> uint32_t {
-    const long long lo = w * 32;
-    if (lo >= p.n_sink) return bits;
-    return (p.n_sink - lo >= 32) ? 0u : (bits & ~((1u << (p.n_sink - lo)) - 1u));
+  const int sink_words = p.n_sink >> 5;                     // words that lie in the sink part entirely
+  const uint32_t sink_tail = ~((1u << (p.n_sink & 31)) - 1u);         // the word after them: its bits outside
+  auto outside_sink = [&](uint32_t bits, int w) -> uint32_t {
+    return (w > sink_words) ? bits : ((w < sink_words) ? 0u : (bits & sink_tail));
   };
+  const int plain_from = sink_words / 4 + 1, plain_to = n_w / 4;      // quads that need no fixing
   auto load_quad = [&](int q) -> uint4 {
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (q >= n_quads) return v;
     if constexpr (kBitmapInSmem) {
       asm volatile("ld.volatile.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                   : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(smem_u32(bm + 4 * q)) : "memory");
+                   : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(smem_u32(bm) + 16u * q) : "memory");
     } else {
       v = __ldcg(reinterpret_cast<const uint4*>(bm) + q);
     }
-    const long long w0 = 4ll * q;
-    if (w0 + 4 > n_words) {                                  // words past the end hold nothing
-      if (w0 + 1 >= n_words) v.y = 0u;
-      if (w0 + 2 >= n_words) v.z = 0u;
-      if (w0 + 3 >= n_words) v.w = 0u;
-    }
-    if (w0 * 32 < p.n_sink) {
-      v.x = outside_sink(v.x, w0); v.y = outside_sink(v.y, w0 + 1);
-      v.z = outside_sink(v.z, w0 + 2); v.w = outside_sink(v.w, w0 + 3);
-    }
+    if (q >= plain_from && q < plain_to) return v;
+    const int w0 = 4 * q;
+    if (w0 + 1 >= n_w) v.y = 0u;                            // words past the end hold nothing
+    if (w0 + 2 >= n_w) v.z = 0u;
+    if (w0 + 3 >= n_w) v.w = 0u;
+    v.x = outside_sink(v.x, w0); v.y = outside_sink(v.y, w0 + 1);
+    v.z = outside_sink(v.z, w0 + 2); v.w = outside_sink(v.w, w0 + 3);
     return v;
   };
   for (int j = threadIdx.x; j < p.n_sink; j += kSelThreads) p.out_idx[j] = j;
