@@ -336,3 +336,42 @@ def test_full_size_1m_config_against_the_full_oracle():
     print("cfg5_L1m in 8 shards", rep8)
     assert np.abs(sc8 - sc).max() <= 2e-5 * sc.max() and np.all(np.abs(sc8 - sc) <= 1e-4 * sc)
     eng.close()
+
+
+def test_recalls_in_a_row_on_a_side_stream_keep_their_own_results():
+    """The kernels of a recall start while the one before them still runs and wait before they
+    read its output.  Recalls queued back to back on one stream without a synchronisation in
+    between -- different keys, queries and lengths each time, work of another library before
+    and between them on the same stream -- must each give the list and the scores that the
+    same recall gives alone."""
+    ws = [small_workload(L, q_len, seed=70 + i, n_spans=3, budget=b, max_sizes=(1, 2), win_sizes=(1, 5),
+                         win_op=i % 2, n_sink=2)
+          for i, (L, q_len, b) in enumerate([(9000, 16, 300), (30000, 4, 700), (5000, 33, 128),
+                                             (30000, 4, 700), (12000, 64, 512)])]
+    xs = [make_inputs(w) for w in ws]
+    w0 = max(ws, key=lambda w: w.L)
+    eng = _engine(w0, max_q_len=max(w.q_len for w in ws), max_budget=max(w.budget for w in ws))
+    alone = []
+    for w, x in zip(ws, xs):
+        idx, sc = _run(eng, x)
+        alone.append((idx, sc))
+    side = torch.cuda.Stream()
+    Ks = [x.K.cuda() for x in xs]
+    Qs = [x.Q.cuda() for x in xs]
+    scratch = torch.zeros(1 << 22, device="cuda")
+    torch.cuda.synchronize()
+    outs = []
+    with torch.cuda.stream(side):
+        for rep in range(3):
+            for w, K, Q in zip(ws, Ks, Qs):
+                scratch.add_(1.0)                              # a foreign kernel before the recall
+                idx, sc = eng.run(K, Q, w.budget, w.max_sizes, w.win_sizes, w.win_op, w.n_sink,
+                                  want_scores=True, stream=side)
+                outs.append((idx, sc))
+    side.synchronize()
+    eng.check_status()
+    for n, (idx, sc) in enumerate(outs):
+        ref_idx, ref_sc = alone[n % len(ws)]
+        assert np.array_equal(idx.cpu().numpy(), ref_idx), f"recall {n}"
+        assert np.array_equal(sc.cpu().numpy(), ref_sc), f"scores of recall {n}"
+    eng.close()
