@@ -23,6 +23,10 @@ CASES = [
     (300, 1000, 4, 4),         # long prefix, no grouping
     (200, 130, 28, 4),         # seven query heads per kv head: one head per CTA
     (2048, 516, 8, 2),         # 16 query tiles, up to 21 key tiles: the K/V ring wraps many times
+    # more widths of the visible part of the last key tile (40, 60 and 90 keys here)
+    (128, 40, 4, 2),
+    (256, 60, 2, 1),
+    (384, 90, 4, 4),
 ]
 
 
