@@ -8,6 +8,8 @@
 #include <cstring>
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "../../include/ilre_recall.h"
 #include "attn_kernels.cuh"
 #include "fill_kernels.cuh"
@@ -95,6 +97,14 @@ struct ilre_recall {
 };
 
 namespace {
+
+// A named range on the host time line for tracing tools that read NVTX (a no-op without one).
+struct TraceRange {
+  explicit TraceRange(const char* name) { nvtxRangePushA(name); }
+  ~TraceRange() { nvtxRangePop(); }
+  TraceRange(const TraceRange&) = delete;
+  TraceRange& operator=(const TraceRange&) = delete;
+};
 
 struct DeviceGuard {
   int prev;
@@ -457,21 +467,29 @@ int recall_impl(ilre_recall_t* h, const void* k_cache_dev, int64_t L, const void
   mp.ext_stats = io.ext_stats; mp.n_ext = io.n_ext;
   if (io.scores_in) { sp.scores = const_cast<float*>(io.scores_in); sp.scores_given = 1; }
   ILRE_MARK(0);
-  ILRE_CUDA(launch_prepare(query_dev, h->qp, pp, h->n_sm, st)); ++launches;
+  {
+    TraceRange r("ilre: prepare");
+    ILRE_CUDA(launch_prepare(query_dev, h->qp, pp, h->n_sm, st)); ++launches;
+  }
   ILRE_MARK(1);
   if (io.stages & kStageStats) {
+    TraceRange r("ilre: row statistics (Eq. 4)");
     ILRE_CUDA(launch_row_stats(map_k, map_q, qk, st)); ++launches;
     if (io.stats_out) { ILRE_CUDA(launch_export_stats(mp, io.stats_out, st)); ++launches; }
   }
   ILRE_MARK(2);
   if (io.stages & kStageScores) {
+    TraceRange r("ilre: scores (Eq. 5)");
     ILRE_CUDA(launch_scores(map_k, map_q, qk, mp, st)); ++launches;
     if (io.shard_scores_out) {
       ILRE_CUDA(launch_decode_scores(h->enc, io.shard_scores_out, L, st)); ++launches;
     }
   }
   ILRE_MARK(3);
-  if (with_select) { ILRE_CUDA(launch_select(tbl, sp, select_grid, select_smem, st)); ++launches; }
+  if (with_select) {
+    TraceRange r("ilre: selection (Algorithm 1)");
+    ILRE_CUDA(launch_select(tbl, sp, select_grid, select_smem, st)); ++launches;
+  }
   ILRE_MARK(4);
 #undef ILRE_MARK
   h->last_launches = launches;
@@ -521,6 +539,7 @@ int ilre_recall_run_host(ilre_recall_t* h, const void* k_cache_host, int64_t L,
                          const void* query_host, int32_t q_len, int32_t budget,
                          const ilre_pool_spec_t* spec, int32_t* out_idx_host,
                          float* out_scores_host, void* cuda_stream) {
+  TraceRange trace("ilre: recall from host memory");
   if (!h || !h->stage_k) return ILRE_ERR_INVALID_ARG;
   const int v = validate_run(h, k_cache_host, L, query_host, q_len, budget, spec, out_idx_host,
                              true, true);
@@ -584,6 +603,7 @@ int ilre_recall_run_host(ilre_recall_t* h, const void* k_cache_host, int64_t L,
 int ilre_recall_chunk_attention(ilre_recall_t* h, const void* q_dev, const void* k_dev,
                                 const void* v_dev, int32_t chunk_len, int32_t n_prefix,
                                 void* out_dev, void* cuda_stream) {
+  TraceRange trace("ilre: chunk attention (Eq. 2)");
   if (!h || !q_dev || !k_dev || !v_dev || !out_dev || chunk_len < 1 || n_prefix < 0)
     return ILRE_ERR_INVALID_ARG;
   if (static_cast<long long>(chunk_len) + n_prefix > 2147483647LL - 256) return ILRE_ERR_CAPACITY;
@@ -615,6 +635,7 @@ int ilre_recall_chunk_attention(ilre_recall_t* h, const void* q_dev, const void*
 int ilre_recall_fill_keys(ilre_recall_t* h, const void* x_dev, int64_t n_tok, int32_t d_model,
                           const void* w_k_dev, const void* bias_dev, int64_t pos0,
                           double rope_theta, void* k_cache_dev, int64_t L, void* cuda_stream) {
+  TraceRange trace("ilre: key fill (Eq. 1, Eq. 3)");
   if (!h || !x_dev || !w_k_dev || !k_cache_dev || n_tok < 0 || d_model < 1 || pos0 < 0 || L < 1 ||
       !(rope_theta > 1.0))
     return ILRE_ERR_INVALID_ARG;
@@ -666,6 +687,7 @@ int ilre_recall_fill_keys(ilre_recall_t* h, const void* x_dev, int64_t n_tok, in
 int ilre_recall_rerope_keys(ilre_recall_t* h, const void* k_cache_dev, void* k_out_dev, int64_t L,
                             int32_t chunk_size, int32_t n_sink, double rope_theta,
                             void* cuda_stream) {
+  TraceRange trace("ilre: re-rotation (Eq. 7)");
   if (!h || !k_cache_dev || !k_out_dev || L < 1 || chunk_size < 1 || n_sink < 0 || n_sink > L ||
       !(rope_theta > 1.0))
     return ILRE_ERR_INVALID_ARG;
