@@ -321,6 +321,14 @@ int ilre_recall_stage_times(ilre_recall_t* h, float* ms_host, int32_t n);
 #define ILRE_SELFTEST_MISSING_KEY_TILE 2
 int ilre_recall_selftest_wait(ilre_recall_t* h, int64_t wait_cycle_limit, int32_t what);
 
+/* Debugging aid (the paper has no counterpart): every workspace buffer of the handle is followed
+ * by a 256-byte guard zone filled with a pattern when the handle is created; no kernel may write
+ * there.  Waits for the device to go idle, reads the zones back and returns how many of them no
+ * longer hold the pattern (0 = none: no kernel of any call so far wrote past the end of a
+ * workspace buffer), or a negative ILRE_ERR_* code (a null handle: ILRE_ERR_INVALID_ARG).  Host
+ * call; synchronises; meant for tests, not for the hot path. */
+int ilre_recall_check_guards(ilre_recall_t* h);
+
 /* Number of kernel launches issued by the last run(). */
 int ilre_recall_last_launch_count(ilre_recall_t* h);
 

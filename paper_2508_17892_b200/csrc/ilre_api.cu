@@ -40,10 +40,16 @@ struct Geometry {
 
 }  // namespace
 
+static constexpr int kGuardBytes = 256;       // written once behind every workspace buffer
+static constexpr int kGuardByte = 0xA5;
+static constexpr int kMaxGuards = 48;
+
 struct ilre_recall {
   ilre_recall_config_t cfg;
   int n_sm;
   EncodeTiledFn encode;
+  const uint8_t* guard[kMaxGuards];           // the guard zones, for ilre_recall_check_guards
+  int n_guards;
   // workspace (device)
   void* qp;
   float* partial;
@@ -141,10 +147,18 @@ Geometry make_geometry(const ilre_recall_config_t& c, int n_sm, long long L, int
   return g;
 }
 
+// One workspace buffer of the handle, followed by a guard zone of kGuardBytes that nothing may
+// write to (checked by ilre_recall_check_guards).
 template <class T>
-bool dev_alloc(T** p, size_t count) {
+bool dev_alloc(ilre_recall* h, T** p, size_t count) {
   *p = nullptr;
-  return cudaMalloc(reinterpret_cast<void**>(p), (count ? count : 1) * sizeof(T)) == cudaSuccess;
+  const size_t bytes = ((count ? count : 1) * sizeof(T) + 15) & ~static_cast<size_t>(15);
+  if (h->n_guards >= kMaxGuards) return false;
+  if (cudaMalloc(reinterpret_cast<void**>(p), bytes + kGuardBytes) != cudaSuccess) return false;
+  uint8_t* zone = reinterpret_cast<uint8_t*>(*p) + bytes;
+  if (cudaMemset(zone, kGuardByte, kGuardBytes) != cudaSuccess) return false;
+  h->guard[h->n_guards++] = zone;
+  return true;
 }
 
 void free_all(ilre_recall* h) {
@@ -263,33 +277,33 @@ int ilre_recall_create(const ilre_recall_config_t* cfg, ilre_recall_t** out) {
   h->cand_stride = (cfg->max_budget + 2 + 3) & ~3;    // rows of the ranked lists start 16-byte aligned
 
   bool ok = true;
-  ok = ok && dev_alloc(reinterpret_cast<uint8_t**>(&h->qp), cfg->n_kv_heads * rows_pad * 256);
-  ok = ok && dev_alloc(&h->partial, max_items * kMaxRbRows * 2);
-  ok = ok && dev_alloc(&h->row_lse, static_cast<size_t>(cfg->max_q_len) * cfg->n_q_heads);
-  ok = ok && dev_alloc(&h->enc, maxL);
-  ok = ok && dev_alloc(&h->scores, maxL);
-  ok = ok && dev_alloc(&h->pooled, ncomb * maxL);
-  ok = ok && dev_alloc(&h->maxpooled, ncomb * (maxL / 2 + 1));   // one array per distinct m > 1
-  ok = ok && dev_alloc(&h->hist, static_cast<size_t>(kSelectPasses) * kMaxCombos * kHistBins);
-  ok = ok && dev_alloc(&h->tile_ties, ncomb * (maxL / kSelTile + 1));
-  ok = ok && dev_alloc(&h->grid_barrier, 1);
-  ok = ok && dev_alloc(&h->rope_table, static_cast<size_t>(kRopeTableRows) * kRopeHalfDim);
+  ok = ok && dev_alloc(h, reinterpret_cast<uint8_t**>(&h->qp), cfg->n_kv_heads * rows_pad * 256);
+  ok = ok && dev_alloc(h, &h->partial, max_items * kMaxRbRows * 2);
+  ok = ok && dev_alloc(h, &h->row_lse, static_cast<size_t>(cfg->max_q_len) * cfg->n_q_heads);
+  ok = ok && dev_alloc(h, &h->enc, maxL);
+  ok = ok && dev_alloc(h, &h->scores, maxL);
+  ok = ok && dev_alloc(h, &h->pooled, ncomb * maxL);
+  ok = ok && dev_alloc(h, &h->maxpooled, ncomb * (maxL / 2 + 1));   // one array per distinct m > 1
+  ok = ok && dev_alloc(h, &h->hist, static_cast<size_t>(kSelectPasses) * kMaxCombos * kHistBins);
+  ok = ok && dev_alloc(h, &h->tile_ties, ncomb * (maxL / kSelTile + 1));
+  ok = ok && dev_alloc(h, &h->grid_barrier, 1);
+  ok = ok && dev_alloc(h, &h->rope_table, static_cast<size_t>(kRopeTableRows) * kRopeHalfDim);
   h->pos_hi_rows = static_cast<int>(cfg->max_L / kRopeLoRows + 2);
-  ok = ok && dev_alloc(&h->pos_lo, static_cast<size_t>(kRopeLoRows) * 64);
-  ok = ok && dev_alloc(&h->pos_hi, static_cast<size_t>(h->pos_hi_rows) * 64);
-  ok = ok && dev_alloc(&h->cand, ncomb * h->cand_stride);
-  ok = ok && dev_alloc(&h->cand_count, 4 * static_cast<size_t>(kMaxCombos));
-  ok = ok && dev_alloc(&h->pending, ncomb * kPendCap);
-  ok = ok && dev_alloc(&h->ranked, ncomb * h->cand_stride);
-  ok = ok && dev_alloc(&h->bitmap, (maxL + 31) / 32 + 4);    // read four words at a time
-  ok = ok && dev_alloc(&h->status, 1);
-  ok = ok && dev_alloc(&h->clk, 2);
+  ok = ok && dev_alloc(h, &h->pos_lo, static_cast<size_t>(kRopeLoRows) * 64);
+  ok = ok && dev_alloc(h, &h->pos_hi, static_cast<size_t>(h->pos_hi_rows) * 64);
+  ok = ok && dev_alloc(h, &h->cand, ncomb * h->cand_stride);
+  ok = ok && dev_alloc(h, &h->cand_count, 4 * static_cast<size_t>(kMaxCombos));
+  ok = ok && dev_alloc(h, &h->pending, ncomb * kPendCap);
+  ok = ok && dev_alloc(h, &h->ranked, ncomb * h->cand_stride);
+  ok = ok && dev_alloc(h, &h->bitmap, (maxL + 31) / 32 + 4);    // read four words at a time
+  ok = ok && dev_alloc(h, &h->status, 1);
+  ok = ok && dev_alloc(h, &h->clk, 2);
   if (ok && cfg->host_staging) {
-    ok = ok && dev_alloc(reinterpret_cast<uint8_t**>(&h->stage_k), maxL * cfg->n_kv_heads * 256);
-    ok = ok && dev_alloc(reinterpret_cast<uint8_t**>(&h->stage_q),
+    ok = ok && dev_alloc(h, reinterpret_cast<uint8_t**>(&h->stage_k), maxL * cfg->n_kv_heads * 256);
+    ok = ok && dev_alloc(h, reinterpret_cast<uint8_t**>(&h->stage_q),
                          static_cast<size_t>(cfg->max_q_len) * cfg->n_q_heads * 256);
-    ok = ok && dev_alloc(&h->stage_idx, static_cast<size_t>(cfg->max_budget) + kMaxSinkStaging);
-    ok = ok && dev_alloc(&h->piece_stats, static_cast<size_t>(kHostPieces) * cfg->max_q_len * cfg->n_q_heads);
+    ok = ok && dev_alloc(h, &h->stage_idx, static_cast<size_t>(cfg->max_budget) + kMaxSinkStaging);
+    ok = ok && dev_alloc(h, &h->piece_stats, static_cast<size_t>(kHostPieces) * cfg->max_q_len * cfg->n_q_heads);
     ok = ok && (cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking) == cudaSuccess);
     ok = ok && (cudaEventCreateWithFlags(&h->copy_begin, cudaEventDisableTiming) == cudaSuccess);
     for (int i = 0; ok && i < kHostPieces; ++i)
@@ -856,6 +870,23 @@ int ilre_recall_stage_times(ilre_recall_t* h, float* ms_host, int32_t n) {
     }
   }
   return cnt;
+}
+
+int ilre_recall_check_guards(ilre_recall_t* h) {
+  if (!h) return ILRE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return ILRE_ERR_CUDA;
+  if (cudaDeviceSynchronize() != cudaSuccess) return ILRE_ERR_CUDA;
+  int damaged = 0;
+  uint8_t zone[kGuardBytes];
+  for (int i = 0; i < h->n_guards; ++i) {
+    if (cudaMemcpy(zone, h->guard[i], kGuardBytes, cudaMemcpyDeviceToHost) != cudaSuccess)
+      return ILRE_ERR_CUDA;
+    bool intact = true;
+    for (int b = 0; b < kGuardBytes; ++b) intact = intact && zone[b] == kGuardByte;
+    damaged += intact ? 0 : 1;
+  }
+  return damaged;
 }
 
 int ilre_recall_last_launch_count(ilre_recall_t* h) {

@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = (
     "ilre_recall_copy_row_lse",
     "ilre_recall_status", "ilre_recall_selftest_wait", "ilre_recall_set_profiling", "ilre_recall_stage_times",
     "ilre_recall_sm_clock",
-    "ilre_recall_last_launch_count", "ilre_recall_destroy", "ilre_strerror",
+    "ilre_recall_last_launch_count", "ilre_recall_check_guards", "ilre_recall_destroy", "ilre_strerror",
     "ilre_topk_positions_noalloc",
 )
 
@@ -86,6 +86,7 @@ def load_library() -> ctypes.CDLL:
     lib.ilre_recall_selftest_wait.argtypes = [vp, i64, i32]
     lib.ilre_recall_stage_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float), i32]
     lib.ilre_recall_last_launch_count.argtypes = [vp]
+    lib.ilre_recall_check_guards.argtypes = [vp]
     lib.ilre_recall_destroy.argtypes = [vp]
     lib.ilre_strerror.argtypes = [ctypes.c_int]
     lib.ilre_topk_positions_noalloc.argtypes = [vp, i64, i32, vp, vp]
@@ -424,6 +425,13 @@ class IlreRecall:
         if rc != 0:
             raise IlreError(rc, "ilre_recall_sm_clock")
         return float(mhz.value)
+
+    def check_guards(self) -> int:
+        """Number of workspace buffers whose guard zone was written to (0 = none); synchronises."""
+        rc = self._lib.ilre_recall_check_guards(self._h)
+        if rc < 0:
+            raise IlreError(rc, "ilre_recall_check_guards")
+        return rc
 
     def last_launch_count(self) -> int:
         return self._lib.ilre_recall_last_launch_count(self._h)

@@ -63,6 +63,7 @@ def test_null_handle_calls_return_invalid_arg(lib):
     assert lib.ilre_recall_set_profiling(None, 1) == -1
     assert lib.ilre_recall_selftest_wait(None, 0, 0) == -1
     assert lib.ilre_recall_last_launch_count(None) == -1
+    assert lib.ilre_recall_check_guards(None) == -1
     assert lib.ilre_recall_run(None, None, 1, None, 1, 0, None, None, None, None) == -1
     assert lib.ilre_recall_run_host(None, None, 1, None, 1, 0, None, None, None, None) == -1
     assert lib.ilre_recall_shard_stats(None, None, 1, None, 1, None, None) == -1

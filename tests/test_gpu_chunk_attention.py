@@ -52,4 +52,5 @@ def test_chunk_attention_matches_oracle(case):
     assert np.all(err <= bound), float((err / bound).max())
     # on average the two roundings are far smaller than their bounds
     assert err.mean() < 2e-3 * vmax
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()

@@ -65,6 +65,7 @@ def test_rerope_matches_oracle(case):
     n_chunks = -(-(L - n_sink) // chunk)
     keep_from = n_sink + max(n_chunks - 2, 0) * chunk
     assert torch.equal(out[keep_from:].cpu(), K[keep_from:])
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -78,6 +79,7 @@ def test_too_many_chunks_is_refused():
     with pytest.raises(IlreError) as e:
         eng.rerope_keys(K, 0)
     assert e.value.code == -1
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -109,6 +111,7 @@ def test_recall_on_rerotated_keys_matches_oracle():
     assert np.quantile(rel, 0.999) < 2e-3 and rel.max() < 0.05
     planted = set(x.planted_positions().tolist())
     assert len(planted & set(idx.cpu().tolist())) == len(planted & set(ref_idx.tolist()))
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -172,6 +175,7 @@ def test_recall_with_dca_against_the_oracle_pipeline(name, chunk, n_sink):
     ref_idx = oracle.allocate(a_ref, *spec)
     print(name, "positions with identical keys", same_rows.mean(), "max delta", delta.max(),
           "delta_lse", delta_lse, "index differences", len(set(idx.tolist()) ^ set(ref_idx.tolist())))
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -207,6 +211,7 @@ def test_sink_rerope_matches_oracle(case):
     eng.rerope_sinks(inplace, chunk, i, out=inplace)
     torch.cuda.synchronize()
     assert torch.equal(inplace, out)
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -231,4 +236,5 @@ def test_sink_rerope_chunk_by_chunk_and_with_eq7_on_one_handle():
         eng.rerope_sinks(src, 256, 0)
     torch.cuda.synchronize()
     eng.check_status()
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()

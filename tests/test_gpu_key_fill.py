@@ -64,6 +64,7 @@ def test_fill_matches_oracle(case):
     _check(cache[pos0:pos0 + n_tok], want, X, W, bias)
     # rows outside the filled range keep their contents
     assert torch.all(cache[:pos0] == 7.0) and torch.all(cache[pos0 + n_tok:] == 7.0)
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -93,6 +94,7 @@ def test_chunked_fill_equals_one_call_and_feeds_the_recall():
     torch.cuda.synchronize()
     eng.check_status()
     parity.check_recall(whole.cpu(), Q, w, idx.cpu().numpy(), sc.cpu().numpy())
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -111,6 +113,7 @@ def test_fill_argument_errors():
         eng.fill_keys(X, W, cache, 2000)                                   # runs past the cache
     assert e.value.code == -3
     assert eng.status() == 0
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 

@@ -88,3 +88,4 @@ def test_sweep_over_candidate_layers_matches_the_oracle():
     assert layer == r_layer
     assert full[layer] == full.max() and np.all(full[:layer] < full.max())
     assert len(set(full.tolist())) >= 3          # the layers do differ
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"

@@ -57,4 +57,5 @@ def test_random_configuration(seed):
     idx3, _ = eng.run_host(x.K, x.Q, *spec)
     eng.check_status()
     assert np.array_equal(idx3.numpy(), idx.cpu().numpy())
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()

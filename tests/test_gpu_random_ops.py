@@ -63,4 +63,5 @@ def test_random_shapes(seed):
     assert np.all(np.abs(got - ref) <= 2.0 ** -8 * (1 + 1e-3) * np.abs(ref) + 1e-6 * pair + 1e-7)
     assert float(cache[pos0 + n_tok:].abs().max()) == 0.0
     assert pos0 == 0 or float(cache[:pos0].abs().max()) == 0.0
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()

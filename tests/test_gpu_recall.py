@@ -58,6 +58,7 @@ def test_benchmark_configs_match_oracle(cases, name):
     planted = set(x.planted_positions().tolist())
     ref_idx = oracle.allocate(a, w.budget, w.max_sizes, w.win_sizes, w.win_op, w.n_sink)
     assert len(planted & set(idx.tolist())) == len(planted & set(ref_idx.tolist()))
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -76,6 +77,7 @@ def test_other_pooling_specs(cases, name, variant):
     idx, sc = _run(eng, x, spec)
     rep = parity.check_recall(x.K, x.Q, w, idx, sc, ref_scores=a, spec=spec)
     print(name, variant, rep)
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -108,6 +110,7 @@ def test_ragged_shapes_match_oracle(case):
     idx, sc = _run(eng, x)
     rep = parity.check_recall(x.K, x.Q, w, idx, sc)
     print(case, rep)
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -137,6 +140,7 @@ def test_selection_kernel_edge_paths(case):
     idx, sc = _run(eng, x)
     rep = parity.check_recall(x.K, x.Q, w, idx, sc)
     print(case, rep)
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -173,6 +177,7 @@ def test_massive_ties_follow_the_cell_order(pattern, win_op):
     if pattern == "all_equal":
         assert np.unique(sc).size == 1
     print(pattern, win_op, rep)
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -187,6 +192,7 @@ def test_handle_reuse_and_determinism(cases):
     again = _run(eng, big)
     np.testing.assert_array_equal(first[0], again[0])
     np.testing.assert_array_equal(first[1], again[1])
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -201,6 +207,7 @@ def test_run_host_matches_run(cases):
     eng.check_status()
     np.testing.assert_array_equal(idx_host.numpy(), idx_dev)
     parity.check_recall(x.K, x.Q, w, idx_host.numpy(), sc_host.numpy(), ref_scores=a)
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -222,6 +229,7 @@ def test_run_host_pipelined_upload_matches_oracle(cases, name):
     # twice in a row on one handle: same result (the staging buffer is reused)
     idx2, _ = eng.run_host(x.K, x.Q, w.budget, w.max_sizes, w.win_sizes, w.win_op, w.n_sink)
     np.testing.assert_array_equal(idx2.numpy(), idx_host.numpy())
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -250,6 +258,7 @@ def test_recall_can_be_captured_in_a_cuda_graph(cases):
         assert torch.equal(out, direct)
     eng.check_status()
     del graph
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -262,6 +271,7 @@ def test_in_kernel_sm_clock_is_plausible(cases):
     mhz = eng.sm_clock_mhz()
     eng.set_profiling(False)
     assert 300.0 < mhz < 2500.0, mhz
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -290,6 +300,7 @@ def test_error_codes_on_device(cases):
     big = torch.zeros(w.L + 1, 8, 128, dtype=torch.bfloat16, device="cuda")
     assert code(K=big) == -3
     assert eng.status() == 0
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -335,6 +346,7 @@ def test_full_size_1m_config_against_the_full_oracle():
     rep8 = parity.check_recall(x.K, x.Q, w, idx8, sc8, ref_scores=a)
     print("cfg5_L1m in 8 shards", rep8)
     assert np.abs(sc8 - sc).max() <= 2e-5 * sc.max() and np.all(np.abs(sc8 - sc) <= 1e-4 * sc)
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -374,4 +386,5 @@ def test_recalls_in_a_row_on_a_side_stream_keep_their_own_results():
         ref_idx, ref_sc = alone[n % len(ws)]
         assert np.array_equal(idx.cpu().numpy(), ref_idx), f"recall {n}"
         assert np.array_equal(sc.cpu().numpy(), ref_sc), f"scores of recall {n}"
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()

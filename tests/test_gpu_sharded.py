@@ -59,6 +59,7 @@ def test_sharded_steps_match_oracle(name, cuts):
     gpu_lse = eng.row_lse(w.q_len).cpu().numpy().reshape(-1)
     assert np.abs(gpu_lse - (m + np.log(z))).max() < 5e-4
     print(name, len(cuts) - 1, rep)
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
 
 
 def test_one_shard_is_the_unsharded_run_bit_for_bit():
@@ -72,6 +73,7 @@ def test_one_shard_is_the_unsharded_run_bit_for_bit():
     idx, sc, _ = _sharded(eng, K, Q, [0, w.L], w)
     assert np.array_equal(sc, sc0)
     assert np.array_equal(idx, idx0)
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
 
 
 def test_ragged_shards_sinks_and_strided_pooling():
@@ -84,6 +86,7 @@ def test_ragged_shards_sinks_and_strided_pooling():
     idx, sc, _ = _sharded(eng, x.K.cuda(), x.Q.cuda(), [0, 100, 1900, 1901, 4000, w.L], w)
     rep = parity.check_recall(x.K, x.Q, w, idx, sc)
     print(rep)
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
 
 
 @pytest.mark.parametrize("win_op", [0, 1])

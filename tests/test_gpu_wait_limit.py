@@ -53,6 +53,7 @@ def test_a_wait_that_cannot_complete_gives_up_and_the_handle_recovers(what):
     # a short budget alone (nothing injected) does not disturb a run of this size
     eng.selftest_wait(50_000_000, 0)
     assert torch.equal(_good_run(eng, x, w, spec, K, Q), want)
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
 
 
@@ -63,4 +64,5 @@ def test_selftest_arguments_are_checked():
         with pytest.raises(IlreError) as e:
             eng.selftest_wait(*bad)
         assert e.value.code == -1
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
