@@ -626,7 +626,7 @@ def run_ours(args, world, rank, local):
                 row = time_side_workload(eng, dev, sw, sx, args.side_steps, flush, peaks_now)
                 del sx
             if name.startswith("probe"):
-                row["note"] = ("not a BASELINE config: q_len 16 puts the key scan below the ridge, "
+                row["note"] = ("not one of the five benchmark configurations: q_len 16 puts the key scan below the ridge, "
                                "so per_pass.*_hbm_frac is the streaming efficiency of each pass")
             configs_block[name] = row
         del flush
