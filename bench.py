@@ -203,12 +203,33 @@ def time_side_workload(eng, dev, w, x, steps, flush, peaks, K=None, Q=None):
     b.record()
     torch.cuda.synchronize()
     ms_warm = a.elapsed_time(b) / steps
+    # short contexts: the same recalls captured once in a CUDA graph and replayed (the call
+    # allocates nothing and never synchronises, so it can be captured)
+    ms_graph = None
+    if w.L <= 131072:
+        side = torch.cuda.Stream(device=dev)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            eng.run(K, Q, *spec, out_idx=out_idx, stream=side)
+            torch.cuda.synchronize()
+            with torch.cuda.graph(graph, stream=side):
+                for _ in range(steps):
+                    eng.run(K, Q, *spec, out_idx=out_idx, stream=side)
+        graph.replay()
+        torch.cuda.synchronize()
+        a.record()
+        graph.replay()
+        b.record()
+        torch.cuda.synchronize()
+        ms_graph = a.elapsed_time(b) / steps
+        eng.check_status()
+        del graph
     ms = ms_all[len(ms_all) // 2]
     k_bytes = K.numel() * 2
     flops = 2.0 * w.q_len * w.n_q_heads * w.L * w.d
     gbs = k_bytes / (ms * 1e-3) / 1e9
     row = dict(workload=workload_string(w), ms_per_recall=ms, ms_mean=sum(ms_all) / len(ms_all),
-               ms_min=ms_all[0], ms_back_to_back=ms_warm, steps=steps,
+               ms_min=ms_all[0], ms_back_to_back=ms_warm, ms_graph_replay=ms_graph, steps=steps,
                l2="flushed before every recall (256 MiB write, untimed)",
                key_cache_gbs=gbs, stages_ms=stages, launches_per_recall=eng.last_launch_count(),
                hbm_frac_one_read_of_K=gbs / peaks["hbm_gbs"],
