@@ -145,7 +145,8 @@ def test_selection_kernel_edge_paths(case):
 
 
 @pytest.mark.parametrize("pattern", ["all_equal", "two_levels", "blocks_of_equal", "all_equal_40k",
-                                     "blocks_of_equal_40k"])
+                                     "blocks_of_equal_40k", "all_equal_40k_B6000",
+                                     "blocks_of_equal_40k_B6000"])
 @pytest.mark.parametrize("win_op", [0, 1])
 def test_massive_ties_follow_the_cell_order(pattern, win_op):
     """Keys that repeat make whole stretches of the scores bit-identical, so the K_m-th value
@@ -153,9 +154,13 @@ def test_massive_ties_follow_the_cell_order(pattern, win_op):
     plateaus are shorter (one CTA sorts the tied cells out) or longer (further passes over the
     whole array) than what the selection sets aside for one CTA, sometimes both in one call."""
     import dataclasses
+    # the larger budget makes lists of 1024 to 8192 candidates: ranked inside value buckets
+    # whose sampled splitters then differ in the cell index only
+    budget = 6000 if pattern.endswith("_B6000") else 700
+    pattern = pattern.replace("_B6000", "")
     L, q_len = (40000, 2) if pattern.endswith("_40k") else (9000, 3)
     pattern = pattern.replace("_40k", "")
-    w = small_workload(L, q_len, seed=3, n_spans=0, budget=700, max_sizes=(1, 2), win_sizes=(1, 3),
+    w = small_workload(L, q_len, seed=3, n_spans=0, budget=budget, max_sizes=(1, 2), win_sizes=(1, 3),
                        win_op=win_op, n_sink=2)
     x = make_inputs(w)
     g = torch.Generator().manual_seed(17)
