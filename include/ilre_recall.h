@@ -186,7 +186,10 @@ int ilre_recall_chunk_attention(ilre_recall_t* h, const void* q_dev, const void*
  * one rounding to bf16.  Asynchronous on cuda_stream; bounded waits report through
  * ilre_recall_status.  The handle keeps the angle tables between calls (they depend on
  * rope_theta only); a call on another stream than the one that built them waits for the build
- * on the device, but calls with different rope_theta on one handle must not overlap.
+ * on the device, but calls with different rope_theta on one handle must not overlap.  Under
+ * CUDA-graph capture: a call that would have to build the tables returns ILRE_ERR_UNSUPPORTED
+ * (make one call with this rope_theta before the capture), and a captured call does not wait
+ * for a build issued on another stream: launch the graph behind that build.
  */
 int ilre_recall_fill_keys(ilre_recall_t* h, const void* x_dev, int64_t n_tok, int32_t d_model,
                           const void* w_k_dev, const void* bias_dev, int64_t pos0,
@@ -207,7 +210,10 @@ int ilre_recall_fill_keys(ilre_recall_t* h, const void* x_dev, int64_t n_tok, in
  * (nearest even).  Asynchronous on cuda_stream.  At most 8192 + 2 chunks
  * (ILRE_ERR_CAPACITY beyond).  The handle keeps the angle table between calls; a call on
  * another stream waits on the device for the table's build, but calls that need different
- * tables (chunk size, theta, more rows) must not overlap on one handle.
+ * tables (chunk size, theta, more rows) must not overlap on one handle.  Under CUDA-graph
+ * capture: a call that would have to (re)build the table returns ILRE_ERR_UNSUPPORTED (make one
+ * call with these arguments before the capture), and a captured call does not wait for a build
+ * issued on another stream: launch the graph behind that build.
  */
 int ilre_recall_rerope_keys(ilre_recall_t* h, const void* k_cache_dev, void* k_out_dev,
                             int64_t L, int32_t chunk_size, int32_t n_sink, double rope_theta,

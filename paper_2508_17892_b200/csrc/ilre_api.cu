@@ -112,6 +112,20 @@ struct TraceRange {
   TraceRange& operator=(const TraceRange&) = delete;
 };
 
+// True while `st` is being captured into a CUDA graph.
+bool capturing(cudaStream_t st) {
+  cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+  return cudaStreamIsCapturing(st, &cs) == cudaSuccess && cs != cudaStreamCaptureStatusNone;
+}
+
+// Makes `st` wait for the table build that `ev` marks, issued on another stream.  A stream
+// under capture may not wait for an event recorded outside the capture: there the caller
+// orders the graph's launch behind the build (the build itself is refused under capture).
+cudaError_t wait_for_tables(cudaStream_t st, cudaEvent_t ev) {
+  if (capturing(st)) return cudaSuccess;
+  return cudaStreamWaitEvent(st, ev, 0);
+}
+
 struct DeviceGuard {
   int prev;
   bool ok;
@@ -665,13 +679,14 @@ int ilre_recall_fill_keys(ilre_recall_t* h, const void* x_dev, int64_t n_tok, in
   h->last_stream = st;
   int launches = 0;
   if (h->pos_theta != rope_theta) {                    // tables depend on theta only
+    if (capturing(st)) return ILRE_ERR_UNSUPPORTED;    // a replay would not know they are stale
     ILRE_CUDA(launch_rope_pos_tables(h->pos_lo, h->pos_hi, h->pos_hi_rows, rope_theta, st));
     ILRE_CUDA(cudaEventRecord(h->pos_ready, st));
     h->pos_theta = rope_theta;
     h->pos_stream = st;
     ++launches;
   } else if (st != h->pos_stream) {                    // built on another stream: wait for it
-    ILRE_CUDA(cudaStreamWaitEvent(st, h->pos_ready, 0));
+    ILRE_CUDA(wait_for_tables(st, h->pos_ready));
   }
   const int n_out = h->cfg.n_kv_heads * kHeadDim;
   const long long m_tiles = (n_tok + kFillTileM - 1) / kFillTileM;
@@ -720,13 +735,14 @@ int ilre_recall_rerope_keys(ilre_recall_t* h, const void* k_cache_dev, void* k_o
   // the reason to rebuild.  Rebuilding is stream-ordered before the rotation.
   if (n_rows > 0 && (h->rope_chunk != chunk_size || h->rope_theta != rope_theta ||
                      h->rope_rows < n_rows)) {
+    if (capturing(st)) return ILRE_ERR_UNSUPPORTED;    // a replay would not know the table is stale
     ILRE_CUDA(launch_rope_table(h->rope_table, static_cast<int>(n_rows), chunk_size, rope_theta, st));
     ILRE_CUDA(cudaEventRecord(h->rope_ready, st));
     h->rope_chunk = chunk_size; h->rope_theta = rope_theta; h->rope_rows = static_cast<int>(n_rows);
     h->rope_stream = st;
     ++launches;
   } else if (n_rows > 0 && st != h->rope_stream) {     // built on another stream: wait for it
-    ILRE_CUDA(cudaStreamWaitEvent(st, h->rope_ready, 0));
+    ILRE_CUDA(wait_for_tables(st, h->rope_ready));
   }
   ReropeParams rp;
   rp.k_in = static_cast<const uint4*>(k_cache_dev);
@@ -762,13 +778,14 @@ int ilre_recall_rerope_sinks(ilre_recall_t* h, const void* k_sink_dev, void* k_o
       long long want = 64;
       while (want < turns) want *= 2;
       if (want > kRopeTableRows) want = kRopeTableRows;
+      if (capturing(st)) return ILRE_ERR_UNSUPPORTED;  // a replay would not know the table is stale
       ILRE_CUDA(launch_rope_table(h->rope_table, static_cast<int>(want), chunk_size, rope_theta, st));
       ILRE_CUDA(cudaEventRecord(h->rope_ready, st));
       h->rope_chunk = chunk_size; h->rope_theta = rope_theta; h->rope_rows = static_cast<int>(want);
       h->rope_stream = st;
       ++launches;
     } else if (st != h->rope_stream) {                 // built on another stream: wait for it
-      ILRE_CUDA(cudaStreamWaitEvent(st, h->rope_ready, 0));
+      ILRE_CUDA(wait_for_tables(st, h->rope_ready));
     }
     row = h->rope_table + (turns - 1) * kRopeHalfDim;
   }

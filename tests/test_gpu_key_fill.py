@@ -129,3 +129,51 @@ def test_gather_input_ids_is_plain_indexing():
     bad = torch.tensor([0, 4999, 5000, -1], dtype=torch.int32)
     out = gather_input_ids(ids.cuda(), bad.cuda(), query[:0].cuda())
     np.testing.assert_array_equal(out.cpu().numpy(), [ids[0].item(), ids[4999].item(), -1, -1])
+
+
+def test_fill_and_re_rotation_replay_from_a_graph_on_another_stream():
+    """Once the handle holds the angle tables (built by a first call, here on the default
+    stream), the fill and the Eq. 7 re-rotation can be captured on another stream and replayed:
+    the replay writes what the direct calls write."""
+    from paper_2508_17892_b200 import IlreRecall
+    n_kv, d_model, L, chunk = 8, 256, 2500, 512
+    X = _rand((L, d_model), 31).cuda()
+    W = _rand((n_kv * 128, d_model), 32, 1.0 / 16).cuda()
+    eng = IlreRecall(max_L=L, max_q_len=8, max_budget=128)
+    direct = torch.zeros(L, n_kv, 128, dtype=torch.bfloat16, device="cuda")
+    eng.fill_keys(X, W, direct, 0)
+    eng.rerope_keys(direct, chunk)
+    torch.cuda.synchronize()
+    replayed = torch.zeros_like(direct)
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    views = [X[a:a + chunk] for a in range(0, L, chunk)]
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for i, v in enumerate(views):
+                eng.fill_keys(v, W, replayed, i * chunk, stream=side)
+            eng.rerope_keys(replayed, chunk, stream=side)
+    assert not replayed.any()                              # nothing ran during the capture
+    graph.replay()
+    torch.cuda.synchronize()
+    eng.check_status()
+    assert torch.equal(replayed, direct)
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
+    eng.close()
+    # a handle without the tables refuses to build them inside a capture (a replay could not
+    # tell that they are stale); the capture itself stays valid
+    from paper_2508_17892_b200.recall import IlreError
+    fresh = IlreRecall(max_L=L, max_q_len=8, max_budget=128)
+    graph2 = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph2, stream=side):
+            with pytest.raises(IlreError) as e1:
+                fresh.fill_keys(views[0], W, replayed, 0, stream=side)
+            with pytest.raises(IlreError) as e2:
+                fresh.rerope_keys(replayed, chunk, stream=side)
+    assert e1.value.code == -2 and e2.value.code == -2
+    torch.cuda.synchronize()
+    fresh.fill_keys(views[0], W, replayed, 0)              # the handle works as before
+    torch.cuda.synchronize()
+    fresh.check_status()
+    fresh.close()
