@@ -164,8 +164,10 @@ def test_fill_and_re_rotation_replay_from_a_graph_on_another_stream():
     # tell that they are stale); the capture itself stays valid
     from paper_2508_17892_b200.recall import IlreError
     fresh = IlreRecall(max_L=L, max_q_len=8, max_budget=128)
+    import warnings
     graph2 = torch.cuda.CUDAGraph()
-    with torch.cuda.stream(side):
+    with torch.cuda.stream(side), warnings.catch_warnings():
+        warnings.simplefilter("ignore")                    # the captured graph stays empty
         with torch.cuda.graph(graph2, stream=side):
             with pytest.raises(IlreError) as e1:
                 fresh.fill_keys(views[0], W, replayed, 0, stream=side)
