@@ -59,3 +59,34 @@ def test_random_configuration(seed):
     assert np.array_equal(idx3.numpy(), idx.cpu().numpy())
     assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
     eng.close()
+
+
+def _draw_many(seed):
+    rng = random.Random(900 + seed)
+    L = rng.choice([rng.randint(200, 3000), rng.randint(3000, 40000), rng.randint(40000, 150000)])
+    n_sink = rng.choice([0, 4, 37])
+    budget = min(rng.choice([rng.randint(48, 600), rng.randint(600, 5000), 4096]), L - n_sink - 1)
+    max_sizes = tuple(sorted(rng.sample([1, 2, 3, 4, 8, 16, 32, 64], rng.randint(2, 6))))
+    win_sizes = tuple(sorted(rng.sample([1, 2, 3, 5, 7, 9, 11, 13, 15, 31, 63], rng.randint(4, 8))))
+    return small_workload(L, rng.choice([1, 2, 4]), seed=5000 + seed, n_spans=3 if L >= 256 else 0,
+                          budget=budget, max_sizes=max_sizes, win_sizes=win_sizes,
+                          win_op=rng.randint(0, 1), n_sink=n_sink,
+                          key_kind=rng.choice(["gauss", "lowrank", "outlier"]))
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_configuration_with_many_combinations(seed):
+    """8 to 48 (max size, window size) combinations at once, as in Algorithm 1's default pooling:
+    many candidate lists of very different lengths share the grid."""
+    from paper_2508_17892_b200 import IlreRecall
+    w = _draw_many(seed)
+    x = make_inputs(w)
+    eng = IlreRecall(max_L=w.L, max_q_len=w.q_len, max_budget=max(w.budget, 1), max_combinations=48,
+                     n_kv_heads=w.n_kv_heads, n_q_heads=w.n_q_heads)
+    idx, sc = eng.run(x.K.cuda(), x.Q.cuda(), w.budget, w.max_sizes, w.win_sizes, w.win_op, w.n_sink,
+                      want_scores=True)
+    torch.cuda.synchronize()
+    eng.check_status()
+    parity.check_recall(x.K, x.Q, w, idx.cpu().numpy(), sc.cpu().numpy())
+    assert eng.check_guards() == 0, "a kernel wrote past the end of a workspace buffer"
+    eng.close()
